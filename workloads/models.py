@@ -1,0 +1,252 @@
+"""Synthetic networks shaped like the paper's workloads (Section 5, Table 2, and
+the VGGNet named in Section 3): ResNet-50 v1.5, VGG-16, MobileNet-V2.
+
+A network is plain data: an ordered list of ops over numbered tensor slots
+(slot 0 is the input image).  Both the CPU oracle's network walker and the CUDA
+library's binding consume this list; nothing here computes a layer.
+
+Gains.  With random weights, activations would vanish or explode over ~50
+layers, so each layer's folded BatchNorm scale is multiplied by a gain derived
+from summary statistics of the generated tensors (kept weight energy), and
+int8 layers get a requantization multiplier derived from the row's sum of
+squared integer weights.  These are recipes for synthetic inputs only.
+"""
+from dataclasses import dataclass, field
+from typing import List, Optional, Tuple
+import numpy as np
+
+from . import gen
+
+
+@dataclass
+class Op:
+    kind: str                      # 'conv' | 'fc' | 'maxpool' | 'gavgpool'
+    name: str
+    src: int
+    dst: int
+    res: int = -1                  # residual slot added in the epilogue, -1 = none
+    c_in: int = 0
+    c_out: int = 0
+    k: int = 1
+    stride: int = 1
+    pad: int = 0
+    groups: int = 1
+    act: str = "none"              # 'none' | 'relu' | 'relu6'
+    w: Optional[np.ndarray] = None     # f32: float32 OHWI; s8: int8 codes OHWI
+    mask: Optional[np.ndarray] = None  # uint8, same shape; None = dense
+    scale: Optional[np.ndarray] = None  # f32: folded BN scale; s8: multiplier M
+    bias: Optional[np.ndarray] = None   # f32: folded BN bias;  s8: offset B
+    out: str = "f32"               # 'f32' | 's8' | 's32'
+    density: float = 1.0
+    in_hw: Tuple[int, int] = (0, 0)
+    out_hw: Tuple[int, int] = (0, 0)
+
+    @property
+    def nnz(self):
+        if self.w is None:
+            return 0
+        return int(self.w.size if self.mask is None else int(self.mask.sum()))
+
+
+@dataclass
+class Model:
+    name: str
+    dtype: str                     # 'f32' | 's8'
+    in_shape: Tuple[int, int, int]  # (h, w, c)
+    ops: List[Op] = field(default_factory=list)
+    seed: int = 0
+    n_slots: int = 1
+
+    def new_slot(self):
+        s = self.n_slots
+        self.n_slots += 1
+        return s
+
+    def weight_ops(self):
+        return [o for o in self.ops if o.kind in ("conv", "fc")]
+
+
+def _hw_out(h, k, s, p):
+    return (h + 2 * p - k) // s + 1
+
+
+_GAMMA_RMS = np.sqrt(1.0 + 1.0 / 12.0)   # rms of U(0.5, 1.5)
+
+
+def _f32_conv(m, g, name, src, c_in, c_out, k, stride, pad, h, act, density,
+              groups=1, res=-1, gain=1.0, prune="magnitude"):
+    cg = c_in // groups
+    w = gen.he_weights(g, c_out, k, k, cg)
+    if density >= 1.0:
+        mask = None
+        kept = 1.0
+    else:
+        mask = gen.magnitude_mask(w, density) if prune == "magnitude" else gen.random_mask(g, w.shape, density)
+        kept = gen.kept_energy(w, mask)
+    # He-initialised weights double the second moment; a ReLU halves it again.
+    layer_gain = gain / (_GAMMA_RMS * np.sqrt(kept))
+    if act == "none":
+        layer_gain /= np.sqrt(2.0)
+    scale, bias = gen.folded_bn(g, c_out, gain=layer_gain)
+    dst = m.new_slot()
+    ho = _hw_out(h, k, stride, pad)
+    m.ops.append(Op("conv", name, src, dst, res, c_in, c_out, k, stride, pad, groups, act,
+                    w, mask, scale, bias, "f32", density, (h, h), (ho, ho)))
+    return dst, ho
+
+
+def _f32_fc(m, g, name, src, k_in, c_out, density):
+    w = gen.he_weights(g, c_out, 1, 1, k_in)
+    mask = None if density >= 1.0 else gen.magnitude_mask(w, density)
+    kept = 1.0 if mask is None else gen.kept_energy(w, mask)
+    scale = np.full(c_out, 1.0 / np.sqrt(2.0 * kept), np.float32)
+    bias = (g.standard_normal(c_out) * 0.1).astype(np.float32)
+    dst = m.new_slot()
+    m.ops.append(Op("fc", name, src, dst, -1, k_in, c_out, 1, 1, 0, 1, "none",
+                    w, mask, scale, bias, "f32", density, (1, 1), (1, 1)))
+    return dst
+
+
+def single_layer(seed=1, c_in=64, c_out=64, hw=56, k=3, stride=1, pad=1, density=0.10):
+    """One 3x3 conv layer: N(0, 0.05^2) weights, exactly-k uniform random mask,
+    max(0, N(0,1)) input, no bias, ReLU."""
+    g = gen.rng(seed)
+    m = Model("single_conv", "f32", (hw, hw, c_in), seed=seed)
+    w = gen.normal_weights(g, (c_out, k, k, c_in), 0.05)
+    mask = None if density >= 1.0 else gen.random_mask(g, w.shape, density)
+    ho = _hw_out(hw, k, stride, pad)
+    m.ops.append(Op("conv", "conv", 0, m.new_slot(), -1, c_in, c_out, k, stride, pad, 1, "relu",
+                    w, mask, None, None, "f32", density, (hw, hw), (ho, ho)))
+    return m
+
+
+def resnet50(seed=2, density=0.125, fc_density=0.10, width=1.0, image=224, classes=1000):
+    """ResNet-50 v1.5: stride 2 sits on the 3x3 conv of the first block of stages
+    3 to 5.  The 7x7 stem stays dense; every other conv is magnitude-pruned per
+    layer to `density`; the classifier to `fc_density`."""
+    g = gen.rng(seed)
+    m = Model("resnet50", "f32", (image, image, 3), seed=seed)
+    ch = lambda c: max(8, int(round(c * width)))
+    cur, h = _f32_conv(m, g, "conv1", 0, 3, ch(64), 7, 2, 3, image, "relu", 1.0)
+    dst = m.new_slot()
+    ho = _hw_out(h, 3, 2, 1)
+    m.ops.append(Op("maxpool", "pool1", cur, dst, k=3, stride=2, pad=1, c_in=ch(64), c_out=ch(64),
+                    in_hw=(h, h), out_hw=(ho, ho)))
+    cur, h, c_in = dst, ho, ch(64)
+    for si, (mid, blocks, stride) in enumerate([(64, 3, 1), (128, 4, 2), (256, 6, 2), (512, 3, 2)]):
+        mid = ch(mid)
+        out = mid * 4
+        for b in range(blocks):
+            s = stride if b == 0 else 1
+            nm = "s%db%d" % (si + 2, b)
+            if b == 0:
+                short, _ = _f32_conv(m, g, nm + ".ds", cur, c_in, out, 1, s, 0, h, "none", density)
+            else:
+                short = cur
+            t, _ = _f32_conv(m, g, nm + ".c1", cur, c_in, mid, 1, 1, 0, h, "relu", density)
+            t, h2 = _f32_conv(m, g, nm + ".c2", t, mid, mid, 3, s, 1, h, "relu", density)
+            cur, _ = _f32_conv(m, g, nm + ".c3", t, mid, out, 1, 1, 0, h2, "relu", density,
+                               res=short, gain=0.4)
+            h, c_in = h2, out
+    dst = m.new_slot()
+    m.ops.append(Op("gavgpool", "avgpool", cur, dst, c_in=c_in, c_out=c_in, in_hw=(h, h), out_hw=(1, 1)))
+    _f32_fc(m, g, "fc", dst, c_in, classes, fc_density)
+    return m
+
+
+def mobilenet_v2(seed=4, density=0.25, width=1.0, image=224, classes=1000):
+    """MobileNet-V2 (width 1.0): stem 3x3 s2 and all depthwise 3x3 dense; pointwise
+    1x1 convs, the 1x1 head and the classifier magnitude-pruned to `density`.
+    ReLU6 after expand and depthwise, no activation after project."""
+    g = gen.rng(seed)
+    m = Model("mobilenet_v2", "f32", (image, image, 3), seed=seed)
+    ch = lambda c: max(8, int(round(c * width / 8.0)) * 8)
+    c_in = ch(32)
+    cur, h = _f32_conv(m, g, "stem", 0, 3, c_in, 3, 2, 1, image, "relu6", 1.0)
+    cfg = [(1, 16, 1, 1), (6, 24, 2, 2), (6, 32, 3, 2), (6, 64, 4, 2), (6, 96, 3, 1), (6, 160, 3, 2), (6, 320, 1, 1)]
+    for t, c, n, s in cfg:
+        c = ch(c)
+        for b in range(n):
+            st = s if b == 0 else 1
+            nm = "ir%d_%d" % (c, b)
+            hid = c_in * t
+            x_in = cur
+            tcur = cur
+            if t != 1:
+                tcur, _ = _f32_conv(m, g, nm + ".expand", tcur, c_in, hid, 1, 1, 0, h, "relu6", density)
+            tcur, h2 = _f32_conv(m, g, nm + ".dw", tcur, hid, hid, 3, st, 1, h, "relu6", 1.0, groups=hid)
+            use_res = (st == 1 and c_in == c)
+            cur, _ = _f32_conv(m, g, nm + ".project", tcur, hid, c, 1, 1, 0, h2, "none", density,
+                               res=x_in if use_res else -1, gain=0.7 if use_res else 1.0)
+            h, c_in = h2, c
+    head = ch(1280)
+    cur, _ = _f32_conv(m, g, "head", cur, c_in, head, 1, 1, 0, h, "relu6", density)
+    dst = m.new_slot()
+    m.ops.append(Op("gavgpool", "avgpool", cur, dst, c_in=head, c_out=head, in_hw=(h, h), out_hw=(1, 1)))
+    _f32_fc(m, g, "fc", dst, head, classes, density)
+    return m
+
+
+# Target rms of the requantized pre-activation, and the input second moments the
+# multiplier recipe assumes (image codes; post-ReLU codes; post-ReLU codes after a
+# 2x2 max pool).  Synthetic-input recipe only.
+_T_RMS = 127.0 / 3.0
+_M2_IMAGE = _T_RMS ** 2
+_M2_RELU = 0.5 * _T_RMS ** 2
+_M2_POOLED = 1.3 * _T_RMS ** 2
+
+
+def _s8_layer(m, g, kind, name, src, c_in, c_out, k, pad, h, act, density, m2_in, out="s8"):
+    shape = (c_out, k, k, c_in)
+    q = gen.int8_weights(g, shape)
+    mask = None if density >= 1.0 else gen.random_mask(g, shape, density)
+    qq = q.astype(np.float64) ** 2
+    if mask is not None:
+        qq = qq * mask
+    row_energy = qq.reshape(c_out, -1).sum(axis=1)
+    mult = np.where(row_energy > 0, _T_RMS / np.sqrt(np.maximum(row_energy, 1.0) * m2_in), 1.0)
+    mult = (mult * g.uniform(0.8, 1.25, size=c_out)).astype(np.float32)
+    offs = (g.standard_normal(c_out) * 0.1 * _T_RMS).astype(np.float32)
+    dst = m.new_slot()
+    ho = _hw_out(h, k, 1, pad)
+    m.ops.append(Op(kind, name, src, dst, -1, c_in, c_out, k, 1, pad, 1, act, q, mask,
+                    mult, offs, out, density, (h, h), (ho, ho)))
+    return dst
+
+
+def vgg16(seed=3, density=0.08, fc_density=0.04, width=1.0, image=224, classes=1000, fc_width=4096):
+    """VGG-16 with int8 weights and activations: 13 convs at `density`, 3 FC layers
+    at `fc_density`, exactly-k uniform random masks, five int8 2x2 max pools.
+    The last layer returns fmaf(acc, M, B) as float32 without rounding."""
+    g = gen.rng(seed)
+    m = Model("vgg16", "s8", (image, image, 3), seed=seed)
+    cfg = [64, 64, "M", 128, 128, "M", 256, 256, 256, "M", 512, 512, 512, "M", 512, 512, 512, "M"]
+    cur, h, c_in, i = 0, image, 3, 0
+    m2 = _M2_IMAGE
+    for c in cfg:
+        if c == "M":
+            dst = m.new_slot()
+            m.ops.append(Op("maxpool", "pool%d" % i, cur, dst, k=2, stride=2, pad=0, c_in=c_in, c_out=c_in,
+                            in_hw=(h, h), out_hw=(h // 2, h // 2), out="s8"))
+            cur, h, m2 = dst, h // 2, _M2_POOLED
+            continue
+        i += 1
+        c = max(8, int(round(c * width)))
+        cur = _s8_layer(m, g, "conv", "conv%d" % i, cur, c_in, c, 3, 1, h, "relu", density, m2)
+        c_in, m2 = c, _M2_RELU
+    # FC input is the NHWC flatten (h, w, c order) of the last feature map.
+    k_in = h * h * c_in
+    cur = _s8_layer(m, g, "fc", "fc6", cur, k_in, fc_width, 1, 0, 1, "relu", fc_density, _M2_POOLED)
+    cur = _s8_layer(m, g, "fc", "fc7", cur, fc_width, fc_width, 1, 0, 1, "relu", fc_density, _M2_RELU)
+    _s8_layer(m, g, "fc", "fc8", cur, fc_width, classes, 1, 0, 1, "none", fc_density, _M2_RELU, out="f32")
+    return m
+
+
+def make_input(model, batch=1, seed=None):
+    g = gen.rng(model.seed * 1000003 + 17 if seed is None else seed)
+    h, w, c = model.in_shape
+    if model.dtype == "s8":
+        return gen.int8_image(g, (batch, h, w, c))
+    if model.name == "single_conv":
+        return gen.relu_normal_input(g, (batch, h, w, c))
+    return gen.normal_input(g, (batch, h, w, c))
