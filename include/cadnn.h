@@ -1,0 +1,243 @@
+/*
+ * cadnn.h - C ABI of the sparse-CNN inference library (CUDA, sm_100a).
+ *
+ * The library runs forward inference of weight-pruned, optionally int8
+ * weight-quantized convolutional networks: every conv / FC layer multiplies a
+ * fixed, compressed sparse weight tensor by dense activations.  It restates, for
+ * one datacenter GPU, the execution stage of CADNN (arXiv 1905.00571, Section 4
+ * "Architecture-aware Optimization"): compressed weight storage with an offline
+ * layout transformation, fused Conv + BatchNorm + Activation kernels, 1x1
+ * convolutions run as a sparse-matrix product, and a per-layer choice of tiling
+ * parameters made once per model.
+ *
+ * Conventions
+ *  - Activations are NHWC, contiguous.  Dense weights handed to the packer are
+ *    OHWI: [c_out][kh][kw][c_in/groups].
+ *  - Every call returns a cadnn_status; nothing aborts or throws across the ABI.
+ *    Output pointers are written only when CADNN_OK is returned.
+ *  - "host" / "device" on each pointer says where the memory must live.  The
+ *    caller owns every buffer it passes; a cadnn_weights / cadnn_net handle owns
+ *    the device memory it allocated and releases it in its *_free call.
+ *  - Kernels are launched asynchronously on the stream given (a cudaStream_t
+ *    passed as void*, NULL = the default stream).  No call synchronizes the
+ *    device unless its comment says so.
+ *  - Inputs must be finite; NaN / Inf behaviour is unspecified (a pruned weight
+ *    contributes exactly 0 only for finite activations).
+ *  - There is no CPU fallback: without a CUDA device every compute call fails
+ *    with CADNN_E_CUDA.
+ */
+#ifndef CADNN_H
+#define CADNN_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CADNN_OK = 0,
+    CADNN_E_ARG = 1,          /* NULL or inconsistent argument */
+    CADNN_E_SHAPE = 2,        /* shape differs from what the handle was packed for, or is invalid */
+    CADNN_E_DTYPE = 3,        /* dtype combination not defined */
+    CADNN_E_UNSUPPORTED = 4,  /* valid request the library does not implement */
+    CADNN_E_ALLOC = 5,        /* host or device allocation failed */
+    CADNN_E_CUDA = 6,         /* a CUDA runtime call failed (cadnn_last_cuda_error) */
+    CADNN_E_DEVICE_STATUS = 7 /* a kernel recorded an error in the device status word */
+} cadnn_status;
+
+typedef enum { CADNN_F32 = 0, CADNN_S8 = 1, CADNN_S32 = 2 } cadnn_dtype;
+typedef enum { CADNN_ACT_NONE = 0, CADNN_ACT_RELU = 1, CADNN_ACT_RELU6 = 2 } cadnn_act;
+
+/* Storage format of a packed layer (reported by cadnn_weights_info). */
+typedef enum {
+    CADNN_FMT_AUTO = 0,        /* let the packer choose (the only value cadnn_pack needs) */
+    CADNN_FMT_TILED_CSR = 1,   /* conv: per channel-chunk CSR by output channel, filters regrouped */
+    CADNN_FMT_ROW_CSR = 2,     /* fc at small batch: CSR by output channel, rows sorted by length */
+    CADNN_FMT_DENSE_DW = 3,    /* dense depthwise filters, tap-major */
+    CADNN_FMT_DENSE_SMALLC = 4 /* dense conv with very few input channels (network stem) */
+} cadnn_fmt;
+
+#define CADNN_PACK_HOST_ONLY 1 /* build the packed image on the host only (no device needed, no compute) */
+
+/*
+ * One layer.  The packer is the offline stage of Section 4 ("Memory layout
+ * transformation", "Optimization parameters selection"): tile sizes and the
+ * filter regrouping depend on the layer's spatial size, so the input size the
+ * layer will run at is part of its description.
+ *   conv: c_in, c_out, kh, kw, stride, pad, groups (1, or c_in == c_out for depthwise),
+ *         in_h, in_w.
+ *   fc:   kh = kw = 1, stride = 1, pad = 0, groups = 1, in_h = in_w = 1, c_in = K.
+ *   batch_hint: batch size the schedule is tuned for (>= 1); any batch still runs.
+ */
+typedef struct {
+    int c_in, c_out, kh, kw, stride, pad, groups;
+    int in_h, in_w;
+    int batch_hint;
+    int dtype; /* cadnn_dtype of weights and activations: CADNN_F32 or CADNN_S8 */
+    int fmt;   /* cadnn_fmt, CADNN_FMT_AUTO */
+    int flags; /* CADNN_PACK_HOST_ONLY or 0 */
+} cadnn_layer_desc;
+
+typedef struct cadnn_weights cadnn_weights;
+typedef struct cadnn_net cadnn_net;
+
+/*
+ * cadnn_pack - compress one layer (Section 4, "Memory layout transformation and
+ * load optimization"; load balance is the obstacle Section 1 names).
+ *   w_ohwi  host, float [c_out][kh][kw][c_in/groups].
+ *   mask    host, uint8 same shape, nonzero = kept; NULL = every weight kept.
+ *           The stored set is exactly the kept positions, even where the value is 0.
+ *   w_scale host, float [c_out], required for CADNN_S8 (q = clamp(rne(w / w_scale[co]),
+ *           -127, 127)); must be NULL for CADNN_F32.
+ *   out     receives a handle owning its buffers (device buffers on the current
+ *           device unless CADNN_PACK_HOST_ONLY).  Immutable afterwards; may be used
+ *           from several streams.
+ * Filters are regrouped so that the warps of a thread block get equal nonzero
+ * counts; the permutation is undone when results are stored.
+ * Errors: E_ARG (NULL, bad desc), E_DTYPE, E_UNSUPPORTED (grouped conv other than
+ * depthwise; int8 depthwise; reduction length whose int32 sum could overflow),
+ * E_ALLOC, E_CUDA.  Synchronizes the device copy before returning.
+ */
+cadnn_status cadnn_pack(const cadnn_layer_desc *desc, const float *w_ohwi, const uint8_t *mask,
+                        const float *w_scale, cadnn_weights **out);
+
+/* Same for weights that are already int8 codes (desc->dtype must be CADNN_S8). */
+cadnn_status cadnn_pack_q8(const cadnn_layer_desc *desc, const int8_t *q_ohwi, const uint8_t *mask,
+                           cadnn_weights **out);
+
+/* nnz = kept positions; packed_bytes = bytes of the device image; fmt = cadnn_fmt used.
+ * Any output pointer may be NULL. */
+cadnn_status cadnn_weights_info(const cadnn_weights *w, int64_t *nnz, int64_t *packed_bytes, int *fmt);
+
+/*
+ * Schedule the packer chose (Section 4, "Optimization parameters selection"):
+ * sched[0..7] = kernel kind, pixels per lane, filters per warp, filters per block,
+ * channel chunk, tile rows, tile columns, shared-memory row pitch.  Host ints.
+ */
+cadnn_status cadnn_weights_schedule(const cadnn_weights *w, int sched[8]);
+
+/*
+ * Per-warp load of the packed image: for every (filter block, warp) the number of
+ * stored nonzeros that warp walks.  n_out receives the count; loads (host, may be
+ * NULL) receives up to cap entries.
+ */
+cadnn_status cadnn_weights_warp_loads(const cadnn_weights *w, int64_t *loads, int cap, int *n_out);
+
+/* Expand the packed image back to dense OHWI (masked-out = 0) and the mask.  Host
+ * pointers; dense_f32 receives floats (int8 layers: the integer codes as floats);
+ * either may be NULL. */
+cadnn_status cadnn_weights_unpack(const cadnn_weights *w, float *dense_f32, uint8_t *mask);
+
+void cadnn_weights_free(cadnn_weights *w);
+
+/*
+ * Fused epilogue (Section 4, "Model computation fusion": Conv/DWConv + BatchNorm +
+ * Activation in one kernel; the residual add of a bottleneck block joins it).
+ * Float layers:  z = acc * scale[co] + bias[co];  z += residual;  z = act(z).
+ * Int8 layers:   t = fmaf((float)acc, scale[co], bias[co])  (one fused multiply-add,
+ *                scale = s_x * s_w[co] / s_y, bias = b[co] / s_y, both precomputed by
+ *                the caller); ReLU; out_dtype S8: clamp to [-127,127], round half even;
+ *                F32: t as is; S32: the raw accumulator (scale / bias / act ignored).
+ *                residual must be NULL and ReLU6 is not defined.
+ * scale, bias: device float [c_out], NULL = 1 / 0.  residual: device, same shape and
+ * dtype as y, or NULL.
+ */
+typedef struct {
+    const float *scale;
+    const float *bias;
+    const void *residual;
+    int act;       /* cadnn_act */
+    int out_dtype; /* cadnn_dtype of y */
+} cadnn_epilogue;
+
+/*
+ * cadnn_conv2d - one sparse convolution layer (Section 4: compressed-model layer
+ * execution; 1x1 filters run as a sparse-matrix product).
+ *   x device NHWC [n][h][w][c_in], h and w must equal the packed in_h, in_w.
+ *   y device NHWC [n][h_out][w_out][c_out], h_out = (h + 2 pad - kh) / stride + 1.
+ *   y must not alias x.  Pointers must be 16-byte aligned.  ep may be NULL
+ *   (no scale, bias, residual or activation; output dtype = layer dtype).
+ * Errors: E_ARG, E_SHAPE, E_DTYPE, E_CUDA (launch failure).
+ */
+cadnn_status cadnn_conv2d(const cadnn_weights *w, const void *x, int n, int h, int wd, void *y,
+                          const cadnn_epilogue *ep, void *stream);
+
+/*
+ * cadnn_fc - one sparse fully connected layer: y[b][co] = sum_k W[co][k] x[b][k],
+ * same epilogue.  x device [n][k], y device [n][c_out].
+ */
+cadnn_status cadnn_fc(const cadnn_weights *w, const void *x, int n, void *y,
+                      const cadnn_epilogue *ep, void *stream);
+
+/* Glue layers the evaluated networks need (not discussed by the paper).
+ * Max pool ignores padded taps; dtype CADNN_F32 or CADNN_S8. */
+cadnn_status cadnn_maxpool2d(const void *x, int n, int h, int wd, int c, int k, int stride, int pad,
+                             int dtype, void *y, void *stream);
+/* Global average pool, float: y[b][c] = mean over h*w. */
+cadnn_status cadnn_global_avgpool(const float *x, int n, int h, int wd, int c, float *y, void *stream);
+
+/* Whole network (Section 5: single-image inference of a complete model). */
+typedef enum { CADNN_OP_CONV = 0, CADNN_OP_FC = 1, CADNN_OP_MAXPOOL = 2, CADNN_OP_GAVGPOOL = 3 } cadnn_op_kind;
+
+typedef struct {
+    int kind;                 /* cadnn_op_kind */
+    const cadnn_weights *w;   /* conv / fc; borrowed, must outlive the net */
+    int src, dst, res;        /* tensor slots; slot 0 is the network input; res = -1 for none */
+    const float *scale;       /* device [c_out] or NULL; borrowed */
+    const float *bias;        /* device [c_out] or NULL; borrowed */
+    int act;                  /* cadnn_act */
+    int out_dtype;            /* cadnn_dtype of the dst slot */
+    int pool_k, pool_stride, pool_pad; /* max pool only */
+} cadnn_op;
+
+/*
+ * cadnn_net_create - shape-check an op list for input [n][h][w][c] of dtype in_dtype
+ * and allocate one device buffer per intermediate slot (owned by the net).  The dst
+ * slot of the last op is the network output and is written straight to the pointer
+ * given to cadnn_forward.  Every slot is written by exactly one op, after which it is
+ * only read.
+ */
+cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int wd, int c, int in_dtype,
+                              cadnn_net **out);
+
+/*
+ * cadnn_forward - run the network: x device input, y device output of the last op.
+ * use_graph != 0 replays a CUDA graph captured on the first call with this (x, y)
+ * pair (re-captured when either pointer changes); 0 launches the layers one by one.
+ * Asynchronous on stream.
+ */
+cadnn_status cadnn_forward(cadnn_net *net, const void *x, void *y, int use_graph, void *stream);
+
+/*
+ * cadnn_forward_host - the same network run from HOST buffers: copies x_host
+ * ([n][h][w][c], pinned memory recommended) to a device staging buffer the net owns
+ * (allocated on the first call), runs the network, copies the output to y_host and
+ * synchronizes stream before returning.
+ */
+cadnn_status cadnn_forward_host(cadnn_net *net, const void *x_host, void *y_host, int use_graph, void *stream);
+
+/* Number of kernel launches one forward issues; bytes of slot memory the net owns. */
+cadnn_status cadnn_net_info(const cadnn_net *net, int *n_launches, int64_t *workspace_bytes);
+
+/*
+ * Measurement aid: run the network once layer by layer on stream with a CUDA event
+ * pair around every op, synchronize, and write the per-op milliseconds to ms[n_ops]
+ * (host).  flush_l2 != 0 overwrites a buffer larger than L2 before each op.
+ */
+cadnn_status cadnn_net_layer_times(cadnn_net *net, const void *x, void *y, int flush_l2, float *ms,
+                                   void *stream);
+
+/* Device pointer and byte size of slot `slot` (for per-layer inspection). */
+cadnn_status cadnn_net_slot(const cadnn_net *net, int slot, void **ptr, int64_t *bytes);
+
+void cadnn_net_free(cadnn_net *net);
+
+const char *cadnn_status_str(cadnn_status s);
+/* Text of the last CUDA error this thread saw inside the library ("" if none). */
+const char *cadnn_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CADNN_H */

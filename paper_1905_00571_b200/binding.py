@@ -1,0 +1,286 @@
+"""Thin ctypes binding of the C ABI declared in include/cadnn.h.
+
+Same names as the C entry points; argument marshalling only - every step of a
+layer or network runs inside the CUDA library.  torch supplies device memory
+and streams.  Importing this module fails if the library has not been built:
+there is no fallback path.
+"""
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcadnn.so")
+if not os.path.exists(LIB_PATH):
+    raise ImportError("libcadnn.so is missing: run `python -m paper_1905_00571_b200.build` "
+                      "(or __graft_entry__.build()) first; there is no fallback implementation")
+_lib = ctypes.CDLL(LIB_PATH)
+
+OK = 0
+F32, S8, S32 = 0, 1, 2
+DTYPE = {"f32": F32, "s8": S8, "s32": S32}
+ACT = {"none": 0, "relu": 1, "relu6": 2, None: 0}
+PACK_HOST_ONLY = 1
+OP_CONV, OP_FC, OP_MAXPOOL, OP_GAVGPOOL = 0, 1, 2, 3
+FMT_NAMES = {1: "tiled_csr", 2: "row_csr", 3: "dense_dw", 4: "dense_smallc"}
+KIND_NAMES = {1: "sconv_spatial", 2: "sconv_linear", 3: "fc_spmv", 4: "dw", 5: "dense_smallc"}
+
+
+class LayerDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in
+                ("c_in", "c_out", "kh", "kw", "stride", "pad", "groups", "in_h", "in_w",
+                 "batch_hint", "dtype", "fmt", "flags")]
+
+
+class Epilogue(ctypes.Structure):
+    _fields_ = [("scale", ctypes.c_void_p), ("bias", ctypes.c_void_p), ("residual", ctypes.c_void_p),
+                ("act", ctypes.c_int), ("out_dtype", ctypes.c_int)]
+
+
+class Op(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int), ("w", ctypes.c_void_p), ("src", ctypes.c_int), ("dst", ctypes.c_int),
+                ("res", ctypes.c_int), ("scale", ctypes.c_void_p), ("bias", ctypes.c_void_p),
+                ("act", ctypes.c_int), ("out_dtype", ctypes.c_int), ("pool_k", ctypes.c_int),
+                ("pool_stride", ctypes.c_int), ("pool_pad", ctypes.c_int)]
+
+
+_vp, _i, _i64p = ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_int64)
+_SIGS = {
+    "cadnn_pack": (_i, [ctypes.POINTER(LayerDesc), _vp, _vp, _vp, ctypes.POINTER(_vp)]),
+    "cadnn_pack_q8": (_i, [ctypes.POINTER(LayerDesc), _vp, _vp, ctypes.POINTER(_vp)]),
+    "cadnn_weights_info": (_i, [_vp, _i64p, _i64p, ctypes.POINTER(_i)]),
+    "cadnn_weights_schedule": (_i, [_vp, ctypes.POINTER(_i)]),
+    "cadnn_weights_warp_loads": (_i, [_vp, _i64p, _i, ctypes.POINTER(_i)]),
+    "cadnn_weights_unpack": (_i, [_vp, _vp, _vp]),
+    "cadnn_weights_free": (None, [_vp]),
+    "cadnn_conv2d": (_i, [_vp, _vp, _i, _i, _i, _vp, ctypes.POINTER(Epilogue), _vp]),
+    "cadnn_fc": (_i, [_vp, _vp, _i, _vp, ctypes.POINTER(Epilogue), _vp]),
+    "cadnn_maxpool2d": (_i, [_vp, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _vp]),
+    "cadnn_global_avgpool": (_i, [_vp, _i, _i, _i, _i, _vp, _vp]),
+    "cadnn_net_create": (_i, [ctypes.POINTER(Op), _i, _i, _i, _i, _i, _i, ctypes.POINTER(_vp)]),
+    "cadnn_forward": (_i, [_vp, _vp, _vp, _i, _vp]),
+    "cadnn_forward_host": (_i, [_vp, _vp, _vp, _i, _vp]),
+    "cadnn_net_info": (_i, [_vp, ctypes.POINTER(_i), _i64p]),
+    "cadnn_net_layer_times": (_i, [_vp, _vp, _vp, _i, ctypes.POINTER(ctypes.c_float), _vp]),
+    "cadnn_net_slot": (_i, [_vp, _i, ctypes.POINTER(_vp), _i64p]),
+    "cadnn_net_free": (None, [_vp]),
+    "cadnn_status_str": (ctypes.c_char_p, [_i]),
+    "cadnn_last_cuda_error": (ctypes.c_char_p, []),
+}
+for _name, (_res, _args) in _SIGS.items():
+    _fn = getattr(_lib, _name)
+    _fn.restype = _res
+    _fn.argtypes = _args
+
+EXPORTED = tuple(_SIGS)
+
+
+class CadnnError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        msg = "%s: %s" % (where, _lib.cadnn_status_str(status).decode())
+        if status == 6:
+            msg += " (%s)" % _lib.cadnn_last_cuda_error().decode()
+        super().__init__(msg)
+
+
+def _check(st, where):
+    if st != OK:
+        raise CadnnError(st, where)
+
+
+def _np_ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _dev_ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    if hasattr(stream, "cuda_stream"):
+        return ctypes.c_void_p(stream.cuda_stream)
+    return ctypes.c_void_p(int(stream))
+
+
+class Weights:
+    """Owner of a cadnn_weights handle."""
+
+    def __init__(self, handle, desc):
+        self.handle = handle
+        self.desc = desc
+
+    def free(self):
+        if self.handle:
+            _lib.cadnn_weights_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def make_desc(c_in, c_out, kh=1, kw=1, stride=1, pad=0, groups=1, in_h=1, in_w=1, batch_hint=1,
+              dtype="f32", host_only=False):
+    return LayerDesc(c_in, c_out, kh, kw, stride, pad, groups, in_h, in_w, batch_hint,
+                     DTYPE[dtype], 0, PACK_HOST_ONLY if host_only else 0)
+
+
+def cadnn_pack(desc, w_ohwi, mask=None, w_scale=None):
+    w = np.ascontiguousarray(w_ohwi, dtype=np.float32)
+    m = None if mask is None else np.ascontiguousarray(mask, dtype=np.uint8)
+    s = None if w_scale is None else np.ascontiguousarray(w_scale, dtype=np.float32)
+    expect = desc.c_out * desc.kh * desc.kw * (desc.c_in // max(1, desc.groups))
+    if w.size != expect or (m is not None and m.size != expect) or (s is not None and s.size != desc.c_out):
+        raise ValueError("weight / mask / scale size does not match the layer description")
+    out = ctypes.c_void_p()
+    _check(_lib.cadnn_pack(ctypes.byref(desc), _np_ptr(w), _np_ptr(m), _np_ptr(s), ctypes.byref(out)), "cadnn_pack")
+    return Weights(out, desc)
+
+
+def cadnn_pack_q8(desc, q_ohwi, mask=None):
+    q = np.ascontiguousarray(q_ohwi, dtype=np.int8)
+    m = None if mask is None else np.ascontiguousarray(mask, dtype=np.uint8)
+    expect = desc.c_out * desc.kh * desc.kw * (desc.c_in // max(1, desc.groups))
+    if q.size != expect or (m is not None and m.size != expect):
+        raise ValueError("weight / mask size does not match the layer description")
+    out = ctypes.c_void_p()
+    _check(_lib.cadnn_pack_q8(ctypes.byref(desc), _np_ptr(q), _np_ptr(m), ctypes.byref(out)), "cadnn_pack_q8")
+    return Weights(out, desc)
+
+
+def cadnn_weights_info(w):
+    nnz, pb, fmt = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int()
+    _check(_lib.cadnn_weights_info(w.handle, ctypes.byref(nnz), ctypes.byref(pb), ctypes.byref(fmt)), "cadnn_weights_info")
+    return {"nnz": nnz.value, "packed_bytes": pb.value, "fmt": fmt.value}
+
+
+def cadnn_weights_schedule(w):
+    arr = (ctypes.c_int * 8)()
+    _check(_lib.cadnn_weights_schedule(w.handle, arr), "cadnn_weights_schedule")
+    keys = ("kind", "T", "RPW", "G", "CIc", "TH", "TW", "pitch")
+    return dict(zip(keys, list(arr)))
+
+
+def cadnn_weights_warp_loads(w):
+    n = ctypes.c_int()
+    _check(_lib.cadnn_weights_warp_loads(w.handle, None, 0, ctypes.byref(n)), "cadnn_weights_warp_loads")
+    buf = (ctypes.c_int64 * max(1, n.value))()
+    _check(_lib.cadnn_weights_warp_loads(w.handle, buf, n.value, ctypes.byref(n)), "cadnn_weights_warp_loads")
+    return np.array(buf[: n.value], dtype=np.int64)
+
+
+def cadnn_weights_unpack(w):
+    d = w.desc
+    shape = (d.c_out, d.kh, d.kw, d.c_in // max(1, d.groups))
+    dense = np.empty(shape, np.float32)
+    mask = np.empty(shape, np.uint8)
+    _check(_lib.cadnn_weights_unpack(w.handle, _np_ptr(dense), _np_ptr(mask)), "cadnn_weights_unpack")
+    return dense, mask
+
+
+def _epilogue(scale, bias, residual, act, out_dtype):
+    return Epilogue(None if scale is None else scale.data_ptr(), None if bias is None else bias.data_ptr(),
+                    None if residual is None else residual.data_ptr(), ACT[act] if not isinstance(act, int) else act,
+                    DTYPE[out_dtype] if not isinstance(out_dtype, int) else out_dtype)
+
+
+def cadnn_conv2d(w, x, y, scale=None, bias=None, residual=None, act="none", out_dtype=None, stream=None):
+    """x, y: torch CUDA tensors, NHWC contiguous; y is written in place."""
+    n, h, wd = int(x.shape[0]), int(x.shape[1]), int(x.shape[2])
+    if out_dtype is None:
+        out_dtype = w.desc.dtype
+    ep = _epilogue(scale, bias, residual, act, out_dtype)
+    _check(_lib.cadnn_conv2d(w.handle, _dev_ptr(x), n, h, wd, _dev_ptr(y), ctypes.byref(ep), _stream(stream)),
+           "cadnn_conv2d")
+    return y
+
+
+def cadnn_fc(w, x, y, scale=None, bias=None, residual=None, act="none", out_dtype=None, stream=None):
+    if out_dtype is None:
+        out_dtype = w.desc.dtype
+    ep = _epilogue(scale, bias, residual, act, out_dtype)
+    _check(_lib.cadnn_fc(w.handle, _dev_ptr(x), int(x.shape[0]), _dev_ptr(y), ctypes.byref(ep), _stream(stream)),
+           "cadnn_fc")
+    return y
+
+
+def cadnn_maxpool2d(x, y, k, stride, pad=0, stream=None):
+    import torch
+    n, h, wd, c = (int(v) for v in x.shape)
+    dt = S8 if x.dtype == torch.int8 else F32
+    _check(_lib.cadnn_maxpool2d(_dev_ptr(x), n, h, wd, c, k, stride, pad, dt, _dev_ptr(y), _stream(stream)),
+           "cadnn_maxpool2d")
+    return y
+
+
+def cadnn_global_avgpool(x, y, stream=None):
+    n, h, wd, c = (int(v) for v in x.shape)
+    _check(_lib.cadnn_global_avgpool(_dev_ptr(x), n, h, wd, c, _dev_ptr(y), _stream(stream)), "cadnn_global_avgpool")
+    return y
+
+
+class Net:
+    def __init__(self, handle, keep):
+        self.handle = handle
+        self._keep = keep   # objects the C side borrows (weights, scale / bias tensors)
+
+    def free(self):
+        if self.handle:
+            _lib.cadnn_net_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def cadnn_net_create(ops, n, h, w, c, in_dtype, keep=None):
+    """ops: list of binding.Op."""
+    arr = (Op * len(ops))(*ops)
+    out = ctypes.c_void_p()
+    _check(_lib.cadnn_net_create(arr, len(ops), n, h, w, c, DTYPE[in_dtype] if not isinstance(in_dtype, int) else in_dtype,
+                                 ctypes.byref(out)), "cadnn_net_create")
+    return Net(out, keep)
+
+
+def cadnn_forward(net, x, y, use_graph=True, stream=None):
+    _check(_lib.cadnn_forward(net.handle, _dev_ptr(x), _dev_ptr(y), 1 if use_graph else 0, _stream(stream)),
+           "cadnn_forward")
+    return y
+
+
+def cadnn_forward_host(net, x_host, y_host, use_graph=True, stream=None):
+    """x_host, y_host: CPU torch tensors (pinned recommended) or numpy arrays; blocks until y_host is filled."""
+    xp = x_host.data_ptr() if hasattr(x_host, "data_ptr") else x_host.ctypes.data
+    yp = y_host.data_ptr() if hasattr(y_host, "data_ptr") else y_host.ctypes.data
+    _check(_lib.cadnn_forward_host(net.handle, ctypes.c_void_p(xp), ctypes.c_void_p(yp), 1 if use_graph else 0,
+                                   _stream(stream)), "cadnn_forward_host")
+    return y_host
+
+
+def cadnn_net_info(net):
+    nl, ws = ctypes.c_int(), ctypes.c_int64()
+    _check(_lib.cadnn_net_info(net.handle, ctypes.byref(nl), ctypes.byref(ws)), "cadnn_net_info")
+    return {"launches": nl.value, "workspace_bytes": ws.value}
+
+
+def cadnn_net_layer_times(net, x, y, n_ops, flush_l2=False, stream=None):
+    ms = (ctypes.c_float * n_ops)()
+    _check(_lib.cadnn_net_layer_times(net.handle, _dev_ptr(x), _dev_ptr(y), 1 if flush_l2 else 0, ms, _stream(stream)),
+           "cadnn_net_layer_times")
+    return [float(v) for v in ms]
+
+
+def cadnn_net_slot(net, slot):
+    ptr, b = ctypes.c_void_p(), ctypes.c_int64()
+    _check(_lib.cadnn_net_slot(net.handle, slot, ctypes.byref(ptr), ctypes.byref(b)), "cadnn_net_slot")
+    return ptr.value, b.value

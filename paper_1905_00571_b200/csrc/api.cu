@@ -1,0 +1,109 @@
+// C-ABI entry points for single layers: argument checks and dispatch to the
+// kernel the packer scheduled.  No arithmetic lives here.
+#include <cstdio>
+#include <cstring>
+#include "cadnn_internal.h"
+
+namespace {
+thread_local char g_cuda_err[256] = "";
+}
+
+cadnn_status cadnn_note_cuda(cudaError_t e)
+{
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+    cudaGetLastError();  // clear a non-sticky error so that later calls are not blamed for it
+    return CADNN_E_CUDA;
+}
+
+namespace {
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+cadnn_status check_epilogue(const cadnn_weights *w, const cadnn_epilogue *ep, LaunchEpilogue &le)
+{
+    const int dt = w->desc.dtype;
+    le = LaunchEpilogue();
+    le.out_dtype = dt;
+    if (!ep) return CADNN_OK;
+    le.scale = ep->scale;
+    le.bias = ep->bias;
+    le.residual = ep->residual;
+    le.act = ep->act;
+    le.out_dtype = ep->out_dtype;
+    if (le.act < CADNN_ACT_NONE || le.act > CADNN_ACT_RELU6) return CADNN_E_ARG;
+    if (dt == CADNN_F32) {
+        if (le.out_dtype != CADNN_F32) return CADNN_E_DTYPE;
+    } else {
+        if (le.out_dtype != CADNN_S8 && le.out_dtype != CADNN_S32 && le.out_dtype != CADNN_F32) return CADNN_E_DTYPE;
+        if (le.residual) return CADNN_E_UNSUPPORTED;
+        if (le.act == CADNN_ACT_RELU6) return CADNN_E_UNSUPPORTED;
+    }
+    if (le.residual && !aligned16(le.residual)) return CADNN_E_ARG;
+    return CADNN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+cadnn_status cadnn_conv2d(const cadnn_weights *w, const void *x, int n, int h, int wd, void *y,
+                          const cadnn_epilogue *ep, void *stream)
+{
+    if (!w || !x || !y || n < 0) return CADNN_E_ARG;
+    if (!w->on_device) return CADNN_E_ARG;
+    if (h != w->desc.in_h || wd != w->desc.in_w) return CADNN_E_SHAPE;
+    if (!aligned16(x) || !aligned16(y) || x == y) return CADNN_E_ARG;
+    LaunchEpilogue le;
+    cadnn_status st = check_epilogue(w, ep, le);
+    if (st != CADNN_OK) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    switch (w->s.kind) {
+        case KK_SCONV_SPATIAL:
+        case KK_SCONV_LINEAR: return launch_sconv(w, x, n, y, le, s);
+        case KK_FC_SPMV: return launch_fc_spmv(w, x, n, y, le, s);
+        case KK_DW: return launch_dw(w, x, n, y, le, s);
+    }
+    return CADNN_E_UNSUPPORTED;
+}
+
+cadnn_status cadnn_fc(const cadnn_weights *w, const void *x, int n, void *y, const cadnn_epilogue *ep, void *stream)
+{
+    if (!w) return CADNN_E_ARG;
+    const cadnn_layer_desc &d = w->desc;
+    if (d.kh != 1 || d.kw != 1 || d.in_h != 1 || d.in_w != 1 || d.groups != 1) return CADNN_E_SHAPE;
+    return cadnn_conv2d(w, x, n, 1, 1, y, ep, stream);
+}
+
+cadnn_status cadnn_maxpool2d(const void *x, int n, int h, int wd, int c, int k, int stride, int pad, int dtype,
+                             void *y, void *stream)
+{
+    if (!x || !y || n < 0 || h < 1 || wd < 1 || c < 1 || k < 1 || stride < 1 || pad < 0) return CADNN_E_ARG;
+    if (pad >= k || h + 2 * pad < k || wd + 2 * pad < k) return CADNN_E_SHAPE;
+    if (dtype != CADNN_F32 && dtype != CADNN_S8) return CADNN_E_DTYPE;
+    return launch_maxpool(x, n, h, wd, c, k, stride, pad, dtype, y, (cudaStream_t)stream);
+}
+
+cadnn_status cadnn_global_avgpool(const float *x, int n, int h, int wd, int c, float *y, void *stream)
+{
+    if (!x || !y || n < 0 || h < 1 || wd < 1 || c < 1) return CADNN_E_ARG;
+    return launch_gavgpool(x, n, h, wd, c, y, (cudaStream_t)stream);
+}
+
+const char *cadnn_status_str(cadnn_status s)
+{
+    switch (s) {
+        case CADNN_OK: return "ok";
+        case CADNN_E_ARG: return "invalid argument";
+        case CADNN_E_SHAPE: return "shape mismatch";
+        case CADNN_E_DTYPE: return "dtype combination not defined";
+        case CADNN_E_UNSUPPORTED: return "not supported";
+        case CADNN_E_ALLOC: return "allocation failed";
+        case CADNN_E_CUDA: return "CUDA runtime error";
+        case CADNN_E_DEVICE_STATUS: return "device status word set";
+    }
+    return "unknown status";
+}
+
+const char *cadnn_last_cuda_error(void) { return g_cuda_err; }
+
+}  // extern "C"

@@ -1,0 +1,282 @@
+// Whole-network runner: shape inference over an op list, one device buffer per
+// intermediate tensor, layer-by-layer launch or CUDA-graph replay.
+//
+// CADNN (arXiv 1905.00571), Section 5, reports single-image inference of complete
+// networks.  At batch 1 a pruned layer's work is far below a kernel launch, so the
+// layer sequence is captured once into a CUDA graph and replayed.
+#include <new>
+#include <vector>
+#include "cadnn_internal.h"
+
+struct SlotInfo {
+    int n = 0, h = 0, w = 0, c = 0, dtype = 0;
+    bool defined = false;
+    void *ptr = nullptr;  // owned unless slot 0 or the output slot
+    int64_t bytes = 0;
+};
+
+struct cadnn_net {
+    std::vector<cadnn_op> ops;
+    std::vector<SlotInfo> slots;
+    int out_slot = -1;
+    int64_t workspace = 0;
+    // graph cache: [0] caller's device pointers, [1] the net's own staging buffers
+    struct GraphCache {
+        cudaGraph_t graph = nullptr;
+        cudaGraphExec_t exec = nullptr;
+        const void *x = nullptr;
+        void *y = nullptr;
+    } cache[2];
+    // device staging for cadnn_forward_host
+    void *stage_x = nullptr, *stage_y = nullptr;
+    int64_t in_bytes = 0, out_bytes = 0;
+    // L2 flush buffer for layer timing
+    void *flush = nullptr;
+    size_t flush_bytes = 0;
+};
+
+namespace {
+
+void *slot_ptr(cadnn_net *net, int slot, const void *x, void *y)
+{
+    if (slot == 0) return const_cast<void *>(x);
+    if (slot == net->out_slot) return y;
+    return net->slots[slot].ptr;
+}
+
+cadnn_status run_op(cadnn_net *net, const cadnn_op &op, const void *x, void *y, cudaStream_t st)
+{
+    const SlotInfo &si = net->slots[op.src];
+    const void *src = slot_ptr(net, op.src, x, y);
+    void *dst = slot_ptr(net, op.dst, x, y);
+    if (op.kind == CADNN_OP_CONV || op.kind == CADNN_OP_FC) {
+        cadnn_epilogue ep;
+        ep.scale = op.scale;
+        ep.bias = op.bias;
+        ep.residual = op.res >= 0 ? slot_ptr(net, op.res, x, y) : nullptr;
+        ep.act = op.act;
+        ep.out_dtype = op.out_dtype;
+        if (op.kind == CADNN_OP_FC) return cadnn_fc(op.w, src, si.n, dst, &ep, st);
+        return cadnn_conv2d(op.w, src, si.n, si.h, si.w, dst, &ep, st);
+    }
+    if (op.kind == CADNN_OP_MAXPOOL)
+        return cadnn_maxpool2d(src, si.n, si.h, si.w, si.c, op.pool_k, op.pool_stride, op.pool_pad, si.dtype, dst, st);
+    if (op.kind == CADNN_OP_GAVGPOOL)
+        return cadnn_global_avgpool((const float *)src, si.n, si.h, si.w, si.c, (float *)dst, st);
+    return CADNN_E_ARG;
+}
+
+cadnn_status run_all(cadnn_net *net, const void *x, void *y, cudaStream_t st)
+{
+    for (const cadnn_op &op : net->ops) {
+        cadnn_status s = run_op(net, op, x, y, st);
+        if (s != CADNN_OK) return s;
+    }
+    return CADNN_OK;
+}
+
+void drop_graph(cadnn_net::GraphCache &gc)
+{
+    if (gc.exec) cudaGraphExecDestroy(gc.exec);
+    if (gc.graph) cudaGraphDestroy(gc.graph);
+    gc.exec = nullptr;
+    gc.graph = nullptr;
+}
+
+cadnn_status forward_impl(cadnn_net *net, const void *x, void *y, int use_graph, cudaStream_t st, int slot)
+{
+    if (!use_graph) return run_all(net, x, y, st);
+    cadnn_net::GraphCache &gc = net->cache[slot];
+    if (!gc.exec || gc.x != x || gc.y != y) {
+        drop_graph(gc);
+        // run every kernel once outside capture (first launches raise function attributes)
+        cadnn_status s = run_all(net, x, y, st);
+        if (s != CADNN_OK) return s;
+        cudaStream_t cap = st;
+        bool own = false;
+        if (cap == nullptr || cap == cudaStreamLegacy) {
+            CADNN_CUDA_TRY(cudaStreamSynchronize(st));
+            CADNN_CUDA_TRY(cudaStreamCreateWithFlags(&cap, cudaStreamNonBlocking));
+            own = true;
+        }
+        cudaError_t e = cudaStreamBeginCapture(cap, cudaStreamCaptureModeThreadLocal);
+        if (e != cudaSuccess) { if (own) cudaStreamDestroy(cap); return cadnn_note_cuda(e); }
+        s = run_all(net, x, y, cap);
+        e = cudaStreamEndCapture(cap, &gc.graph);
+        if (own) cudaStreamDestroy(cap);
+        if (s != CADNN_OK) { drop_graph(gc); return s; }
+        if (e != cudaSuccess) { drop_graph(gc); return cadnn_note_cuda(e); }
+        e = cudaGraphInstantiate(&gc.exec, gc.graph, 0);
+        if (e != cudaSuccess) { drop_graph(gc); return cadnn_note_cuda(e); }
+        gc.x = x;
+        gc.y = y;
+    }
+    CADNN_CUDA_TRY(cudaGraphLaunch(gc.exec, st));
+    return CADNN_OK;
+}
+
+__global__ void flush_kernel(float *buf, size_t n)
+{
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        buf[i] = 0.0f;
+}
+
+}  // namespace
+
+extern "C" {
+
+cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int wd, int c, int in_dtype,
+                              cadnn_net **out)
+{
+    if (!ops || !out || n_ops < 1 || n < 1 || h < 1 || wd < 1 || c < 1) return CADNN_E_ARG;
+    if (in_dtype != CADNN_F32 && in_dtype != CADNN_S8) return CADNN_E_DTYPE;
+    cadnn_net *net = new (std::nothrow) cadnn_net();
+    if (!net) return CADNN_E_ALLOC;
+    cadnn_status st = CADNN_OK;
+    int max_slot = 0;
+    for (int i = 0; i < n_ops; ++i) {
+        if (ops[i].src < 0 || ops[i].dst < 1 || ops[i].res < -1) { st = CADNN_E_ARG; break; }
+        max_slot = std::max(max_slot, std::max(ops[i].src, std::max(ops[i].dst, ops[i].res)));
+    }
+    if (st == CADNN_OK) {
+        net->ops.assign(ops, ops + n_ops);
+        net->slots.assign(max_slot + 1, SlotInfo());
+        SlotInfo &in = net->slots[0];
+        in.n = n; in.h = h; in.w = wd; in.c = c; in.dtype = in_dtype; in.defined = true;
+        net->out_slot = ops[n_ops - 1].dst;
+        net->in_bytes = (int64_t)n * h * wd * c * dtype_size(in_dtype);
+    }
+    for (int i = 0; i < n_ops && st == CADNN_OK; ++i) {
+        const cadnn_op &op = ops[i];
+        const SlotInfo si = net->slots[op.src];
+        SlotInfo &so = net->slots[op.dst];
+        if (!si.defined || so.defined) { st = CADNN_E_ARG; break; }
+        so.n = si.n;
+        if (op.kind == CADNN_OP_CONV || op.kind == CADNN_OP_FC) {
+            if (!op.w || !op.w->on_device) { st = CADNN_E_ARG; break; }
+            const cadnn_layer_desc &d = op.w->desc;
+            if (d.dtype != si.dtype) { st = CADNN_E_DTYPE; break; }
+            if (op.kind == CADNN_OP_FC) {
+                if ((long long)si.h * si.w * si.c != d.c_in) { st = CADNN_E_SHAPE; break; }
+            } else if (si.h != d.in_h || si.w != d.in_w || si.c != d.c_in) { st = CADNN_E_SHAPE; break; }
+            so.h = op.w->h_out; so.w = op.w->w_out; so.c = d.c_out; so.dtype = op.out_dtype;
+            if (op.res >= 0) {
+                const SlotInfo &sr = net->slots[op.res];
+                if (!sr.defined || sr.h != so.h || sr.w != so.w || sr.c != so.c || sr.dtype != so.dtype) {
+                    st = CADNN_E_SHAPE;
+                    break;
+                }
+            }
+        } else if (op.kind == CADNN_OP_MAXPOOL) {
+            if (op.pool_k < 1 || op.pool_stride < 1 || op.pool_pad < 0 || op.pool_pad >= op.pool_k ||
+                si.h + 2 * op.pool_pad < op.pool_k || si.w + 2 * op.pool_pad < op.pool_k) { st = CADNN_E_SHAPE; break; }
+            so.h = (si.h + 2 * op.pool_pad - op.pool_k) / op.pool_stride + 1;
+            so.w = (si.w + 2 * op.pool_pad - op.pool_k) / op.pool_stride + 1;
+            so.c = si.c; so.dtype = si.dtype;
+        } else if (op.kind == CADNN_OP_GAVGPOOL) {
+            if (si.dtype != CADNN_F32) { st = CADNN_E_DTYPE; break; }
+            so.h = 1; so.w = 1; so.c = si.c; so.dtype = CADNN_F32;
+        } else { st = CADNN_E_ARG; break; }
+        so.defined = true;
+        so.bytes = (int64_t)so.n * so.h * so.w * so.c * dtype_size(so.dtype);
+        if (op.dst != net->out_slot) {
+            size_t alloc = (size_t)((so.bytes + 255) / 256 * 256);
+            cudaError_t e = cudaMalloc(&so.ptr, alloc ? alloc : 256);
+            if (e != cudaSuccess) {
+                cadnn_note_cuda(e);
+                st = e == cudaErrorMemoryAllocation ? CADNN_E_ALLOC : CADNN_E_CUDA;
+                break;
+            }
+            net->workspace += (int64_t)alloc;
+        }
+    }
+    if (st != CADNN_OK) {
+        cadnn_net_free(net);
+        return st;
+    }
+    net->out_bytes = net->slots[net->out_slot].bytes;
+    *out = net;
+    return CADNN_OK;
+}
+
+cadnn_status cadnn_forward(cadnn_net *net, const void *x, void *y, int use_graph, void *stream)
+{
+    if (!net || !x || !y) return CADNN_E_ARG;
+    return forward_impl(net, x, y, use_graph, (cudaStream_t)stream, 0);
+}
+
+cadnn_status cadnn_forward_host(cadnn_net *net, const void *x_host, void *y_host, int use_graph, void *stream)
+{
+    if (!net || !x_host || !y_host) return CADNN_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!net->stage_x) {
+        cudaError_t e = cudaMalloc(&net->stage_x, (size_t)((net->in_bytes + 255) / 256 * 256));
+        if (e == cudaSuccess) e = cudaMalloc(&net->stage_y, (size_t)((net->out_bytes + 255) / 256 * 256));
+        if (e != cudaSuccess) {
+            cadnn_note_cuda(e);
+            return e == cudaErrorMemoryAllocation ? CADNN_E_ALLOC : CADNN_E_CUDA;
+        }
+    }
+    CADNN_CUDA_TRY(cudaMemcpyAsync(net->stage_x, x_host, (size_t)net->in_bytes, cudaMemcpyHostToDevice, st));
+    cadnn_status s = forward_impl(net, net->stage_x, net->stage_y, use_graph, st, 1);
+    if (s != CADNN_OK) return s;
+    CADNN_CUDA_TRY(cudaMemcpyAsync(y_host, net->stage_y, (size_t)net->out_bytes, cudaMemcpyDeviceToHost, st));
+    CADNN_CUDA_TRY(cudaStreamSynchronize(st));
+    return CADNN_OK;
+}
+
+cadnn_status cadnn_net_info(const cadnn_net *net, int *n_launches, int64_t *workspace_bytes)
+{
+    if (!net) return CADNN_E_ARG;
+    if (n_launches) *n_launches = (int)net->ops.size();
+    if (workspace_bytes) *workspace_bytes = net->workspace;
+    return CADNN_OK;
+}
+
+cadnn_status cadnn_net_layer_times(cadnn_net *net, const void *x, void *y, int flush_l2, float *ms, void *stream)
+{
+    if (!net || !x || !y || !ms) return CADNN_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t nops = net->ops.size();
+    if (flush_l2 && !net->flush) {
+        net->flush_bytes = 256u << 20;
+        CADNN_CUDA_TRY(cudaMalloc(&net->flush, net->flush_bytes));
+    }
+    std::vector<cudaEvent_t> ev(2 * nops);
+    for (auto &e : ev) CADNN_CUDA_TRY(cudaEventCreate(&e));
+    cadnn_status s = CADNN_OK;
+    for (size_t i = 0; i < nops && s == CADNN_OK; ++i) {
+        if (flush_l2) flush_kernel<<<148 * 8, 256, 0, st>>>((float *)net->flush, net->flush_bytes / 4);
+        cudaEventRecord(ev[2 * i], st);
+        s = run_op(net, net->ops[i], x, y, st);
+        cudaEventRecord(ev[2 * i + 1], st);
+    }
+    cudaError_t e = cudaStreamSynchronize(st);
+    if (s == CADNN_OK && e != cudaSuccess) s = cadnn_note_cuda(e);
+    for (size_t i = 0; i < nops && s == CADNN_OK; ++i) cudaEventElapsedTime(&ms[i], ev[2 * i], ev[2 * i + 1]);
+    for (auto &ev1 : ev) cudaEventDestroy(ev1);
+    return s;
+}
+
+cadnn_status cadnn_net_slot(const cadnn_net *net, int slot, void **ptr, int64_t *bytes)
+{
+    if (!net || slot < 0 || slot >= (int)net->slots.size() || !net->slots[slot].defined) return CADNN_E_ARG;
+    if (ptr) *ptr = net->slots[slot].ptr;
+    if (bytes) *bytes = net->slots[slot].bytes;
+    return CADNN_OK;
+}
+
+void cadnn_net_free(cadnn_net *net)
+{
+    if (!net) return;
+    drop_graph(net->cache[0]);
+    drop_graph(net->cache[1]);
+    if (net->stage_x) cudaFree(net->stage_x);
+    if (net->stage_y) cudaFree(net->stage_y);
+    for (SlotInfo &s : net->slots)
+        if (s.ptr) cudaFree(s.ptr);
+    if (net->flush) cudaFree(net->flush);
+    delete net;
+}
+
+}  // extern "C"

@@ -1,0 +1,76 @@
+// Glue layers of the evaluated networks: max pooling (float and int8) and global
+// average pooling.  The paper (arXiv 1905.00571) does not discuss them; they are
+// bound by one read and one write of the feature map, so lanes map to channels.
+#include <cfloat>
+#include "cadnn_internal.h"
+
+namespace {
+
+template <typename XT>
+__global__ void __launch_bounds__(256) maxpool_kernel(const XT *x, XT *y, int n, int h, int w, int c, int h_out,
+                                                      int w_out, int k, int stride, int pad)
+{
+    const long long total = (long long)n * h_out * w_out * c;
+    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int ch = (int)(idx % c);
+        long long pix = idx / c;
+        const int ox = (int)(pix % w_out);
+        long long r = pix / w_out;
+        const int oy = (int)(r % h_out);
+        const int b = (int)(r / h_out);
+        bool any = false;
+        XT best = 0;
+        for (int ky = 0; ky < k; ++ky) {
+            const int iy = oy * stride + ky - pad;
+            if (iy < 0 || iy >= h) continue;
+            for (int kx = 0; kx < k; ++kx) {
+                const int ix = ox * stride + kx - pad;
+                if (ix < 0 || ix >= w) continue;
+                const XT v = x[(((size_t)b * h + iy) * w + ix) * c + ch];
+                if (!any || v > best) best = v;
+                any = true;
+            }
+        }
+        y[idx] = best;
+    }
+}
+
+__global__ void __launch_bounds__(256) gavgpool_kernel(const float *x, float *y, int n, int hw, int c, float inv)
+{
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= n * c) return;
+    const int b = idx / c, ch = idx - b * c;
+    const float *src = x + (size_t)b * hw * c + ch;
+    float s = 0.0f;
+    for (int i = 0; i < hw; ++i) s += src[(size_t)i * c];
+    y[idx] = s * inv;
+}
+
+}  // namespace
+
+cadnn_status launch_maxpool(const void *x, int n, int h, int wd, int c, int k, int stride, int pad, int dtype,
+                            void *y, cudaStream_t st)
+{
+    const int h_out = (h + 2 * pad - k) / stride + 1, w_out = (wd + 2 * pad - k) / stride + 1;
+    long long total = (long long)n * h_out * w_out * c;
+    if (total <= 0) return CADNN_OK;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148LL * 64) blocks = 148LL * 64;
+    if (dtype == CADNN_S8)
+        maxpool_kernel<int8_t><<<(int)blocks, 256, 0, st>>>((const int8_t *)x, (int8_t *)y, n, h, wd, c, h_out, w_out, k,
+                                                           stride, pad);
+    else
+        maxpool_kernel<float><<<(int)blocks, 256, 0, st>>>((const float *)x, (float *)y, n, h, wd, c, h_out, w_out, k,
+                                                          stride, pad);
+    CADNN_CUDA_TRY(cudaGetLastError());
+    return CADNN_OK;
+}
+
+cadnn_status launch_gavgpool(const float *x, int n, int h, int wd, int c, float *y, cudaStream_t st)
+{
+    if (n * c <= 0) return CADNN_OK;
+    gavgpool_kernel<<<(n * c + 255) / 256, 256, 0, st>>>(x, y, n, h * wd, c, 1.0f / (float)(h * wd));
+    CADNN_CUDA_TRY(cudaGetLastError());
+    return CADNN_OK;
+}

@@ -1,0 +1,133 @@
+"""CPU-side checks of the C ABI: the library loads, exports every symbol the header
+declares, and the host-only packer round-trips and balances (no GPU needed)."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+from workloads import gen, models
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_1905_00571_b200 import build
+    build.build()
+    from paper_1905_00571_b200 import binding
+    return binding
+
+
+def test_every_declared_symbol_is_exported(B):
+    import ctypes
+    hdr = open(os.path.join(ROOT, "include", "cadnn.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    names = set(re.findall(r"\b(cadnn_[a-z0-9_]+)\s*\(", hdr))
+    assert len(names) >= 19
+    lib = ctypes.CDLL(B.LIB_PATH)
+    for n in sorted(names):
+        assert hasattr(lib, n), n
+    assert names == set(B.EXPORTED)
+
+
+def _host_pack(B, w, mask, in_hw, stride=1, pad=1, dtype="f32", hint=1, q8=False, scale=None):
+    c_out, kh, kw, c_in = w.shape
+    d = B.make_desc(c_in, c_out, kh, kw, stride, pad, 1, in_hw, in_hw, hint, dtype, host_only=True)
+    return B.cadnn_pack_q8(d, w, mask) if q8 else B.cadnn_pack(d, w, mask, scale)
+
+
+@pytest.mark.parametrize("shape,hw,density", [((64, 3, 3, 64), 56, 0.1), ((70, 3, 3, 130), 20, 0.05),
+                                               ((256, 1, 1, 64), 56, 0.125), ((16, 7, 7, 3), 224, 1.0),
+                                               ((32, 3, 3, 16), 14, 0.0)])
+@pytest.mark.parametrize("hint", [1, 64])
+def test_pack_unpack_round_trip(B, shape, hw, density, hint):
+    g = gen.rng(11)
+    w = gen.he_weights(g, *shape)
+    mask = None if density >= 1.0 else gen.random_mask(g, shape, density)
+    pad = shape[1] // 2
+    wh = _host_pack(B, w, mask, hw, 1, pad, hint=hint)
+    dense, m2 = B.cadnn_weights_unpack(wh)
+    want_mask = np.ones(shape, np.uint8) if mask is None else mask
+    np.testing.assert_array_equal(m2, want_mask)
+    np.testing.assert_array_equal(dense, w * want_mask)
+    info = B.cadnn_weights_info(wh)
+    assert info["nnz"] == int(want_mask.sum())
+    # canonical accounting: value + 16-bit offset per stored nonzero, plus row pointers
+    assert info["packed_bytes"] >= 6 * info["nnz"]
+
+
+def test_pack_keeps_masked_in_zero_values(B):
+    w = np.zeros((8, 1, 1, 8), np.float32)
+    mask = np.eye(8, dtype=np.uint8).reshape(8, 1, 1, 8)
+    wh = _host_pack(B, w, mask, 4, 1, 0)
+    assert B.cadnn_weights_info(wh)["nnz"] == 8
+    _, m2 = B.cadnn_weights_unpack(wh)
+    np.testing.assert_array_equal(m2, mask)
+
+
+def test_fc_row_csr_round_trip_and_s8(B):
+    g = gen.rng(12)
+    q = gen.int8_weights(g, (100, 1, 1, 3000))
+    mask = gen.random_mask(g, q.shape, 0.04)
+    d = B.make_desc(3000, 100, batch_hint=1, dtype="s8", host_only=True)
+    wh = B.cadnn_pack_q8(d, q, mask)
+    assert B.cadnn_weights_info(wh)["fmt"] == 2
+    dense, m2 = B.cadnn_weights_unpack(wh)
+    np.testing.assert_array_equal(m2, mask)
+    np.testing.assert_array_equal(dense, (q * mask).astype(np.float32))
+
+
+def test_float_to_int8_quantization_in_the_packer(B):
+    w = np.array([0.25, 0.75, 1.25, -0.75, 100.0, -100.0, 0.3, 0.0], np.float32).reshape(1, 1, 1, 8)
+    s = np.array([0.5], np.float32)
+    d = B.make_desc(8, 1, in_h=2, in_w=2, dtype="s8", host_only=True)
+    wh = B.cadnn_pack(d, w, None, s)
+    dense, _ = B.cadnn_weights_unpack(wh)
+    np.testing.assert_array_equal(dense.reshape(-1), np.array([0, 2, 2, -2, 127, -127, 1, 0], np.float32))
+
+
+def test_regrouping_balances_warp_loads_on_a_skewed_mask(B):
+    g = gen.rng(13)
+    shape = (256, 3, 3, 64)
+    w = gen.he_weights(g, *shape)
+    mask = gen.skewed_mask(g, shape, 0.125, skew=8.0)
+    wh = _host_pack(B, w, mask, 28, hint=64)
+    s = B.cadnn_weights_schedule(wh)
+    assert s["RPW"] >= 2
+    loads = B.cadnn_weights_warp_loads(wh).reshape(-1, 8)          # [block][warp]
+    per_row = mask.reshape(256, -1).sum(1)
+    naive = per_row.reshape(-1, 8, s["RPW"]).sum(2)                 # consecutive filters per warp
+    spread = lambda a: float((a.max(1) / np.maximum(a.mean(1), 1)).mean())
+    assert loads.sum() == mask.sum()
+    assert spread(loads) < spread(naive)
+    assert spread(loads) < 1.25
+
+
+def test_pack_rejects_bad_arguments(B):
+    w = np.zeros((8, 3, 3, 8), np.float32)
+    d = B.make_desc(8, 8, 3, 3, 1, 1, 2, 10, 10, 1, "f32", host_only=True)      # grouped, not depthwise
+    with pytest.raises(B.CadnnError) as e:
+        B.cadnn_pack(d, np.zeros((8, 3, 3, 4), np.float32))
+    assert e.value.status == 4
+    d = B.make_desc(8, 8, 3, 3, 0, 1, 1, 10, 10, 1, "f32", host_only=True)      # stride 0
+    with pytest.raises(B.CadnnError) as e:
+        B.cadnn_pack(d, w)
+    assert e.value.status == 1
+    d = B.make_desc(8, 8, 3, 3, 1, 1, 1, 10, 10, 1, "s8", host_only=True)       # int8 without scale
+    with pytest.raises(B.CadnnError) as e:
+        B.cadnn_pack(d, w)
+    assert e.value.status == 1
+    d = B.make_desc(140000, 4, dtype="s8", host_only=True)                       # int32 sum could overflow
+    with pytest.raises(B.CadnnError) as e:
+        B.cadnn_pack_q8(d, np.zeros((4, 1, 1, 140000), np.int8))
+    assert e.value.status == 4
+
+
+def test_compute_without_device_image_is_refused(B):
+    d = B.make_desc(8, 8, 1, 1, in_h=4, in_w=4, host_only=True)
+    wh = B.cadnn_pack(d, np.zeros((8, 1, 1, 8), np.float32))
+    import ctypes
+    ep = None
+    st = B._lib.cadnn_conv2d(wh.handle, ctypes.c_void_p(256), 1, 4, 4, ctypes.c_void_p(512), ep, None)
+    assert st == 1
