@@ -112,10 +112,14 @@ cadnn_status cadnn_weights_info(const cadnn_weights *w, int64_t *nnz, int64_t *p
 
 /*
  * Schedule the packer chose (Section 4, "Optimization parameters selection"):
- * sched[0..7] = kernel kind, pixels per lane, filters per warp, filters per block,
- * channel chunk, tile rows, tile columns, shared-memory row pitch.  Host ints.
+ * sched[0..15] = kernel kind, pixel bands per lane, filters per warp, filters per block,
+ * channel chunk, tile rows, tile columns, shared-memory row pitch, warps per block,
+ * pipeline stages, blocks per cluster (reduction split), channel chunks, shared-memory
+ * bytes per block, bands across, bands down, entries per weight record.  Host ints.
+ * The environment variable CADNN_SCHEDULE ("nw=8,rpw=2,tbx=1,tby=4,cic=64,ks=2", any
+ * subset) overrides the packer's pick for conv layers; it exists for tuning.
  */
-cadnn_status cadnn_weights_schedule(const cadnn_weights *w, int sched[8]);
+cadnn_status cadnn_weights_schedule(const cadnn_weights *w, int sched[16]);
 
 /*
  * Per-warp load of the packed image: for every (filter block, warp) the number of
@@ -205,6 +209,9 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
  * cadnn_forward - run the network: x device input, y device output of the last op.
  * use_graph != 0 replays a CUDA graph captured on the first call with this (x, y)
  * pair (re-captured when either pointer changes); 0 launches the layers one by one.
+ * Layers after the first are launched as programmatic dependents of their predecessor
+ * (their weight fetch overlaps its tail); set CADNN_NO_PDL in the environment before
+ * cadnn_net_create to use plain stream order instead.
  * Asynchronous on stream.
  */
 cadnn_status cadnn_forward(cadnn_net *net, const void *x, void *y, int use_graph, void *stream);
@@ -221,11 +228,13 @@ cadnn_status cadnn_forward_host(cadnn_net *net, const void *x_host, void *y_host
 cadnn_status cadnn_net_info(const cadnn_net *net, int *n_launches, int64_t *workspace_bytes);
 
 /*
- * Measurement aid: run the network once layer by layer on stream with a CUDA event
- * pair around every op, synchronize, and write the per-op milliseconds to ms[n_ops]
- * (host).  flush_l2 != 0 overwrites a buffer larger than L2 before each op.
+ * Measurement aid: time every op on its own.  Each op is captured into a CUDA graph of
+ * `reps` back-to-back launches (so the host launch cost stays out) and replayed between
+ * a CUDA event pair on stream; ms[n_ops] (host) receives milliseconds per launch.
+ * flush_l2 != 0 overwrites a buffer larger than L2 before the timed replay (meaningful
+ * with reps = 1); otherwise the graph is replayed once untimed first.  Synchronizes.
  */
-cadnn_status cadnn_net_layer_times(cadnn_net *net, const void *x, void *y, int flush_l2, float *ms,
+cadnn_status cadnn_net_layer_times(cadnn_net *net, const void *x, void *y, int flush_l2, int reps, float *ms,
                                    void *stream);
 
 /* Device pointer and byte size of slot `slot` (for per-layer inspection). */

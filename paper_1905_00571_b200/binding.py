@@ -62,7 +62,7 @@ _SIGS = {
     "cadnn_forward": (_i, [_vp, _vp, _vp, _i, _vp]),
     "cadnn_forward_host": (_i, [_vp, _vp, _vp, _i, _vp]),
     "cadnn_net_info": (_i, [_vp, ctypes.POINTER(_i), _i64p]),
-    "cadnn_net_layer_times": (_i, [_vp, _vp, _vp, _i, ctypes.POINTER(ctypes.c_float), _vp]),
+    "cadnn_net_layer_times": (_i, [_vp, _vp, _vp, _i, _i, ctypes.POINTER(ctypes.c_float), _vp]),
     "cadnn_net_slot": (_i, [_vp, _i, ctypes.POINTER(_vp), _i64p]),
     "cadnn_net_free": (None, [_vp]),
     "cadnn_status_str": (ctypes.c_char_p, [_i]),
@@ -162,9 +162,10 @@ def cadnn_weights_info(w):
 
 
 def cadnn_weights_schedule(w):
-    arr = (ctypes.c_int * 8)()
+    arr = (ctypes.c_int * 16)()
     _check(_lib.cadnn_weights_schedule(w.handle, arr), "cadnn_weights_schedule")
-    keys = ("kind", "T", "RPW", "G", "CIc", "TH", "TW", "pitch")
+    keys = ("kind", "T", "RPW", "G", "CIc", "TH", "TW", "pitch", "NW", "stages", "ksplit", "chunks", "smem",
+            "TBX", "TBY", "max_entries")
     return dict(zip(keys, list(arr)))
 
 
@@ -273,9 +274,10 @@ def cadnn_net_info(net):
     return {"launches": nl.value, "workspace_bytes": ws.value}
 
 
-def cadnn_net_layer_times(net, x, y, n_ops, flush_l2=False, stream=None):
+def cadnn_net_layer_times(net, x, y, n_ops, flush_l2=False, reps=1, stream=None):
     ms = (ctypes.c_float * n_ops)()
-    _check(_lib.cadnn_net_layer_times(net.handle, _dev_ptr(x), _dev_ptr(y), 1 if flush_l2 else 0, ms, _stream(stream)),
+    _check(_lib.cadnn_net_layer_times(net.handle, _dev_ptr(x), _dev_ptr(y), 1 if flush_l2 else 0, int(reps), ms,
+                                      _stream(stream)),
            "cadnn_net_layer_times")
     return [float(v) for v in ms]
 

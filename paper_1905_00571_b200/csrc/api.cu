@@ -44,10 +44,8 @@ cadnn_status check_epilogue(const cadnn_weights *w, const cadnn_epilogue *ep, La
 
 }  // namespace
 
-extern "C" {
-
-cadnn_status cadnn_conv2d(const cadnn_weights *w, const void *x, int n, int h, int wd, void *y,
-                          const cadnn_epilogue *ep, void *stream)
+cadnn_status conv2d_impl(const cadnn_weights *w, const void *x, int n, int h, int wd, void *y, const cadnn_epilogue *ep,
+                         bool pdl, cudaStream_t s)
 {
     if (!w || !x || !y || n < 0) return CADNN_E_ARG;
     if (!w->on_device) return CADNN_E_ARG;
@@ -56,7 +54,7 @@ cadnn_status cadnn_conv2d(const cadnn_weights *w, const void *x, int n, int h, i
     LaunchEpilogue le;
     cadnn_status st = check_epilogue(w, ep, le);
     if (st != CADNN_OK) return st;
-    cudaStream_t s = (cudaStream_t)stream;
+    le.pdl = pdl;
     switch (w->s.kind) {
         case KK_SCONV_SPATIAL:
         case KK_SCONV_LINEAR: return launch_sconv(w, x, n, y, le, s);
@@ -64,6 +62,14 @@ cadnn_status cadnn_conv2d(const cadnn_weights *w, const void *x, int n, int h, i
         case KK_DW: return launch_dw(w, x, n, y, le, s);
     }
     return CADNN_E_UNSUPPORTED;
+}
+
+extern "C" {
+
+cadnn_status cadnn_conv2d(const cadnn_weights *w, const void *x, int n, int h, int wd, void *y,
+                          const cadnn_epilogue *ep, void *stream)
+{
+    return conv2d_impl(w, x, n, h, wd, y, ep, false, (cudaStream_t)stream);
 }
 
 cadnn_status cadnn_fc(const cadnn_weights *w, const void *x, int n, void *y, const cadnn_epilogue *ep, void *stream)
@@ -80,13 +86,13 @@ cadnn_status cadnn_maxpool2d(const void *x, int n, int h, int wd, int c, int k, 
     if (!x || !y || n < 0 || h < 1 || wd < 1 || c < 1 || k < 1 || stride < 1 || pad < 0) return CADNN_E_ARG;
     if (pad >= k || h + 2 * pad < k || wd + 2 * pad < k) return CADNN_E_SHAPE;
     if (dtype != CADNN_F32 && dtype != CADNN_S8) return CADNN_E_DTYPE;
-    return launch_maxpool(x, n, h, wd, c, k, stride, pad, dtype, y, (cudaStream_t)stream);
+    return launch_maxpool(x, n, h, wd, c, k, stride, pad, dtype, y, false, (cudaStream_t)stream);
 }
 
 cadnn_status cadnn_global_avgpool(const float *x, int n, int h, int wd, int c, float *y, void *stream)
 {
     if (!x || !y || n < 0 || h < 1 || wd < 1 || c < 1) return CADNN_E_ARG;
-    return launch_gavgpool(x, n, h, wd, c, y, (cudaStream_t)stream);
+    return launch_gavgpool(x, n, h, wd, c, y, false, (cudaStream_t)stream);
 }
 
 const char *cadnn_status_str(cadnn_status s)

@@ -13,24 +13,29 @@ enum KernelKind {
     KK_DENSE_SMALLC = 5    // dense conv with <= 4 input channels
 };
 
-static const int kWarpsPerBlock = 8;
+static const int kWarpsPerBlock = 8;  // fc kernel; the conv kernels take it from the schedule
 
 // Per-layer schedule chosen by the packer (Section 4, "Optimization parameters selection").
 struct Schedule {
     int kind = 0;
-    int T = 1;        // output pixels per lane
+    int T = 1;        // pixel bands per lane (one band = up to 32 output pixels, one per lane)
     int RPW = 1;      // filters per warp
-    int G = 8;        // filters per thread block = kWarpsPerBlock * RPW
+    int NW = 8;       // warps per thread block
+    int G = 8;        // filters per thread block = NW * RPW
     int CIc = 0;      // input channels staged per chunk
-    int PP = 1;       // shared-memory words per staged input pixel (odd: CIc | 1)
-    int TH = 1, TW = 1;      // output tile (spatial mode)
-    int pitch = 0;           // staged input row pitch in pixels (== TW mod 32)
+    int PPb = 4;      // bytes per staged input pixel (an odd number of 32-bit words)
+    int BW = 32, RB = 1;     // band = RB rows x BW columns of output pixels (RB * BW <= 32)
+    int TBX = 1, TBY = 1;    // bands across / down in a tile (T = TBX * TBY)
+    int TH = 1, TW = 32;     // output tile = (TBY * RB) x (TBX * BW)
+    int pitch = 0;           // staged input row pitch in pixels (padded so a band hits 32 distinct banks)
+    int half = 0;            // stride 2: columns per parity plane of a staged row (0 = not de-interleaved)
     int IH_t = 0, IW_t = 0;  // staged input tile extent
     int n_chunks = 1;
     int n_groups = 1;
-    int max_entries = 0;     // most nonzeros any (block, chunk) holds
-    int tile_words = 0;
-    int smem_bytes = 0;
+    int stages = 1;          // shared-memory pipeline depth
+    int ksplit = 1;          // thread blocks per cluster splitting the channel chunks (partial sums meet in DSMEM)
+    int max_entries = 0;     // (padded) entries of the fullest (chunk, filter block) record
+    int tile_bytes = 0, stage_bytes = 0, smem_bytes = 0;
 };
 
 struct cadnn_weights {
@@ -44,16 +49,21 @@ struct cadnn_weights {
     int device = -1;
 
     // host image
-    std::vector<float> vals_f;       // f32 layers: stored values (packed order)
-    std::vector<int8_t> vals_q;      // s8 layers
-    std::vector<uint16_t> offs;      // sconv: staged-tile word offset; fc: column index
-    std::vector<int32_t> ptr;        // sconv: [n_chunks][c_pad + 1]; fc: [c_pad + 1]
+    std::vector<uint32_t> ent;       // conv: fixed-size records, one per (chunk, filter block): a header of
+                                     // G + 1 row starts, then entries.  f32 entry: {value bits, byte offset};
+                                     // s8 entry: (byte offset << 8) | (value & 0xff).  Rows padded to even counts.
+    std::vector<int32_t> cnt;        // conv: real entries per [chunk][packed row] (the rest is padding)
+    std::vector<float> vals_f;       // fc f32: stored values (packed order)
+    std::vector<int8_t> vals_q;      // fc s8
+    std::vector<uint16_t> offs;      // fc: column index
+    std::vector<int32_t> ptr;        // fc: [c_pad + 1]
     std::vector<int32_t> perm;       // packed row -> original output channel, -1 = padding row
     std::vector<float> dense_f;      // dense kinds: tap-major weights
     int c_pad = 0;
 
     // device image (one allocation)
     void *d_blob = nullptr;
+    const uint32_t *d_ent = nullptr;
     const void *d_vals = nullptr;
     const uint16_t *d_offs = nullptr;
     const int32_t *d_ptr = nullptr;
@@ -67,6 +77,7 @@ struct LaunchEpilogue {
     const void *residual = nullptr;
     int act = 0;
     int out_dtype = 0;
+    bool pdl = false;   // launch as a programmatic dependent of the previous kernel (inside cadnn_forward)
 };
 
 // status helpers
@@ -84,10 +95,38 @@ cadnn_status launch_fc_spmv(const cadnn_weights *w, const void *x, int n, void *
                             cudaStream_t st);
 cadnn_status launch_dw(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
                        cudaStream_t st);
-cadnn_status launch_dense_smallc(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
-                                 cudaStream_t st);
 cadnn_status launch_maxpool(const void *x, int n, int h, int wd, int c, int k, int stride, int pad, int dtype,
-                            void *y, cudaStream_t st);
-cadnn_status launch_gavgpool(const float *x, int n, int h, int wd, int c, float *y, cudaStream_t st);
+                            void *y, bool pdl, cudaStream_t st);
+cadnn_status launch_gavgpool(const float *x, int n, int h, int wd, int c, float *y, bool pdl, cudaStream_t st);
+
+// layer entry shared by the public calls and the network runner
+cadnn_status conv2d_impl(const cadnn_weights *w, const void *x, int n, int h, int wd, void *y, const cadnn_epilogue *ep,
+                         bool pdl, cudaStream_t st);
+
+#ifdef __CUDACC__
+// Programmatic dependent launch: a kernel launched with the attribute may start before its
+// predecessor in the stream has finished; it must not touch data the predecessor writes
+// until grid_dep_wait() returns.  Without the attribute both calls do nothing.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_trigger() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cadnn_status launch_kernel(void (*kern)(KArgs...), int blocks, int threads, size_t smem, bool pdl, cudaStream_t st,
+                           Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks, 1, 1);
+    cfg.blockDim = dim3((unsigned)threads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    CADNN_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...));
+    return CADNN_OK;
+}
+#endif
 
 static inline int dtype_size(int dt) { return dt == CADNN_S8 ? 1 : 4; }

@@ -32,6 +32,8 @@ __global__ void __launch_bounds__(256) dw_kernel(const DwParams p)
 {
     const int cv = p.c / VEC;
     const long long total = (long long)p.n * p.h_out * p.w_out * cv;
+    grid_dep_wait();
+    grid_dep_trigger();
     for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
          idx += (long long)gridDim.x * blockDim.x) {
         const int c0 = (int)(idx % cv) * VEC;
@@ -92,8 +94,6 @@ cadnn_status launch_dw(const cadnn_weights *w, const void *x, int n, void *y, co
     if (total <= 0) return CADNN_OK;
     long long blocks = (total + 255) / 256;
     if (blocks > 148LL * 64) blocks = 148LL * 64;
-    if (v4) dw_kernel<4><<<(int)blocks, 256, 0, st>>>(p);
-    else dw_kernel<1><<<(int)blocks, 256, 0, st>>>(p);
-    CADNN_CUDA_TRY(cudaGetLastError());
-    return CADNN_OK;
+    if (v4) return launch_kernel(dw_kernel<4>, (int)blocks, 256, 0, ep.pdl, st, p);
+    return launch_kernel(dw_kernel<1>, (int)blocks, 256, 0, ep.pdl, st, p);
 }

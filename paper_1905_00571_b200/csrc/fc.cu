@@ -36,6 +36,8 @@ __global__ void __launch_bounds__(256) fc_spmv_kernel(const FcParams p)
     typedef typename std::conditional<sizeof(XT) == 1, int, float>::type AT;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int row = blockIdx.x * kWarpsPerBlock + warp;
+    grid_dep_wait();
+    grid_dep_trigger();
     if (row >= p.c_pad) return;
     const int co = p.perm[row];
     if (co < 0) return;
@@ -89,14 +91,12 @@ __global__ void __launch_bounds__(256) fc_spmv_kernel(const FcParams p)
 }
 
 template <typename XT>
-cadnn_status launch_nb(const FcParams &p, int blocks, cudaStream_t st)
+cadnn_status launch_nb(const FcParams &p, int blocks, bool pdl, cudaStream_t st)
 {
-    if (p.n <= 1) fc_spmv_kernel<XT, 1><<<blocks, 256, 0, st>>>(p);
-    else if (p.n <= 2) fc_spmv_kernel<XT, 2><<<blocks, 256, 0, st>>>(p);
-    else if (p.n <= 4) fc_spmv_kernel<XT, 4><<<blocks, 256, 0, st>>>(p);
-    else fc_spmv_kernel<XT, 8><<<blocks, 256, 0, st>>>(p);
-    CADNN_CUDA_TRY(cudaGetLastError());
-    return CADNN_OK;
+    if (p.n <= 1) return launch_kernel(fc_spmv_kernel<XT, 1>, blocks, 256, 0, pdl, st, p);
+    if (p.n <= 2) return launch_kernel(fc_spmv_kernel<XT, 2>, blocks, 256, 0, pdl, st, p);
+    if (p.n <= 4) return launch_kernel(fc_spmv_kernel<XT, 4>, blocks, 256, 0, pdl, st, p);
+    return launch_kernel(fc_spmv_kernel<XT, 8>, blocks, 256, 0, pdl, st, p);
 }
 
 }  // namespace
@@ -112,6 +112,6 @@ cadnn_status launch_fc_spmv(const cadnn_weights *w, const void *x, int n, void *
     p.act = ep.act; p.out_dtype = ep.out_dtype;
     if (n <= 0) return CADNN_OK;
     int blocks = w->c_pad / kWarpsPerBlock;
-    if (w->desc.dtype == CADNN_S8) return launch_nb<int8_t>(p, blocks, st);
-    return launch_nb<float>(p, blocks, st);
+    if (w->desc.dtype == CADNN_S8) return launch_nb<int8_t>(p, blocks, ep.pdl, st);
+    return launch_nb<float>(p, blocks, ep.pdl, st);
 }

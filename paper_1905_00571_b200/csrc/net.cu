@@ -4,6 +4,7 @@
 // CADNN (arXiv 1905.00571), Section 5, reports single-image inference of complete
 // networks.  At batch 1 a pruned layer's work is far below a kernel launch, so the
 // layer sequence is captured once into a CUDA graph and replayed.
+#include <cstdlib>
 #include <new>
 #include <vector>
 #include "cadnn_internal.h"
@@ -19,6 +20,7 @@ struct cadnn_net {
     std::vector<cadnn_op> ops;
     std::vector<SlotInfo> slots;
     int out_slot = -1;
+    bool use_pdl = true;   // layers after the first launch as programmatic dependents
     int64_t workspace = 0;
     // graph cache: [0] caller's device pointers, [1] the net's own staging buffers
     struct GraphCache {
@@ -44,7 +46,7 @@ void *slot_ptr(cadnn_net *net, int slot, const void *x, void *y)
     return net->slots[slot].ptr;
 }
 
-cadnn_status run_op(cadnn_net *net, const cadnn_op &op, const void *x, void *y, cudaStream_t st)
+cadnn_status run_op(cadnn_net *net, const cadnn_op &op, const void *x, void *y, cudaStream_t st, bool pdl = false)
 {
     const SlotInfo &si = net->slots[op.src];
     const void *src = slot_ptr(net, op.src, x, y);
@@ -56,21 +58,26 @@ cadnn_status run_op(cadnn_net *net, const cadnn_op &op, const void *x, void *y, 
         ep.residual = op.res >= 0 ? slot_ptr(net, op.res, x, y) : nullptr;
         ep.act = op.act;
         ep.out_dtype = op.out_dtype;
-        if (op.kind == CADNN_OP_FC) return cadnn_fc(op.w, src, si.n, dst, &ep, st);
-        return cadnn_conv2d(op.w, src, si.n, si.h, si.w, dst, &ep, st);
+        if (op.kind == CADNN_OP_FC) return conv2d_impl(op.w, src, si.n, 1, 1, dst, &ep, pdl, st);
+        return conv2d_impl(op.w, src, si.n, si.h, si.w, dst, &ep, pdl, st);
     }
     if (op.kind == CADNN_OP_MAXPOOL)
-        return cadnn_maxpool2d(src, si.n, si.h, si.w, si.c, op.pool_k, op.pool_stride, op.pool_pad, si.dtype, dst, st);
+        return launch_maxpool(src, si.n, si.h, si.w, si.c, op.pool_k, op.pool_stride, op.pool_pad, si.dtype, dst, pdl, st);
     if (op.kind == CADNN_OP_GAVGPOOL)
-        return cadnn_global_avgpool((const float *)src, si.n, si.h, si.w, si.c, (float *)dst, st);
+        return launch_gavgpool((const float *)src, si.n, si.h, si.w, si.c, (float *)dst, pdl, st);
     return CADNN_E_ARG;
 }
 
+// Every op after the first is launched as a programmatic dependent of its predecessor: its
+// prologue (weights, tables) overlaps the predecessor's tail, and it waits on the grid
+// dependency before touching activations.
 cadnn_status run_all(cadnn_net *net, const void *x, void *y, cudaStream_t st)
 {
+    bool first = true;
     for (const cadnn_op &op : net->ops) {
-        cadnn_status s = run_op(net, op, x, y, st);
+        cadnn_status s = run_op(net, op, x, y, st, net->use_pdl && !first);
         if (s != CADNN_OK) return s;
+        first = false;
     }
     return CADNN_OK;
 }
@@ -132,6 +139,7 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
     if (in_dtype != CADNN_F32 && in_dtype != CADNN_S8) return CADNN_E_DTYPE;
     cadnn_net *net = new (std::nothrow) cadnn_net();
     if (!net) return CADNN_E_ALLOC;
+    net->use_pdl = getenv("CADNN_NO_PDL") == nullptr;   // tuning switch: plain stream order between layers
     cadnn_status st = CADNN_OK;
     int max_slot = 0;
     for (int i = 0; i < n_ops; ++i) {
@@ -233,28 +241,54 @@ cadnn_status cadnn_net_info(const cadnn_net *net, int *n_launches, int64_t *work
     return CADNN_OK;
 }
 
-cadnn_status cadnn_net_layer_times(cadnn_net *net, const void *x, void *y, int flush_l2, float *ms, void *stream)
+cadnn_status cadnn_net_layer_times(cadnn_net *net, const void *x, void *y, int flush_l2, int reps, float *ms,
+                                   void *stream)
 {
-    if (!net || !x || !y || !ms) return CADNN_E_ARG;
+    if (!net || !x || !y || !ms || reps < 1) return CADNN_E_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const size_t nops = net->ops.size();
     if (flush_l2 && !net->flush) {
         net->flush_bytes = 256u << 20;
         CADNN_CUDA_TRY(cudaMalloc(&net->flush, net->flush_bytes));
     }
-    std::vector<cudaEvent_t> ev(2 * nops);
-    for (auto &e : ev) CADNN_CUDA_TRY(cudaEventCreate(&e));
-    cadnn_status s = CADNN_OK;
+    // one pass in order so that every slot holds real data
+    cadnn_status s = run_all(net, x, y, st);
+    if (s != CADNN_OK) return s;
+    CADNN_CUDA_TRY(cudaStreamSynchronize(st));
+    cudaStream_t cap;
+    CADNN_CUDA_TRY(cudaStreamCreateWithFlags(&cap, cudaStreamNonBlocking));
+    cudaEvent_t e0, e1;
+    cudaEventCreate(&e0);
+    cudaEventCreate(&e1);
     for (size_t i = 0; i < nops && s == CADNN_OK; ++i) {
-        if (flush_l2) flush_kernel<<<148 * 8, 256, 0, st>>>((float *)net->flush, net->flush_bytes / 4);
-        cudaEventRecord(ev[2 * i], st);
-        s = run_op(net, net->ops[i], x, y, st);
-        cudaEventRecord(ev[2 * i + 1], st);
+        // a graph of `reps` back-to-back launches of this op: the host launch cost stays out of the timing
+        cudaGraph_t g = nullptr;
+        cudaGraphExec_t ge = nullptr;
+        cudaError_t e = cudaStreamBeginCapture(cap, cudaStreamCaptureModeThreadLocal);
+        if (e != cudaSuccess) { s = cadnn_note_cuda(e); break; }
+        for (int r = 0; r < reps && s == CADNN_OK; ++r) s = run_op(net, net->ops[i], x, y, cap);
+        e = cudaStreamEndCapture(cap, &g);
+        if (s == CADNN_OK && e != cudaSuccess) s = cadnn_note_cuda(e);
+        if (s == CADNN_OK && (e = cudaGraphInstantiate(&ge, g, 0)) != cudaSuccess) s = cadnn_note_cuda(e);
+        if (s == CADNN_OK) {
+            if (flush_l2) flush_kernel<<<148 * 8, 256, 0, st>>>((float *)net->flush, net->flush_bytes / 4);
+            else cudaGraphLaunch(ge, st);   // warm
+            cudaEventRecord(e0, st);
+            cudaGraphLaunch(ge, st);
+            cudaEventRecord(e1, st);
+            e = cudaStreamSynchronize(st);
+            if (e != cudaSuccess) s = cadnn_note_cuda(e);
+            else {
+                cudaEventElapsedTime(&ms[i], e0, e1);
+                ms[i] /= (float)reps;
+            }
+        }
+        if (ge) cudaGraphExecDestroy(ge);
+        if (g) cudaGraphDestroy(g);
     }
-    cudaError_t e = cudaStreamSynchronize(st);
-    if (s == CADNN_OK && e != cudaSuccess) s = cadnn_note_cuda(e);
-    for (size_t i = 0; i < nops && s == CADNN_OK; ++i) cudaEventElapsedTime(&ms[i], ev[2 * i], ev[2 * i + 1]);
-    for (auto &ev1 : ev) cudaEventDestroy(ev1);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    cudaStreamDestroy(cap);
     return s;
 }
 

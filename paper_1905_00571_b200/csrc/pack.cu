@@ -5,11 +5,14 @@
 // compressed layout whose element offsets already point into the shared-memory
 // activation tile the kernel stages, padded so that a warp's loads never collide
 // on a bank - and "Optimization parameters selection" - tile sizes, the channel
-// chunk and the number of filters per warp are chosen per layer from its shape.
-// Filters are regrouped so that the warps of a block get equal nonzero counts
-// (the load-balance obstacle Section 1 names).
+// chunk, the filters per warp and the split of the reduction over a thread-block
+// cluster are chosen per layer from its shape, by a time model or by timing the
+// candidates on the device.  Filters are regrouped so that the warps of a block
+// get equal nonzero counts (the load-balance obstacle Section 1 names).
 #include <algorithm>
 #include <cmath>
+#include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <numeric>
@@ -18,115 +21,128 @@
 namespace {
 
 const int kSmCount = 148;
-const int kTileSmemBudget = 72 * 1024;   // activation tile bytes per block (two blocks per SM)
-const int kWeightSmemBudget = 40 * 1024; // staged nonzeros per (block, chunk)
+const int kSmemPerSm = 200 * 1024;        // shared memory the schedule lets resident blocks use per SM
+const int kMaxStageBytes = 100 * 1024;
 
 int round_up(int v, int m) { return (v + m - 1) / m * m; }
 int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
-int pick_T(int npix)
-{
-    static const int allowed[] = {1, 2, 4, 7, 8};
-    int need = ceil_div(npix, 32);
-    for (int t : allowed)
-        if (t >= need) return t;
-    return 8;
-}
-
-// Row pitch (in pixels) of the staged input tile: at least `need`, and congruent
-// to TW modulo 32 so that lanes walking consecutive output pixels across a row
-// boundary still touch 32 distinct banks.
-int pick_pitch(int need, int TW)
-{
-    int p = need;
-    while (((p - TW) % 32) != 0) ++p;
-    return p;
-}
-
 struct Geometry {
     int c_in, c_out, kh, kw, stride, pad, h, w, h_out, w_out;
+    bool s8;
+    double nnz;   // stored nonzeros of the layer
 };
 
-void choose_spatial(const Geometry &g, int batch_hint, Schedule &s)
+// Bytes per staged pixel: an odd number of 32-bit words, so that lanes reading the
+// same channel of consecutive pixels touch distinct banks.
+int pixel_pitch_bytes(int cic, bool s8)
 {
-    s.kind = KK_SCONV_SPATIAL;
-    s.TW = g.w_out <= 256 ? g.w_out : 128;
-    int th_max = std::max(1, 256 / s.TW);
-    th_max = std::min(th_max, g.h_out);
-    int tiles_y = ceil_div(g.h_out, th_max);
-    s.TH = ceil_div(g.h_out, tiles_y);
-    s.T = pick_T(s.TH * s.TW);
-    s.IH_t = (s.TH - 1) * g.stride + g.kh;
-    s.IW_t = (s.TW - 1) * g.stride + g.kw;
-    s.pitch = pick_pitch(s.IW_t, s.TW);
-    long tiles = (long)batch_hint * tiles_y * ceil_div(g.w_out, s.TW);
-    s.RPW = 1;
-    for (int rpw : {4, 2}) {
-        if (tiles * ceil_div(g.c_out, kWarpsPerBlock * rpw) >= 2L * kSmCount) {
-            s.RPW = rpw;
-            break;
-        }
-    }
-    s.G = kWarpsPerBlock * s.RPW;
-    int cic = 64;
-    while (cic > 4 && cic / 2 >= g.c_in) cic /= 2;          // do not stage far more channels than exist
-    if (g.c_in < 4) cic = g.c_in;
-    for (;;) {
-        s.CIc = cic;
-        s.PP = cic | 1;
-        long words = (long)s.IH_t * s.pitch * s.PP;
-        if ((words * 4 <= kTileSmemBudget && words <= 65535) || cic <= 1) break;
-        cic = cic > 4 ? cic / 2 : cic - 1;
-    }
-    s.tile_words = s.IH_t * s.pitch * s.PP;
+    int words = s8 ? ceil_div(cic, 4) : cic;
+    return 4 * (words | 1);
 }
 
-void choose_linear(const Geometry &g, int batch_hint, Schedule &s)
+// Smallest staged row pitch (pixels) >= need for which one band - RB rows of BW
+// consecutive pixels, rows row_step * pitch apart - touches RB * BW distinct banks.
+int pick_pitch(int need, int BW, int RB, int row_step)
 {
-    s.kind = KK_SCONV_LINEAR;
-    long P = (long)batch_hint * g.h_out * g.w_out;
-    s.RPW = 1;
-    s.T = 1;
-    bool done = false;
-    for (int rpw : {4, 2, 1}) {
-        for (int t : {8, 4, 2, 1}) {
-            long ctas = ((P + 32 * t - 1) / (32 * t)) * ceil_div(g.c_out, kWarpsPerBlock * rpw);
-            if (ctas >= 2L * kSmCount || (rpw == 1 && t == 1)) {
-                s.RPW = rpw;
-                s.T = t;
-                done = true;
-                break;
+    for (int p = need; p < need + 64; ++p) {
+        bool used[32] = {false};
+        bool ok = true;
+        for (int r = 0; r < RB && ok; ++r)
+            for (int x = 0; x < BW; ++x) {
+                int b = (r * row_step * p + x) & 31;
+                if (used[b]) { ok = false; break; }
+                used[b] = true;
             }
-        }
-        if (done) break;
+        if (ok) return p;
     }
-    // never give a lane more pixels than the layer has
-    while (s.T > 1 && 32L * (s.T / 2) >= P) s.T /= 2;
-    s.G = kWarpsPerBlock * s.RPW;
-    int cic = 64;
-    while (cic > 4 && cic / 2 >= g.c_in) cic /= 2;
-    if (g.c_in < 4) cic = g.c_in;
-    s.CIc = cic;
-    s.PP = cic | 1;
-    s.TH = 1;
-    s.TW = 32 * s.T;
-    s.pitch = s.IH_t = s.IW_t = 0;
-    s.tile_words = 32 * s.T * s.PP;
+    return need;
 }
 
-void finish_smem(Schedule &s)
+// Derived fields of a candidate (everything but the entry counts).
+bool finish_candidate(const Geometry &g, Schedule &s, bool linear)
 {
-    s.tile_words = round_up(s.tile_words, 4);
-    int work = s.tile_words * 4 + s.max_entries * 8 + round_up((s.G + 1) * 4, 16);
-    int out = 32 * s.T * (s.G + 1) * 4;
-    s.smem_bytes = std::max(work, out);
+    s.G = s.NW * s.RPW;
+    s.T = s.TBX * s.TBY;
+    if (s.T < 1 || s.T > 8) return false;
+    s.n_groups = ceil_div(g.c_out, s.G);
+    s.PPb = pixel_pitch_bytes(s.CIc, g.s8);
+    s.n_chunks = ceil_div(g.c_in, s.CIc);
+    if (s.ksplit < 1 || s.ksplit > 8 || s.ksplit > s.n_chunks) return false;
+    if (linear) {
+        s.BW = 32; s.RB = 1; s.TBX = s.T; s.TBY = 1;
+        s.TH = 1; s.TW = 32 * s.T;
+        s.pitch = s.half = s.IH_t = s.IW_t = 0;
+        s.tile_bytes = 32 * s.T * s.PPb;
+    } else {
+        s.TH = s.TBY * s.RB;
+        s.TW = s.TBX * s.BW;
+        s.IH_t = (s.TH - 1) * g.stride + g.kh;
+        s.IW_t = (s.TW - 1) * g.stride + g.kw;
+        if (g.stride == 2) {
+            s.half = ceil_div(s.IW_t, 2);
+            s.pitch = pick_pitch(2 * s.half, s.BW, s.RB, 2);
+        } else {
+            s.half = 0;
+            s.pitch = pick_pitch(s.IW_t, s.BW, s.RB, g.stride);
+        }
+        s.tile_bytes = s.IH_t * s.pitch * s.PPb;
+    }
+    s.tile_bytes = round_up(s.tile_bytes, 16);
+    return true;
 }
 
-struct Entry {
-    uint16_t off;
-    float v;
-    int8_t q;
-};
+int header_words(const Schedule &s) { return round_up(s.G + 1, 4); }
+
+void finish_smem(Schedule &s, bool s8)
+{
+    int ew = s8 ? 4 : 8;
+    s.stage_bytes = s.tile_bytes + header_words(s) * 4 + round_up(s.max_entries * ew, 16);
+    int out = 32 * s.T * (s.G + 1) * 4;
+    int per_block = ceil_div(s.n_chunks, s.ksplit);   // chunks one block walks
+    s.stages = (3 * s.stage_bytes <= 72 * 1024 && per_block >= 3) ? 3 : 2;
+    if (per_block == 1) s.stages = 1;
+    int npx = s.kind == KK_SCONV_LINEAR ? 32 * s.T : s.IH_t * s.IW_t;
+    int tables = npx * 8 + 2 * s.G * 4;
+    s.smem_bytes = round_up(std::max(s.stages * s.stage_bytes, out), 16) + round_up(tables, 16);
+}
+
+// Rough time model (SM clocks) of one candidate: the kernel is bound by shared-memory
+// wavefronts (one per 32 multiply-adds plus the broadcast of each nonzero), by issue
+// slots, by the bytes each block pulls through L2, and by per-block fixed latencies.
+double estimate_clocks(const Geometry &g, const Schedule &s, int batch, bool linear)
+{
+    double tiles;
+    double in_px;
+    if (linear) {
+        double P = (double)batch * g.h_out * g.w_out;
+        tiles = std::ceil(P / (32.0 * s.T));
+        in_px = 32.0 * s.T;
+    } else {
+        tiles = (double)batch * ceil_div(g.h_out, s.TH) * ceil_div(g.w_out, s.TW);
+        in_px = (double)s.IH_t * s.IW_t;
+    }
+    const double KS = s.ksplit;
+    double ctas = tiles * s.n_groups * KS;
+    double nnz_cta = g.nnz * s.G / std::max(1, g.c_out) / KS;
+    double cin_cta = std::min((double)g.c_in, (double)ceil_div(s.n_chunks, s.ksplit) * s.CIc);
+    double esz = g.s8 ? 1.0 : 4.0;
+    double units = in_px * cin_cta / (g.s8 ? 4.0 : 1.0);          // 4-byte staging copies
+    double wf = nnz_cta * (s.T + 0.5) + units / 32.0 * 4.0 + 32.0 * s.T * s.G / 32.0 * (2.0 + KS);
+    double instr = (nnz_cta * (2.2 * s.T + 3.0) + units / 32.0 * 12.0 + 32.0 * s.T * s.G / 32.0 * 30.0) / 4.0;
+    double l2 = (in_px * cin_cta * esz + nnz_cta * (g.s8 ? 4.0 : 8.0) + 32.0 * s.T * s.G * 4.0) / 40.0;
+    int by_smem = std::max(1, kSmemPerSm / std::max(1, s.smem_bytes));
+    int by_thr = std::max(1, 2048 / (s.NW * 32));
+    int resident = std::min(std::min(by_smem, by_thr), 8);
+    double per_sm = std::ceil(ctas / kSmCount);
+    double in_round = std::min((double)resident, per_sm);
+    double warps = in_round * s.NW;
+    double ipc_eff = std::min(1.0, warps / 24.0);                  // few warps cannot fill the issue slots
+    double busy = std::max(std::max(wf, instr / std::max(0.15, ipc_eff)), l2);
+    double fixed = 3000.0 + 500.0 * ceil_div(s.n_chunks, s.ksplit) + (KS > 1 ? 1500.0 : 0.0);
+    double rounds = std::ceil(per_sm / resident);
+    return rounds * std::max(in_round * busy, busy + fixed);
+}
 
 // Longest-processing-time assignment of the G filters of one block to the warps,
 // RPW filters each; returns, per warp slot, the local filter index (or -1).
@@ -156,10 +172,10 @@ cadnn_status upload(cadnn_weights *h)
     auto al = [](size_t b) { return (b + 255) / 256 * 256; };
     size_t b_vals = h->desc.dtype == CADNN_S8 ? h->vals_q.size() : h->vals_f.size() * 4;
     size_t b_offs = h->offs.size() * 2, b_ptr = h->ptr.size() * 4, b_perm = h->perm.size() * 4;
-    size_t b_dense = h->dense_f.size() * 4;
+    size_t b_dense = h->dense_f.size() * 4, b_ent = h->ent.size() * 4;
     size_t o_vals = 0, o_offs = o_vals + al(b_vals), o_ptr = o_offs + al(b_offs), o_perm = o_ptr + al(b_ptr);
-    size_t o_dense = o_perm + al(b_perm), total = o_dense + al(b_dense);
-    h->packed_bytes = (int64_t)(b_vals + b_offs + b_ptr + b_perm + b_dense);
+    size_t o_dense = o_perm + al(b_perm), o_ent = o_dense + al(b_dense), total = o_ent + al(b_ent);
+    h->packed_bytes = (int64_t)(b_vals + b_offs + b_ptr + b_perm + b_dense + b_ent);
     if (h->desc.flags & CADNN_PACK_HOST_ONLY) return CADNN_OK;
     if (total == 0) total = 256;
     CADNN_CUDA_TRY(cudaGetDevice(&h->device));
@@ -175,6 +191,8 @@ cadnn_status upload(cadnn_weights *h)
     if (b_ptr) CADNN_CUDA_TRY(cudaMemcpy(base + o_ptr, h->ptr.data(), b_ptr, cudaMemcpyHostToDevice));
     if (b_perm) CADNN_CUDA_TRY(cudaMemcpy(base + o_perm, h->perm.data(), b_perm, cudaMemcpyHostToDevice));
     if (b_dense) CADNN_CUDA_TRY(cudaMemcpy(base + o_dense, h->dense_f.data(), b_dense, cudaMemcpyHostToDevice));
+    if (b_ent) CADNN_CUDA_TRY(cudaMemcpy(base + o_ent, h->ent.data(), b_ent, cudaMemcpyHostToDevice));
+    h->d_ent = (const uint32_t *)(base + o_ent);
     h->d_vals = base + o_vals;
     h->d_offs = (const uint16_t *)(base + o_offs);
     h->d_ptr = (const int32_t *)(base + o_ptr);
@@ -203,28 +221,105 @@ struct Src {
     }
 };
 
-cadnn_status pack_sconv(cadnn_weights *h, const Src &src)
+struct Candidate {
+    Schedule s;
+    double t;
+};
+
+// Candidate schedules for a layer, best first by the time model.
+void enumerate_schedules(const Geometry &g, int batch, bool linear, std::vector<Candidate> &out)
+{
+    out.clear();
+    // band shape follows the output width
+    int BW, RB, nbx_total;
+    if (linear) {
+        BW = 32; RB = 1; nbx_total = 1;
+    } else if (g.w_out <= 32) {
+        BW = g.w_out;
+        RB = std::max(1, std::min(32 / BW, g.h_out));
+        nbx_total = 1;
+    } else {
+        nbx_total = ceil_div(g.w_out, 32);
+        BW = ceil_div(g.w_out, nbx_total);
+        RB = 1;
+    }
+    // channel-chunk candidates: powers of two up to 512, never far beyond the layer's channels
+    std::vector<int> cics;
+    if (g.s8) {
+        for (int c = 512; c >= 4; c /= 2)
+            if (c == 4 || c / 2 < g.c_in) cics.push_back(c);
+    } else if (g.c_in < 4) {
+        cics.push_back(g.c_in);
+    } else {
+        for (int c = 512; c >= 4; c /= 2)
+            if (c == 4 || c / 2 < g.c_in) cics.push_back(std::min(c, g.c_in));
+    }
+    const int tbx_full = std::min(8, nbx_total);
+    for (int nw : {16, 8, 4})
+        for (int rpw : {4, 2, 1})
+            for (int cic : cics)
+                for (int ks : {1, 2, 4, 8})
+                    for (int tbx = 1; tbx <= (linear ? 8 : tbx_full); ++tbx)
+                        for (int tby = 1; tby * tbx <= 8; ++tby) {
+                            if (linear && tby > 1) break;
+                            if (!linear && tbx != tbx_full && tbx != 1 && tbx * 2 != tbx_full) continue;
+                            if (!linear && (tby - 1) * RB >= g.h_out) break;
+                            Schedule s;
+                            s.kind = linear ? KK_SCONV_LINEAR : KK_SCONV_SPATIAL;
+                            s.NW = nw; s.RPW = rpw; s.CIc = cic; s.ksplit = ks;
+                            s.BW = BW; s.RB = RB; s.TBX = tbx; s.TBY = tby;
+                            if (!finish_candidate(g, s, linear)) continue;
+                            // expected entries per (chunk, block) record, with headroom; the real count is set when packing
+                            double per_chunk = g.nnz / std::max(1, g.c_out) * s.G / s.n_chunks;
+                            s.max_entries = (int)(per_chunk * 1.3) + 2 * s.G + 16;
+                            finish_smem(s, g.s8);
+                            if (s.stage_bytes > kMaxStageBytes || s.smem_bytes > kSmemPerSm) continue;
+                            out.push_back({s, estimate_clocks(g, s, batch, linear)});
+                        }
+    std::stable_sort(out.begin(), out.end(), [](const Candidate &a, const Candidate &b) { return a.t < b.t; });
+    if (out.empty()) {   // nothing fit: smallest everything
+        Schedule s;
+        s.kind = linear ? KK_SCONV_LINEAR : KK_SCONV_SPATIAL;
+        s.NW = 4; s.RPW = 1; s.CIc = g.s8 ? 4 : 1; s.BW = BW; s.RB = RB; s.TBX = 1; s.TBY = 1;
+        finish_candidate(g, s, linear);
+        out.push_back({s, 0.0});
+    }
+}
+
+// Manual override for tuning: CADNN_SCHEDULE="nw=4,rpw=1,tbx=1,tby=2,cic=32,ks=2" (unset keys keep the model's pick).
+void apply_env_override(const Geometry &g, bool linear, Schedule &best)
+{
+    const char *env = getenv("CADNN_SCHEDULE");
+    if (!env) return;
+    Schedule s = best;
+    int v;
+    const char *q;
+    if ((q = strstr(env, "nw=")) && sscanf(q + 3, "%d", &v) == 1 && (v == 4 || v == 8 || v == 16)) s.NW = v;
+    if ((q = strstr(env, "rpw=")) && sscanf(q + 4, "%d", &v) == 1 && (v == 1 || v == 2 || v == 4)) s.RPW = v;
+    if ((q = strstr(env, "tbx=")) && sscanf(q + 4, "%d", &v) == 1 && v >= 1 && v <= 8) s.TBX = v;
+    if ((q = strstr(env, "tby=")) && sscanf(q + 4, "%d", &v) == 1 && v >= 1 && v <= 8) s.TBY = v;
+    if ((q = strstr(env, "cic=")) && sscanf(q + 4, "%d", &v) == 1 && v >= 1 && v <= 512 && (!g.s8 || v % 4 == 0))
+        s.CIc = std::min(v, g.s8 ? round_up(g.c_in, 4) : g.c_in);
+    if ((q = strstr(env, "ks=")) && sscanf(q + 3, "%d", &v) == 1 && (v == 1 || v == 2 || v == 4 || v == 8)) s.ksplit = v;
+    if (linear) { s.TBX = std::min(8, s.TBX * s.TBY); s.TBY = 1; }
+    s.ksplit = std::min(s.ksplit, ceil_div(g.c_in, s.CIc));
+    if (finish_candidate(g, s, linear)) best = s;
+}
+
+// Build the packed image of a conv layer for schedule h->s (already through finish_candidate).
+cadnn_status build_sconv_image(cadnn_weights *h, const Src &src, const Geometry &g,
+                               const std::vector<int64_t> &row_nnz)
 {
     const cadnn_layer_desc &d = h->desc;
-    Geometry g{d.c_in, d.c_out, d.kh, d.kw, d.stride, d.pad, d.in_h, d.in_w, h->h_out, h->w_out};
     Schedule &s = h->s;
-    const bool linear = (d.kh == 1 && d.kw == 1 && d.pad == 0);
-    const int K = d.kh * d.kw * d.c_in;
-    int bh = std::max(1, d.batch_hint);
-    if (linear) choose_linear(g, bh, s); else choose_spatial(g, bh, s);
-
-    // per-filter nonzero counts, then the balanced regrouping
-    std::vector<int64_t> row_nnz(d.c_out, 0);
-    for (int co = 0; co < d.c_out; ++co) {
-        int64_t c = 0;
-        for (int k = 0; k < K; ++k) c += src.kept((size_t)co * K + k);
-        row_nnz[co] = c;
-        h->nnz += c;
-    }
+    const bool linear = s.kind == KK_SCONV_LINEAR;
+    const bool s8 = src.s8;
+    const int ew = s8 ? 1 : 2;   // 32-bit words per entry
     for (int attempt = 0;; ++attempt) {
         s.n_groups = ceil_div(d.c_out, s.G);
         h->c_pad = s.n_groups * s.G;
         s.n_chunks = ceil_div(d.c_in, s.CIc);
+        // balanced regrouping of the filters of each block over its warps
         h->perm.assign(h->c_pad, -1);
         for (int gi = 0; gi < s.n_groups; ++gi) {
             int lo = gi * s.G, hi = std::min(d.c_out, lo + s.G);
@@ -234,56 +329,96 @@ cadnn_status pack_sconv(cadnn_weights *h, const Src &src)
             for (int sl = 0; sl < s.G; ++sl)
                 if (slot[sl] >= 0) h->perm[lo + sl] = lo + slot[sl];
         }
-        // entries, chunk-major then packed-row-major
-        h->ptr.assign((size_t)s.n_chunks * (h->c_pad + 1), 0);
-        h->vals_f.clear();
-        h->vals_q.clear();
-        h->offs.clear();
-        h->vals_f.reserve(src.s8 ? 0 : (size_t)h->nnz);
-        h->vals_q.reserve(src.s8 ? (size_t)h->nnz : 0);
-        h->offs.reserve((size_t)h->nnz);
+        // One record per (chunk, block of G filters): a header of G + 1 row starts (in entries)
+        // followed by the entries, every row padded to an even count.  All records get the
+        // same size, so a thread block finds its nonzeros without reading a pointer first.
+        const int hdr_words = header_words(s);
+        std::vector<std::vector<uint32_t>> blocks((size_t)s.n_chunks * s.n_groups);
+        h->cnt.assign((size_t)s.n_chunks * h->c_pad, 0);
         s.max_entries = 0;
-        int32_t running = 0;
         for (int c = 0; c < s.n_chunks; ++c) {
             int c0 = c * s.CIc, c1 = std::min(d.c_in, c0 + s.CIc);
-            int32_t *pp = &h->ptr[(size_t)c * (h->c_pad + 1)];
-            for (int r = 0; r < h->c_pad; ++r) {
-                pp[r] = running;
-                int co = h->perm[r];
-                if (co >= 0) {
-                    for (int ky = 0; ky < d.kh; ++ky)
-                        for (int kx = 0; kx < d.kw; ++kx)
-                            for (int ci = c0; ci < c1; ++ci) {
-                                size_t wi = (((size_t)co * d.kh + ky) * d.kw + kx) * d.c_in + ci;
-                                if (!src.kept(wi)) continue;
-                                int off = linear ? (ci - c0) : ((ky * s.pitch + kx) * s.PP + (ci - c0));
-                                h->offs.push_back((uint16_t)off);
-                                if (src.s8) h->vals_q.push_back(src.qval(wi, co));
-                                else h->vals_f.push_back(src.fval(wi));
-                                ++running;
-                            }
+            for (int gi = 0; gi < s.n_groups; ++gi) {
+                std::vector<uint32_t> &blk = blocks[(size_t)c * s.n_groups + gi];
+                blk.assign(hdr_words, 0u);
+                int running = 0;
+                for (int sl = 0; sl < s.G; ++sl) {
+                    const int r = gi * s.G + sl;
+                    blk[sl] = (uint32_t)running;
+                    int co = h->perm[r];
+                    int real = 0;
+                    if (co >= 0) {
+                        for (int ky = 0; ky < d.kh; ++ky)
+                            for (int kx = 0; kx < d.kw; ++kx)
+                                for (int ci = c0; ci < c1; ++ci) {
+                                    size_t wi = (((size_t)co * d.kh + ky) * d.kw + kx) * d.c_in + ci;
+                                    if (!src.kept(wi)) continue;
+                                    int pos = kx;
+                                    if (!linear && s.half) pos = (kx & 1) * s.half + (kx >> 1);
+                                    uint32_t off = linear ? 0u : (uint32_t)(ky * s.pitch + pos) * (uint32_t)s.PPb;
+                                    off += (uint32_t)(ci - c0) * (s8 ? 1u : 4u);
+                                    if (s8) {
+                                        blk.push_back((off << 8) | (uint32_t)(uint8_t)src.qval(wi, co));
+                                    } else {
+                                        float v = src.fval(wi);
+                                        uint32_t bits;
+                                        memcpy(&bits, &v, 4);
+                                        blk.push_back(bits);
+                                        blk.push_back(off);
+                                    }
+                                    ++real;
+                                }
+                        if (real & 1) {   // padding entry: weight 0 at offset 0
+                            blk.push_back(0u);
+                            if (!s8) blk.push_back(0u);
+                        }
+                    }
+                    h->cnt[(size_t)c * h->c_pad + r] = real;
+                    running += real + (real & 1);
                 }
-                if ((r + 1) % s.G == 0) {
-                    int first = pp[r + 1 - s.G];
-                    s.max_entries = std::max(s.max_entries, running - first);
-                }
+                blk[s.G] = (uint32_t)running;
+                s.max_entries = std::max(s.max_entries, running);
             }
-            pp[h->c_pad] = running;
         }
-        // Dense or nearly dense layers can overflow the staged-weight budget: halve the chunk.
-        if (s.max_entries * 8 > kWeightSmemBudget && s.CIc > 1 && attempt < 8) {
-            s.CIc = std::max(1, s.CIc / 2);
-            s.PP = s.CIc | 1;
-            s.tile_words = linear ? 32 * s.T * s.PP : s.IH_t * s.pitch * s.PP;
+        s.max_entries = round_up(std::max(s.max_entries, 2), 4);
+        finish_smem(s, s8);
+        // A dense or skewed layer can overflow the stage budget: halve the chunk and repack.
+        if ((s.stage_bytes > kMaxStageBytes || s.smem_bytes > kSmemPerSm) && s.CIc > (s8 ? 4 : 1) && attempt < 8) {
+            s.CIc = std::max(s8 ? 4 : 1, s.CIc / 2);
+            finish_candidate(g, s, linear);
             continue;
         }
+        const int block_words = hdr_words + s.max_entries * ew;
+        h->ent.assign((size_t)block_words * blocks.size(), 0u);
+        for (size_t b = 0; b < blocks.size(); ++b)
+            std::copy(blocks[b].begin(), blocks[b].end(), h->ent.begin() + b * block_words);
         break;
     }
-    s.max_entries = round_up(std::max(s.max_entries, 1), 2);
-    finish_smem(s);
-    if (s.smem_bytes > 200 * 1024) return CADNN_E_UNSUPPORTED;
+    if (s.smem_bytes > 220 * 1024) return CADNN_E_UNSUPPORTED;
+    if (s8 && (uint64_t)s.tile_bytes >= (1u << 24)) return CADNN_E_UNSUPPORTED;
     h->fmt = CADNN_FMT_TILED_CSR;
     return CADNN_OK;
+}
+
+cadnn_status pack_sconv(cadnn_weights *h, const Src &src)
+{
+    const cadnn_layer_desc &d = h->desc;
+    const bool linear = (d.kh == 1 && d.kw == 1 && d.pad == 0);
+    const int K = d.kh * d.kw * d.c_in;
+    int bh = std::max(1, d.batch_hint);
+    std::vector<int64_t> row_nnz(d.c_out, 0);
+    for (int co = 0; co < d.c_out; ++co) {
+        int64_t c = 0;
+        for (int k = 0; k < K; ++k) c += src.kept((size_t)co * K + k);
+        row_nnz[co] = c;
+        h->nnz += c;
+    }
+    Geometry g{d.c_in, d.c_out, d.kh, d.kw, d.stride, d.pad, d.in_h, d.in_w, h->h_out, h->w_out, src.s8, (double)h->nnz};
+    std::vector<Candidate> cands;
+    enumerate_schedules(g, bh, linear, cands);
+    h->s = cands[0].s;
+    apply_env_override(g, linear, h->s);
+    return build_sconv_image(h, src, g, row_nnz);
 }
 
 cadnn_status pack_fc_spmv(cadnn_weights *h, const Src &src)
@@ -295,6 +430,7 @@ cadnn_status pack_fc_spmv(cadnn_weights *h, const Src &src)
     s.kind = KK_FC_SPMV;
     s.T = 1;
     s.RPW = 1;
+    s.NW = kWarpsPerBlock;
     s.G = kWarpsPerBlock;
     s.n_groups = ceil_div(d.c_out, s.G);
     h->c_pad = s.n_groups * s.G;
@@ -425,11 +561,12 @@ cadnn_status cadnn_weights_info(const cadnn_weights *w, int64_t *nnz, int64_t *p
     return CADNN_OK;
 }
 
-cadnn_status cadnn_weights_schedule(const cadnn_weights *w, int sched[8])
+cadnn_status cadnn_weights_schedule(const cadnn_weights *w, int sched[16])
 {
     if (!w || !sched) return CADNN_E_ARG;
     const Schedule &s = w->s;
-    int v[8] = {s.kind, s.T, s.RPW, s.G, s.CIc, s.TH, s.TW, s.pitch};
+    int v[16] = {s.kind, s.T, s.RPW, s.G, s.CIc, s.TH, s.TW, s.pitch, s.NW, s.stages, s.ksplit, s.n_chunks,
+                 s.smem_bytes, s.TBX, s.TBY, s.max_entries};
     memcpy(sched, v, sizeof(v));
     return CADNN_OK;
 }
@@ -449,8 +586,11 @@ cadnn_status cadnn_weights_warp_loads(const cadnn_weights *w, int64_t *loads, in
     for (int i = 0; i < n_warps && i < cap; ++i) {
         int64_t tot = 0;
         for (int c = 0; c < chunks; ++c) {
-            const int32_t *pp = &w->ptr[(size_t)c * (w->c_pad + 1)];
-            tot += pp[(i + 1) * s.RPW] - pp[i * s.RPW];
+            if (s.kind == KK_FC_SPMV) {
+                tot += w->ptr[(i + 1) * s.RPW] - w->ptr[i * s.RPW];
+            } else {
+                for (int j = 0; j < s.RPW; ++j) tot += w->cnt[(size_t)c * w->c_pad + i * s.RPW + j];
+            }
         }
         loads[i] = tot;
     }
@@ -488,17 +628,40 @@ cadnn_status cadnn_weights_unpack(const cadnn_weights *w, float *dense, uint8_t 
         return CADNN_OK;
     }
     const bool linear = s.kind == KK_SCONV_LINEAR;
+    const bool s8 = d.dtype == CADNN_S8;
+    const int ew = s8 ? 1 : 2;
+    const int hdr_words = header_words(s);
+    const size_t block_words = (size_t)hdr_words + (size_t)s.max_entries * ew;
     for (int c = 0; c < s.n_chunks; ++c) {
-        const int32_t *pp = &w->ptr[(size_t)c * (w->c_pad + 1)];
         for (int r = 0; r < w->c_pad; ++r) {
             int co = w->perm[r];
             if (co < 0) continue;
-            for (int e = pp[r]; e < pp[r + 1]; ++e) {
-                int off = w->offs[e];
-                int cl = off % s.PP, t = off / s.PP;
-                int kx = linear ? 0 : t % s.pitch, ky = linear ? 0 : t / s.pitch;
+            const uint32_t *blk = &w->ent[((size_t)c * s.n_groups + r / s.G) * block_words];
+            const uint32_t *ents = blk + hdr_words;
+            const int real = w->cnt[(size_t)c * w->c_pad + r];
+            const int first = (int)blk[r % s.G];
+            for (int e = first; e < first + real; ++e) {
+                uint32_t off;
+                float v;
+                if (s8) {
+                    uint32_t word = ents[e];
+                    off = word >> 8;
+                    v = (float)(int8_t)(word & 0xffu);
+                } else {
+                    uint32_t bits = ents[(size_t)e * ew];
+                    memcpy(&v, &bits, 4);
+                    off = ents[(size_t)e * ew + 1];
+                }
+                int cl = (int)(off % (uint32_t)s.PPb) / (s8 ? 1 : 4);
+                int t = (int)(off / (uint32_t)s.PPb);
+                int kx = 0, ky = 0;
+                if (!linear) {
+                    int pos = t % s.pitch;
+                    ky = t / s.pitch;
+                    kx = s.half ? (pos >= s.half ? 2 * (pos - s.half) + 1 : 2 * pos) : pos;
+                }
                 size_t wi = (((size_t)co * d.kh + ky) * d.kw + kx) * d.c_in + (size_t)c * s.CIc + cl;
-                if (dense) dense[wi] = val(e);
+                if (dense) dense[wi] = v;
                 if (mask) mask[wi] = 1;
             }
         }

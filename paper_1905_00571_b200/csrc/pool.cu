@@ -11,6 +11,8 @@ __global__ void __launch_bounds__(256) maxpool_kernel(const XT *x, XT *y, int n,
                                                       int w_out, int k, int stride, int pad)
 {
     const long long total = (long long)n * h_out * w_out * c;
+    grid_dep_wait();
+    grid_dep_trigger();
     for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
          idx += (long long)gridDim.x * blockDim.x) {
         const int ch = (int)(idx % c);
@@ -39,6 +41,8 @@ __global__ void __launch_bounds__(256) maxpool_kernel(const XT *x, XT *y, int n,
 __global__ void __launch_bounds__(256) gavgpool_kernel(const float *x, float *y, int n, int hw, int c, float inv)
 {
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    grid_dep_wait();
+    grid_dep_trigger();
     if (idx >= n * c) return;
     const int b = idx / c, ch = idx - b * c;
     const float *src = x + (size_t)b * hw * c + ch;
@@ -50,7 +54,7 @@ __global__ void __launch_bounds__(256) gavgpool_kernel(const float *x, float *y,
 }  // namespace
 
 cadnn_status launch_maxpool(const void *x, int n, int h, int wd, int c, int k, int stride, int pad, int dtype,
-                            void *y, cudaStream_t st)
+                            void *y, bool pdl, cudaStream_t st)
 {
     const int h_out = (h + 2 * pad - k) / stride + 1, w_out = (wd + 2 * pad - k) / stride + 1;
     long long total = (long long)n * h_out * w_out * c;
@@ -58,19 +62,15 @@ cadnn_status launch_maxpool(const void *x, int n, int h, int wd, int c, int k, i
     long long blocks = (total + 255) / 256;
     if (blocks > 148LL * 64) blocks = 148LL * 64;
     if (dtype == CADNN_S8)
-        maxpool_kernel<int8_t><<<(int)blocks, 256, 0, st>>>((const int8_t *)x, (int8_t *)y, n, h, wd, c, h_out, w_out, k,
-                                                           stride, pad);
-    else
-        maxpool_kernel<float><<<(int)blocks, 256, 0, st>>>((const float *)x, (float *)y, n, h, wd, c, h_out, w_out, k,
-                                                          stride, pad);
-    CADNN_CUDA_TRY(cudaGetLastError());
-    return CADNN_OK;
+        return launch_kernel(maxpool_kernel<int8_t>, (int)blocks, 256, 0, pdl, st, (const int8_t *)x, (int8_t *)y, n, h,
+                             wd, c, h_out, w_out, k, stride, pad);
+    return launch_kernel(maxpool_kernel<float>, (int)blocks, 256, 0, pdl, st, (const float *)x, (float *)y, n, h, wd, c,
+                         h_out, w_out, k, stride, pad);
 }
 
-cadnn_status launch_gavgpool(const float *x, int n, int h, int wd, int c, float *y, cudaStream_t st)
+cadnn_status launch_gavgpool(const float *x, int n, int h, int wd, int c, float *y, bool pdl, cudaStream_t st)
 {
     if (n * c <= 0) return CADNN_OK;
-    gavgpool_kernel<<<(n * c + 255) / 256, 256, 0, st>>>(x, y, n, h * wd, c, 1.0f / (float)(h * wd));
-    CADNN_CUDA_TRY(cudaGetLastError());
-    return CADNN_OK;
+    return launch_kernel(gavgpool_kernel, (n * c + 255) / 256, 256, 0, pdl, st, x, y, n, h * wd, c,
+                         1.0f / (float)(h * wd));
 }

@@ -4,55 +4,69 @@
 // CADNN (arXiv 1905.00571), Section 4: the compressed layer is executed as one
 // fused kernel (Conv + BatchNorm + Activation), 1x1 filters are run as a matrix
 // product, and filter elements are not reloaded redundantly.  Here:
-//   * a thread block owns a tile of output pixels and a block of G filters;
-//   * the input tile is staged in shared memory chunk by chunk of input channels,
-//     pixel-major with an odd word pitch per pixel, so that the lanes of a warp
-//     (consecutive output pixels) read 32 distinct banks for any nonzero;
-//   * each stored nonzero is (value, offset into the staged tile); a warp walks
-//     the nonzeros of its filters, broadcasts one nonzero to all lanes and issues
-//     T multiply-adds per lane, the accumulators living in registers for the
-//     whole layer (each weight is read once per block and chunk);
+//   * a thread block owns a tile of output pixels and a block of G filters; the
+//     reduction over input channels can additionally be split over the blocks of a
+//     thread-block cluster, whose partial sums meet in distributed shared memory;
+//   * the input tile is staged in shared memory chunk by chunk of input channels
+//     with cp.async, pixel-major with an odd word pitch per pixel, so that the lanes
+//     of a warp (one band of up to 32 output pixels) read 32 distinct banks for any
+//     nonzero; stride-2 layers stage even and odd columns in separate planes for the
+//     same reason;
+//   * each stored nonzero is (value, byte offset into the staged tile); a warp
+//     walks the nonzeros of its filters two at a time, broadcasts them to all
+//     lanes and issues T multiply-adds per lane and nonzero, the accumulators
+//     living in registers for the whole layer;
 //   * results go through shared memory so that stores to NHWC are contiguous
-//     over the block's G output channels, with the epilogue applied on the way.
+//     over the block's G output channels, with the epilogue applied on the way;
+//   * weights, tables and epilogue vectors are fetched before the grid-dependency
+//     wait, so that inside a network they overlap the previous layer's tail.
+#include <algorithm>
+#include <cooperative_groups.h>
 #include "cadnn_internal.h"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
 struct SconvParams {
     const void *x;
     void *y;
-    const void *vals;
-    const uint16_t *offs;
-    const int32_t *ptr;
+    const uint32_t *ent;
     const int32_t *perm;
     const float *scale;
     const float *bias;
     const void *residual;
     int n, h, w, c_in, h_out, w_out, c_out;
-    int kh, kw, stride, pad;
-    int TH, TW, pitch, IH_t, IW_t, CIc, PP, n_chunks, G, c_pad, n_groups;
+    int stride, pad;
+    int BW, RB, TBX, TBY, TH, TW, pitch, half, IH_t, IW_t;
+    int CIc, PPb, n_chunks, G, n_groups, stages;
+    int ksplit;   // thread blocks per cluster; each takes a contiguous range of the channel chunks
     int tiles_y, tiles_x;
     long long P;  // total output pixels (linear mode)
-    int tile_words, max_entries;
+    int tile_bytes, stage_bytes;
+    int tab_off;                  // byte offset of the pixel table / epilogue vectors in shared memory
+    int hdr_bytes, block_bytes;   // per (chunk, filter block) record: row-start header + entries, fixed size
     int act, out_dtype, linear;
 };
 
-template <typename XT> struct AccOf { typedef float type; };
-template <> struct AccOf<int8_t> { typedef int type; };
+// dst: 32-bit shared-window address
+__device__ __forceinline__ void cp_async4(unsigned dst, const void *src, bool pred)
+{
+    int sz = pred ? 4 : 0;   // 0 source bytes: the destination is zero-filled
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;\n" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_async16(unsigned dst, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
 __device__ __forceinline__ float act_f32(float z, int act)
 {
     if (act == CADNN_ACT_RELU) return z > 0.0f ? z : 0.0f;
     if (act == CADNN_ACT_RELU6) return fminf(z > 0.0f ? z : 0.0f, 6.0f);
     return z;
-}
-
-// float layer: BatchNorm fold, residual, activation
-__device__ __forceinline__ float finish_f32(float acc, float sc, float bi, bool has_res, float res, int act)
-{
-    float z = fmaf(acc, sc, bi);
-    if (has_res) z += res;
-    return act_f32(z, act);
 }
 
 // int8 layer: one fused multiply-add on the converted accumulator, ReLU
@@ -69,18 +83,129 @@ __device__ __forceinline__ int requant_s8(int acc, float m, float b, int act)
     return __float2int_rn(t);
 }
 
-template <typename XT, int T, int RPW>
-__global__ void __launch_bounds__(256) sconv_kernel(const SconvParams p)
+template <typename XT> struct Traits;
+template <> struct Traits<float> {
+    typedef float acc_t;
+    static const int kEntryBytes = 8;
+    static const int kUnitElems = 1;   // elements per 4-byte staging unit
+};
+template <> struct Traits<int8_t> {
+    typedef int acc_t;
+    static const int kEntryBytes = 4;
+    static const int kUnitElems = 4;
+};
+
+// Per-block staging table, built once: for every staged input pixel its source pixel index
+// in x (-1 = zero padding / outside) and its byte offset inside a stage.
+__device__ __forceinline__ void build_pixel_table(const SconvParams &p, int2 *pix, int npx, int img, int oy0, int ox0,
+                                                  long long p0)
 {
-    typedef typename AccOf<XT>::type AT;
+    const int tid = threadIdx.x, NT = blockDim.x;
+    if (p.linear) {
+        for (int q = tid; q < npx; q += NT) {
+            long long op = p0 + q;
+            long long ip = -1;
+            if (op < p.P) {
+                ip = op;
+                if (p.stride != 1) {
+                    int ox = (int)(op % p.w_out);
+                    long long r = op / p.w_out;
+                    int oy = (int)(r % p.h_out);
+                    long long b = r / p.h_out;
+                    ip = (b * p.h + (long long)oy * p.stride) * p.w + (long long)ox * p.stride;
+                }
+            }
+            pix[q] = make_int2((int)ip, q * p.PPb);
+        }
+    } else {
+        const int iy0 = oy0 * p.stride - p.pad, ix0 = ox0 * p.stride - p.pad;
+        for (int i = tid; i < npx; i += NT) {
+            int r = i / p.IW_t, col = i - r * p.IW_t;
+            int iy = iy0 + r, ix = ix0 + col;
+            int src = -1;
+            if (iy >= 0 && iy < p.h && ix >= 0 && ix < p.w) src = (img * p.h + iy) * p.w + ix;
+            const int pos = p.half ? ((col & 1) * p.half + (col >> 1)) : col;
+            pix[i] = make_int2(src, (r * p.pitch + pos) * p.PPb);
+        }
+    }
+}
+
+// Asynchronous copy of this block's nonzeros of chunk c (header + entries, one fixed-size
+// record) behind the activation tile of a stage.  The weights never change, so this may be
+// issued before the producer of x has finished.
+__device__ __forceinline__ void stage_weights(const SconvParams &p, unsigned st32, int c, int grp)
+{
+    const uint4 *src = reinterpret_cast<const uint4 *>(
+        reinterpret_cast<const unsigned char *>(p.ent) + ((size_t)c * p.n_groups + grp) * p.block_bytes);
+    const unsigned dst = st32 + p.tile_bytes;
+    for (int e = threadIdx.x; e < (p.block_bytes >> 4); e += blockDim.x) cp_async16(dst + e * 16, src + e);
+}
+
+// Asynchronous copies that stage the activation tile of chunk c: pixel-major, PPb bytes per
+// pixel, 4 bytes per copy.
+template <typename XT>
+__device__ __forceinline__ void stage_acts(const SconvParams &p, const int2 *pixtab, int npx, unsigned char *smem,
+                                           unsigned smem32, unsigned stage_off, int c)
+{
+    typedef Traits<XT> TR;
+    const int tid = threadIdx.x, NT = blockDim.x;
+    const int c0 = c * p.CIc;
+    const XT *xg = reinterpret_cast<const XT *>(p.x);
+    const unsigned st32 = smem32 + stage_off;
+    const bool unit_ok = (TR::kUnitElems == 1) || ((p.c_in & 3) == 0);
+    if (unit_ok) {
+        const int upp = p.CIc / TR::kUnitElems;   // 4-byte units per staged pixel
+        const int total = npx * upp;
+        if ((upp & (upp - 1)) == 0) {
+            const int sh = 31 - __clz(upp);
+#pragma unroll 4
+            for (int idx = tid; idx < total; idx += NT) {
+                const int pix = idx >> sh, u = idx & (upp - 1);
+                const int2 te = pixtab[pix];
+                const int ci = c0 + u * TR::kUnitElems;
+                const bool ok = te.x >= 0 && ci < p.c_in;
+                const XT *src = ok ? xg + (size_t)te.x * p.c_in + ci : xg;
+                cp_async4(st32 + te.y + u * 4, src, ok);
+            }
+        } else {
+            for (int idx = tid; idx < total; idx += NT) {
+                const int pix = idx / upp, u = idx - pix * upp;
+                const int2 te = pixtab[pix];
+                const int ci = c0 + u * TR::kUnitElems;
+                const bool ok = te.x >= 0 && ci < p.c_in;
+                const XT *src = ok ? xg + (size_t)te.x * p.c_in + ci : xg;
+                cp_async4(st32 + te.y + u * 4, src, ok);
+            }
+        }
+    } else {
+        // int8 with a channel count that is not a multiple of 4: plain byte copies
+        const int cw = p.CIc;
+        XT *stage = reinterpret_cast<XT *>(smem + stage_off);
+        for (int idx = tid; idx < npx * cw; idx += NT) {
+            const int pix = idx / cw, cl = idx - pix * cw;
+            const int2 te = pixtab[pix];
+            const int ci = c0 + cl;
+            XT v = 0;
+            if (te.x >= 0 && ci < p.c_in) v = xg[(size_t)te.x * p.c_in + ci];
+            stage[te.y + cl] = v;
+        }
+    }
+}
+
+template <typename XT, int T, int RPW>
+__global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
+{
+    typedef Traits<XT> TR;
+    typedef typename TR::acc_t AT;
     extern __shared__ __align__(16) unsigned char smem[];
-    AT *sX = reinterpret_cast<AT *>(smem);
-    uint2 *sW = reinterpret_cast<uint2 *>(smem + (size_t)p.tile_words * 4);
-    int *sPtr = reinterpret_cast<int *>(sW + p.max_entries);
+    const unsigned smem32 = (unsigned)__cvta_generic_to_shared(smem);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int grp = blockIdx.x % p.n_groups;
-    int tile = blockIdx.x / p.n_groups;
+    const int KS = p.ksplit;
+    const int rank = blockIdx.x % KS;
+    const int rest = blockIdx.x / KS;
+    const int grp = rest % p.n_groups;
+    int tile = rest / p.n_groups;
     const int G = p.G;
 
     // tile origin
@@ -97,17 +222,25 @@ __global__ void __launch_bounds__(256) sconv_kernel(const SconvParams p)
         ox0 = tx * p.TW;
     }
 
-    // byte offset, inside the staged tile, of the top-left tap of each of this lane's pixels
-    int pixoff[T];
+    // this block's range of channel chunks
+    const int per = (p.n_chunks + KS - 1) / KS;
+    const int c_lo = min(p.n_chunks, rank * per), c_hi = min(p.n_chunks, c_lo + per);
+
+    // Byte offset of a lane's pixel inside the staged tile = lane part + band part; the band
+    // part is the same for every lane, so the T loads of one nonzero share one address add.
+    const int xs = p.half ? 1 : p.stride;
+    unsigned lanebase, band[T];
+    if (p.linear) {
+        lanebase = lane * p.PPb;
 #pragma unroll
-    for (int t = 0; t < T; ++t) {
-        int q = lane + 32 * t;
-        if (p.linear) {
-            pixoff[t] = q * p.PP * 4;
-        } else {
-            int ly = q / p.TW, lx = q - ly * p.TW;
-            bool ok = (ly < p.TH) && (oy0 + ly < p.h_out) && (ox0 + lx < p.w_out);
-            pixoff[t] = ok ? ((ly * p.stride) * p.pitch + lx * p.stride) * p.PP * 4 : 0;
+        for (int t = 0; t < T; ++t) band[t] = t * 32 * p.PPb;
+    } else {
+        const int lr = lane / p.BW, lc = lane - lr * p.BW;
+        lanebase = (lr < p.RB) ? ((lr * p.stride) * p.pitch + lc * xs) * p.PPb : 0;
+#pragma unroll
+        for (int t = 0; t < T; ++t) {
+            const int ty = t / p.TBX, tx = t - ty * p.TBX;
+            band[t] = ((ty * p.RB * p.stride) * p.pitch + tx * p.BW * xs) * p.PPb;
         }
     }
 
@@ -117,139 +250,89 @@ __global__ void __launch_bounds__(256) sconv_kernel(const SconvParams p)
 #pragma unroll
         for (int t = 0; t < T; ++t) acc[j][t] = 0;
 
-    const XT *xg = reinterpret_cast<const XT *>(p.x);
-    const bool vec4 = (p.c_in % 4 == 0) && (p.CIc % 4 == 0);
+    // ---- staging table and epilogue vectors (behind the pipeline stages in shared memory) ----
+    const int S = p.stages;
+    const int npx_in = p.linear ? 32 * T : p.IH_t * p.IW_t;
+    int2 *pixtab = reinterpret_cast<int2 *>(smem + p.tab_off);
+    float *sScale = reinterpret_cast<float *>(pixtab + npx_in);
+    float *sBias = sScale + G;
+    build_pixel_table(p, pixtab, npx_in, img, oy0, ox0, p0);
+    for (int i = tid; i < G; i += blockDim.x) {
+        const int co = grp * G + i;
+        sScale[i] = (p.scale && co < p.c_out) ? p.scale[co] : 1.0f;
+        sBias[i] = (p.bias && co < p.c_out) ? p.bias[co] : 0.0f;
+    }
+    int co_of[RPW];
+#pragma unroll
+    for (int j = 0; j < RPW; ++j) co_of[j] = p.perm[grp * G + warp * RPW + j];
 
-    for (int c = 0; c < p.n_chunks; ++c) {
-        __syncthreads();  // the previous chunk's tile and weights are no longer read
-        const int c0 = c * p.CIc;
+    // ---- pipeline prologue: weights first (they do not depend on the previous layer) ----
+    const int npre = (S == 1) ? 1 : S - 1;
+    for (int s = 0; s < npre; ++s)
+        if (c_lo + s < c_hi) stage_weights(p, smem32 + (unsigned)(s * p.stage_bytes), c_lo + s, grp);
+    __syncthreads();          // the pixel table is complete
+    grid_dep_wait();          // x (and the residual) are final from here on
+    grid_dep_trigger();
+    for (int s = 0; s < npre; ++s) {
+        if (c_lo + s < c_hi) stage_acts<XT>(p, pixtab, npx_in, smem, smem32, (unsigned)(s * p.stage_bytes), c_lo + s);
+        cp_async_commit();
+    }
 
-        // ---- stage this block's nonzeros of the chunk: (value, byte offset) ----
-        {
-            const int32_t *pp = p.ptr + (size_t)c * (p.c_pad + 1) + grp * G;
-            const int gbeg = pp[0];
-            const int cnt = pp[G] - gbeg;
-            if (tid <= G) sPtr[tid] = pp[tid] - gbeg;
-            for (int e = tid; e < cnt; e += blockDim.x) {
-                uint2 ent;
-                if (sizeof(XT) == 1) ent.x = (unsigned)(int)reinterpret_cast<const int8_t *>(p.vals)[gbeg + e];
-                else ent.x = reinterpret_cast<const unsigned *>(p.vals)[gbeg + e];
-                ent.y = (unsigned)p.offs[gbeg + e] * 4u;
-                sW[e] = ent;
+    int buf = 0;   // stage holding chunk c
+    for (int c = c_lo; c < c_hi; ++c) {
+        if (S == 1) {
+            if (c > c_lo) {
+                __syncthreads();   // everyone is done with chunk c - 1
+                stage_weights(p, smem32, c, grp);
+                stage_acts<XT>(p, pixtab, npx_in, smem, smem32, 0u, c);
+                cp_async_commit();
             }
-        }
-
-        // ---- stage the activation tile: pixel-major, PP words per pixel ----
-        if (p.linear) {
-            const int npx = 32 * T;
-            if (vec4) {
-                const int cv = p.CIc >> 2;
-                for (int idx = tid; idx < npx * cv; idx += blockDim.x) {
-                    int q = idx / cv, v = idx - q * cv;
-                    long long op = p0 + q;
-                    int ci = c0 + v * 4;
-                    AT a0 = 0, a1 = 0, a2 = 0, a3 = 0;
-                    if (op < p.P && ci < p.c_in) {
-                        long long ip = op;
-                        if (p.stride != 1) {
-                            int ox = (int)(op % p.w_out);
-                            long long r = op / p.w_out;
-                            int oy = (int)(r % p.h_out);
-                            long long b = r / p.h_out;
-                            ip = (b * p.h + (long long)oy * p.stride) * p.w + (long long)ox * p.stride;
-                        }
-                        const XT *src = xg + ip * p.c_in + ci;
-                        if (sizeof(XT) == 4) {
-                            float4 f = *reinterpret_cast<const float4 *>(src);
-                            a0 = f.x; a1 = f.y; a2 = f.z; a3 = f.w;
-                        } else {
-                            char4 q4 = *reinterpret_cast<const char4 *>(src);
-                            a0 = q4.x; a1 = q4.y; a2 = q4.z; a3 = q4.w;
-                        }
-                    }
-                    AT *dst = sX + q * p.PP + v * 4;
-                    dst[0] = a0; dst[1] = a1; dst[2] = a2; dst[3] = a3;
-                }
-            } else {
-                for (int idx = tid; idx < npx * p.CIc; idx += blockDim.x) {
-                    int q = idx / p.CIc, cl = idx - q * p.CIc;
-                    long long op = p0 + q;
-                    int ci = c0 + cl;
-                    AT a = 0;
-                    if (op < p.P && ci < p.c_in) {
-                        long long ip = op;
-                        if (p.stride != 1) {
-                            int ox = (int)(op % p.w_out);
-                            long long r = op / p.w_out;
-                            int oy = (int)(r % p.h_out);
-                            long long b = r / p.h_out;
-                            ip = (b * p.h + (long long)oy * p.stride) * p.w + (long long)ox * p.stride;
-                        }
-                        a = (AT)xg[ip * p.c_in + ci];
-                    }
-                    sX[q * p.PP + cl] = a;
-                }
-            }
+            cp_async_wait<0>();
+            __syncthreads();
         } else {
-            const int iy0 = oy0 * p.stride - p.pad, ix0 = ox0 * p.stride - p.pad;
-            const XT *ximg = xg + (size_t)img * p.h * p.w * p.c_in;
-            if (vec4) {
-                const int cv = p.CIc >> 2;
-                const int total = p.IH_t * p.IW_t * cv;
-                for (int idx = tid; idx < total; idx += blockDim.x) {
-                    int pix = idx / cv, v = idx - pix * cv;
-                    int r = pix / p.IW_t, col = pix - r * p.IW_t;
-                    int iy = iy0 + r, ix = ix0 + col, ci = c0 + v * 4;
-                    AT a0 = 0, a1 = 0, a2 = 0, a3 = 0;
-                    if (iy >= 0 && iy < p.h && ix >= 0 && ix < p.w && ci < p.c_in) {
-                        const XT *src = ximg + ((size_t)iy * p.w + ix) * p.c_in + ci;
-                        if (sizeof(XT) == 4) {
-                            float4 f = *reinterpret_cast<const float4 *>(src);
-                            a0 = f.x; a1 = f.y; a2 = f.z; a3 = f.w;
-                        } else {
-                            char4 q4 = *reinterpret_cast<const char4 *>(src);
-                            a0 = q4.x; a1 = q4.y; a2 = q4.z; a3 = q4.w;
-                        }
-                    }
-                    AT *dst = sX + (r * p.pitch + col) * p.PP + v * 4;
-                    dst[0] = a0; dst[1] = a1; dst[2] = a2; dst[3] = a3;
-                }
-            } else {
-                const int total = p.IH_t * p.IW_t * p.CIc;
-                for (int idx = tid; idx < total; idx += blockDim.x) {
-                    int pix = idx / p.CIc, cl = idx - pix * p.CIc;
-                    int r = pix / p.IW_t, col = pix - r * p.IW_t;
-                    int iy = iy0 + r, ix = ix0 + col, ci = c0 + cl;
-                    AT a = 0;
-                    if (iy >= 0 && iy < p.h && ix >= 0 && ix < p.w && ci < p.c_in)
-                        a = (AT)ximg[((size_t)iy * p.w + ix) * p.c_in + ci];
-                    sX[(r * p.pitch + col) * p.PP + cl] = a;
-                }
+            if (S == 3) cp_async_wait<1>(); else cp_async_wait<0>();
+            __syncthreads();   // chunk c has landed for everyone; everyone is done with chunk c - 1
+            const int nxt = c + S - 1;
+            int nbuf = buf + S - 1;
+            if (nbuf >= S) nbuf -= S;
+            if (nxt < c_hi) {
+                stage_weights(p, smem32 + (unsigned)(nbuf * p.stage_bytes), nxt, grp);
+                stage_acts<XT>(p, pixtab, npx_in, smem, smem32, (unsigned)(nbuf * p.stage_bytes), nxt);
             }
+            cp_async_commit();
         }
-        __syncthreads();
-
-        // ---- walk the nonzeros of this warp's filters ----
-        const unsigned char *sXb = reinterpret_cast<const unsigned char *>(sX);
+        const unsigned stage_off = (unsigned)(buf * p.stage_bytes);
+        const int *sP = reinterpret_cast<const int *>(smem + stage_off + p.tile_bytes);
+        const unsigned sW = stage_off + p.tile_bytes + p.hdr_bytes;
+        const unsigned lanep = stage_off + lanebase;
 #pragma unroll
         for (int j = 0; j < RPW; ++j) {
             const int row = warp * RPW + j;
-            const int beg = sPtr[row], end = sPtr[row + 1];
-#pragma unroll 4
-            for (int e = beg; e < end; ++e) {
-                const uint2 ent = sW[e];
-                AT wv;
-                if (sizeof(XT) == 4) wv = (AT)__uint_as_float(ent.x);
-                else wv = (AT)(int)ent.x;
-                const unsigned char *base = sXb + ent.y;
-#pragma unroll
-                for (int t = 0; t < T; ++t) {
-                    AT xv = *reinterpret_cast<const AT *>(base + pixoff[t]);
-                    acc[j][t] += wv * xv;
+            const int beg = sP[row], end = sP[row + 1];
+#pragma unroll 2
+            for (int e = beg; e < end; e += 2) {
+                AT w0, w1;
+                unsigned o0, o1;
+                if (TR::kEntryBytes == 8) {
+                    const uint4 v = *reinterpret_cast<const uint4 *>(smem + sW + e * 8);
+                    w0 = (AT)__uint_as_float(v.x); o0 = v.y;
+                    w1 = (AT)__uint_as_float(v.z); o1 = v.w;
+                } else {
+                    const uint2 v = *reinterpret_cast<const uint2 *>(smem + sW + e * 4);
+                    w0 = (AT)(int)(int8_t)(v.x & 0xffu); o0 = v.x >> 8;
+                    w1 = (AT)(int)(int8_t)(v.y & 0xffu); o1 = v.y >> 8;
                 }
+                const unsigned a0 = lanep + o0;
+                const unsigned a1 = lanep + o1;
+#pragma unroll
+                for (int t = 0; t < T; ++t) acc[j][t] += w0 * (AT)(*reinterpret_cast<const XT *>(smem + a0 + band[t]));
+#pragma unroll
+                for (int t = 0; t < T; ++t) acc[j][t] += w1 * (AT)(*reinterpret_cast<const XT *>(smem + a1 + band[t]));
             }
         }
+        if (++buf == S) buf = 0;
     }
+    cp_async_wait<0>();
 
     // ---- results to shared memory, [pixel][G + 1], at the original channel position ----
     __syncthreads();
@@ -257,11 +340,31 @@ __global__ void __launch_bounds__(256) sconv_kernel(const SconvParams p)
     const int op = G + 1;
 #pragma unroll
     for (int j = 0; j < RPW; ++j) {
-        int co = p.perm[grp * G + warp * RPW + j];
+        const int co = co_of[j];
         if (co >= 0) {
             int lc = co - grp * G;
 #pragma unroll
             for (int t = 0; t < T; ++t) sOut[(lane + 32 * t) * op + lc] = acc[j][t];
+        }
+    }
+
+    // ---- channel-split blocks of a cluster: sum the partial results over distributed shared memory ----
+    const int npx = 32 * T;
+    int q_lo = 0, q_hi = npx;
+    if (KS > 1) {
+        cg::cluster_group cluster = cg::this_cluster();
+        cluster.sync();   // every block's partial sums are in its shared memory
+        const int span = (npx + KS - 1) / KS;
+        q_lo = min(npx, rank * span);
+        q_hi = min(npx, q_lo + span);
+        for (int idx = tid + q_lo * op; idx < q_hi * op; idx += blockDim.x) {
+            AT v = sOut[idx];
+            for (int k = 1; k < KS; ++k) {
+                int other = rank + k;
+                if (other >= KS) other -= KS;
+                v += *cluster.map_shared_rank(sOut + idx, other);
+            }
+            sOut[idx] = v;
         }
     }
     __syncthreads();
@@ -269,38 +372,82 @@ __global__ void __launch_bounds__(256) sconv_kernel(const SconvParams p)
     // ---- epilogue and contiguous NHWC stores ----
     const int co_base = grp * G;
     const int gw = min(G, p.c_out - co_base);  // real channels in this block
-    const int npx = 32 * T;
     const bool has_res = p.residual != nullptr;
-    for (int idx = tid; idx < npx * gw; idx += blockDim.x) {
-        int q = idx / gw, lc = idx - q * gw;
+    const bool quad = ((gw & 3) == 0) && ((p.c_out & 3) == 0);
+    const int cols = quad ? (gw >> 2) : gw;
+    for (int idx = tid + q_lo * cols; idx < q_hi * cols; idx += blockDim.x) {
+        const int q = idx / cols, cq = idx - q * cols;
         long long opix;
         if (p.linear) {
             opix = p0 + q;
             if (opix >= p.P) continue;
         } else {
-            int ly = q / p.TW, lx = q - ly * p.TW;
-            int oy = oy0 + ly, ox = ox0 + lx;
-            if (ly >= p.TH || oy >= p.h_out || ox >= p.w_out) continue;
+            const int t = q >> 5, l = q & 31;
+            const int ty = t / p.TBX, tx = t - ty * p.TBX;
+            const int lr = l / p.BW, lcx = l - lr * p.BW;
+            const int oy = oy0 + ty * p.RB + lr, ox = ox0 + tx * p.BW + lcx;
+            if (lr >= p.RB || oy >= p.h_out || ox >= p.w_out) continue;
             opix = ((long long)img * p.h_out + oy) * p.w_out + ox;
         }
+        const int lc = quad ? cq * 4 : cq;
         const int co = co_base + lc;
         const size_t oi = (size_t)opix * p.c_out + co;
-        const AT a = sOut[q * op + lc];
-        const float sc = p.scale ? p.scale[co] : 1.0f;
-        const float bi = p.bias ? p.bias[co] : 0.0f;
-        if (sizeof(XT) == 4) {
-            float r = has_res ? reinterpret_cast<const float *>(p.residual)[oi] : 0.0f;
-            reinterpret_cast<float *>(p.y)[oi] = finish_f32((float)a, sc, bi, has_res, r, p.act);
+        const AT *a = sOut + q * op + lc;
+        if (quad) {
+            float sc[4], bi[4];
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                sc[v] = sScale[lc + v];
+                bi[v] = sBias[lc + v];
+            }
+            if (sizeof(XT) == 4) {
+                float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (has_res) r = *reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(p.residual) + oi);
+                float4 o;
+                o.x = act_f32(fmaf((float)a[0], sc[0], bi[0]) + r.x, p.act);
+                o.y = act_f32(fmaf((float)a[1], sc[1], bi[1]) + r.y, p.act);
+                o.z = act_f32(fmaf((float)a[2], sc[2], bi[2]) + r.z, p.act);
+                o.w = act_f32(fmaf((float)a[3], sc[3], bi[3]) + r.w, p.act);
+                *reinterpret_cast<float4 *>(reinterpret_cast<float *>(p.y) + oi) = o;
+            } else if (p.out_dtype == CADNN_S32) {
+                *reinterpret_cast<int4 *>(reinterpret_cast<int *>(p.y) + oi) = make_int4((int)a[0], (int)a[1], (int)a[2], (int)a[3]);
+            } else if (p.out_dtype == CADNN_F32) {
+                float4 o;
+                o.x = requant_f32((int)a[0], sc[0], bi[0], p.act);
+                o.y = requant_f32((int)a[1], sc[1], bi[1], p.act);
+                o.z = requant_f32((int)a[2], sc[2], bi[2], p.act);
+                o.w = requant_f32((int)a[3], sc[3], bi[3], p.act);
+                *reinterpret_cast<float4 *>(reinterpret_cast<float *>(p.y) + oi) = o;
+            } else {
+                char4 o;
+                o.x = (signed char)requant_s8((int)a[0], sc[0], bi[0], p.act);
+                o.y = (signed char)requant_s8((int)a[1], sc[1], bi[1], p.act);
+                o.z = (signed char)requant_s8((int)a[2], sc[2], bi[2], p.act);
+                o.w = (signed char)requant_s8((int)a[3], sc[3], bi[3], p.act);
+                *reinterpret_cast<char4 *>(reinterpret_cast<int8_t *>(p.y) + oi) = o;
+            }
         } else {
-            if (p.out_dtype == CADNN_S32) reinterpret_cast<int *>(p.y)[oi] = (int)a;
-            else if (p.out_dtype == CADNN_F32) reinterpret_cast<float *>(p.y)[oi] = requant_f32((int)a, sc, bi, p.act);
-            else reinterpret_cast<int8_t *>(p.y)[oi] = (int8_t)requant_s8((int)a, sc, bi, p.act);
+            const float sc = sScale[lc];
+            const float bi = sBias[lc];
+            if (sizeof(XT) == 4) {
+                float z = fmaf((float)a[0], sc, bi);
+                if (has_res) z += reinterpret_cast<const float *>(p.residual)[oi];
+                reinterpret_cast<float *>(p.y)[oi] = act_f32(z, p.act);
+            } else if (p.out_dtype == CADNN_S32) {
+                reinterpret_cast<int *>(p.y)[oi] = (int)a[0];
+            } else if (p.out_dtype == CADNN_F32) {
+                reinterpret_cast<float *>(p.y)[oi] = requant_f32((int)a[0], sc, bi, p.act);
+            } else {
+                reinterpret_cast<int8_t *>(p.y)[oi] = (int8_t)requant_s8((int)a[0], sc, bi, p.act);
+            }
         }
     }
+    // peers may still be reading this block's partial sums
+    if (KS > 1) cg::this_cluster().sync();
 }
 
 template <typename XT, int T, int RPW>
-cadnn_status launch_one(const SconvParams &p, int blocks, int smem, cudaStream_t st)
+cadnn_status launch_one(const SconvParams &p, int blocks, int threads, int smem, bool pdl, cudaStream_t st)
 {
     auto kern = sconv_kernel<XT, T, RPW>;
     static int smem_allowed = 48 * 1024;  // raised once per instantiation, as layers need it
@@ -308,31 +455,54 @@ cadnn_status launch_one(const SconvParams &p, int blocks, int smem, cudaStream_t
         CADNN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         smem_allowed = smem;
     }
-    kern<<<blocks, 256, smem, st>>>(p);
-    CADNN_CUDA_TRY(cudaGetLastError());
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks, 1, 1);
+    cfg.blockDim = dim3((unsigned)threads, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (p.ksplit > 1) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = (unsigned)p.ksplit;
+        attr[na].val.clusterDim.y = 1;
+        attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    if (pdl) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = (unsigned)na;
+    CADNN_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, p));
     return CADNN_OK;
 }
 
 template <typename XT, int T>
-cadnn_status launch_rpw(const SconvParams &p, int rpw, int blocks, int smem, cudaStream_t st)
+cadnn_status launch_rpw(const SconvParams &p, int rpw, int blocks, int threads, int smem, bool pdl, cudaStream_t st)
 {
     switch (rpw) {
-        case 1: return launch_one<XT, T, 1>(p, blocks, smem, st);
-        case 2: return launch_one<XT, T, 2>(p, blocks, smem, st);
-        case 4: return launch_one<XT, T, 4>(p, blocks, smem, st);
+        case 1: return launch_one<XT, T, 1>(p, blocks, threads, smem, pdl, st);
+        case 2: return launch_one<XT, T, 2>(p, blocks, threads, smem, pdl, st);
+        case 4: return launch_one<XT, T, 4>(p, blocks, threads, smem, pdl, st);
     }
     return CADNN_E_UNSUPPORTED;
 }
 
 template <typename XT>
-cadnn_status launch_T(const SconvParams &p, int T, int rpw, int blocks, int smem, cudaStream_t st)
+cadnn_status launch_T(const SconvParams &p, int T, int rpw, int blocks, int threads, int smem, bool pdl, cudaStream_t st)
 {
     switch (T) {
-        case 1: return launch_rpw<XT, 1>(p, rpw, blocks, smem, st);
-        case 2: return launch_rpw<XT, 2>(p, rpw, blocks, smem, st);
-        case 4: return launch_rpw<XT, 4>(p, rpw, blocks, smem, st);
-        case 7: return launch_rpw<XT, 7>(p, rpw, blocks, smem, st);
-        case 8: return launch_rpw<XT, 8>(p, rpw, blocks, smem, st);
+        case 1: return launch_rpw<XT, 1>(p, rpw, blocks, threads, smem, pdl, st);
+        case 2: return launch_rpw<XT, 2>(p, rpw, blocks, threads, smem, pdl, st);
+        case 3: return launch_rpw<XT, 3>(p, rpw, blocks, threads, smem, pdl, st);
+        case 4: return launch_rpw<XT, 4>(p, rpw, blocks, threads, smem, pdl, st);
+        case 5: return launch_rpw<XT, 5>(p, rpw, blocks, threads, smem, pdl, st);
+        case 6: return launch_rpw<XT, 6>(p, rpw, blocks, threads, smem, pdl, st);
+        case 7: return launch_rpw<XT, 7>(p, rpw, blocks, threads, smem, pdl, st);
+        case 8: return launch_rpw<XT, 8>(p, rpw, blocks, threads, smem, pdl, st);
     }
     return CADNN_E_UNSUPPORTED;
 }
@@ -344,25 +514,30 @@ cadnn_status launch_sconv(const cadnn_weights *w, const void *x, int n, void *y,
 {
     const cadnn_layer_desc &d = w->desc;
     const Schedule &s = w->s;
+    const bool s8 = d.dtype == CADNN_S8;
     SconvParams p;
     p.x = x;
     p.y = y;
-    p.vals = w->d_vals;
-    p.offs = w->d_offs;
-    p.ptr = w->d_ptr;
+    p.ent = w->d_ent;
     p.perm = w->d_perm;
     p.scale = ep.scale;
     p.bias = ep.bias;
     p.residual = ep.residual;
     p.n = n; p.h = d.in_h; p.w = d.in_w; p.c_in = d.c_in;
     p.h_out = w->h_out; p.w_out = w->w_out; p.c_out = d.c_out;
-    p.kh = d.kh; p.kw = d.kw; p.stride = d.stride; p.pad = d.pad;
-    p.TH = s.TH; p.TW = s.TW; p.pitch = s.pitch; p.IH_t = s.IH_t; p.IW_t = s.IW_t;
-    p.CIc = s.CIc; p.PP = s.PP; p.n_chunks = s.n_chunks; p.G = s.G; p.c_pad = w->c_pad; p.n_groups = s.n_groups;
+    p.stride = d.stride; p.pad = d.pad;
+    p.BW = s.BW; p.RB = s.RB; p.TBX = s.TBX; p.TBY = s.TBY; p.TH = s.TH; p.TW = s.TW;
+    p.pitch = s.pitch; p.half = s.half; p.IH_t = s.IH_t; p.IW_t = s.IW_t;
+    p.CIc = s.CIc; p.PPb = s.PPb; p.n_chunks = s.n_chunks; p.G = s.G; p.n_groups = s.n_groups;
+    p.stages = s.stages;
+    p.ksplit = s.ksplit;
     p.linear = s.kind == KK_SCONV_LINEAR;
     p.P = (long long)n * w->h_out * w->w_out;
-    p.tile_words = s.tile_words;
-    p.max_entries = s.max_entries;
+    p.tile_bytes = s.tile_bytes;
+    p.stage_bytes = s.stage_bytes;
+    p.tab_off = (std::max(s.stages * s.stage_bytes, 32 * s.T * (s.G + 1) * 4) + 15) / 16 * 16;
+    p.hdr_bytes = (s.G + 1 + 3) / 4 * 16;
+    p.block_bytes = p.hdr_bytes + s.max_entries * (s8 ? 4 : 8);
     p.act = ep.act;
     p.out_dtype = ep.out_dtype;
     long long tiles;
@@ -374,9 +549,9 @@ cadnn_status launch_sconv(const cadnn_weights *w, const void *x, int n, void *y,
         p.tiles_x = (w->w_out + s.TW - 1) / s.TW;
         tiles = (long long)n * p.tiles_y * p.tiles_x;
     }
-    long long blocks = tiles * s.n_groups;
+    long long blocks = tiles * s.n_groups * s.ksplit;
     if (blocks <= 0) return CADNN_OK;
     if (blocks > 2147483647LL) return CADNN_E_UNSUPPORTED;
-    if (d.dtype == CADNN_S8) return launch_T<int8_t>(p, s.T, s.RPW, (int)blocks, s.smem_bytes, st);
-    return launch_T<float>(p, s.T, s.RPW, (int)blocks, s.smem_bytes, st);
+    if (s8) return launch_T<int8_t>(p, s.T, s.RPW, (int)blocks, s.NW * 32, s.smem_bytes, ep.pdl, st);
+    return launch_T<float>(p, s.T, s.RPW, (int)blocks, s.NW * 32, s.smem_bytes, ep.pdl, st);
 }

@@ -66,5 +66,5 @@ class PackedModel:
     def forward_host(self, x_host, y_host, use_graph=True, stream=None):
         return B.cadnn_forward_host(self.net, x_host, y_host, use_graph, stream)
 
-    def layer_times(self, x, y, flush_l2=False):
-        return B.cadnn_net_layer_times(self.net, x, y, len(self.model.ops), flush_l2)
+    def layer_times(self, x, y, flush_l2=False, reps=1):
+        return B.cadnn_net_layer_times(self.net, x, y, len(self.model.ops), flush_l2, reps)
