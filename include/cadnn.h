@@ -59,6 +59,9 @@ typedef enum {
 } cadnn_fmt;
 
 #define CADNN_PACK_HOST_ONLY 1 /* build the packed image on the host only (no device needed, no compute) */
+#define CADNN_PACK_AUTOTUNE 2  /* conv layers: time the candidate schedules on the current device (batch_hint
+                                  images of zeros, scratch buffers allocated and freed inside the call) and
+                                  keep the fastest, instead of trusting the packer's time model */
 
 /*
  * One layer.  The packer is the offline stage of Section 4 ("Memory layout
@@ -76,7 +79,7 @@ typedef struct {
     int batch_hint;
     int dtype; /* cadnn_dtype of weights and activations: CADNN_F32 or CADNN_S8 */
     int fmt;   /* cadnn_fmt, CADNN_FMT_AUTO */
-    int flags; /* CADNN_PACK_HOST_ONLY or 0 */
+    int flags; /* CADNN_PACK_HOST_ONLY, CADNN_PACK_AUTOTUNE or 0 */
 } cadnn_layer_desc;
 
 typedef struct cadnn_weights cadnn_weights;

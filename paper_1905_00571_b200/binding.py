@@ -22,6 +22,7 @@ F32, S8, S32 = 0, 1, 2
 DTYPE = {"f32": F32, "s8": S8, "s32": S32}
 ACT = {"none": 0, "relu": 1, "relu6": 2, None: 0}
 PACK_HOST_ONLY = 1
+PACK_AUTOTUNE = 2
 OP_CONV, OP_FC, OP_MAXPOOL, OP_GAVGPOOL = 0, 1, 2, 3
 FMT_NAMES = {1: "tiled_csr", 2: "row_csr", 3: "dense_dw", 4: "dense_smallc"}
 KIND_NAMES = {1: "sconv_spatial", 2: "sconv_linear", 3: "fc_spmv", 4: "dw", 5: "dense_smallc"}
@@ -127,9 +128,9 @@ class Weights:
 
 
 def make_desc(c_in, c_out, kh=1, kw=1, stride=1, pad=0, groups=1, in_h=1, in_w=1, batch_hint=1,
-              dtype="f32", host_only=False):
-    return LayerDesc(c_in, c_out, kh, kw, stride, pad, groups, in_h, in_w, batch_hint,
-                     DTYPE[dtype], 0, PACK_HOST_ONLY if host_only else 0)
+              dtype="f32", host_only=False, autotune=False):
+    flags = (PACK_HOST_ONLY if host_only else 0) | (PACK_AUTOTUNE if autotune else 0)
+    return LayerDesc(c_in, c_out, kh, kw, stride, pad, groups, in_h, in_w, batch_hint, DTYPE[dtype], 0, flags)
 
 
 def cadnn_pack(desc, w_ohwi, mask=None, w_scale=None):

@@ -193,6 +193,9 @@ cadnn_status upload(cadnn_weights *h)
     if (b_dense) CADNN_CUDA_TRY(cudaMemcpy(base + o_dense, h->dense_f.data(), b_dense, cudaMemcpyHostToDevice));
     if (b_ent) CADNN_CUDA_TRY(cudaMemcpy(base + o_ent, h->ent.data(), b_ent, cudaMemcpyHostToDevice));
     h->d_ent = (const uint32_t *)(base + o_ent);
+    // A copy from pageable host memory may return before its DMA has landed; kernels on
+    // non-blocking streams are not ordered behind it, so wait for it here.
+    CADNN_CUDA_TRY(cudaStreamSynchronize(cudaStreamLegacy));
     h->d_vals = base + o_vals;
     h->d_offs = (const uint16_t *)(base + o_offs);
     h->d_ptr = (const int32_t *)(base + o_ptr);
@@ -400,6 +403,109 @@ cadnn_status build_sconv_image(cadnn_weights *h, const Src &src, const Geometry 
     return CADNN_OK;
 }
 
+// Time one packed conv layer on the current device: a CUDA graph of `reps` back-to-back
+// launches on zero-filled activations, replayed once untimed and once between events.
+// Returns microseconds per launch, or a negative value if the schedule cannot run.
+float time_schedule(cadnn_weights *h, int batch, const void *x, void *y, cudaStream_t st, int reps)
+{
+    LaunchEpilogue ep;
+    ep.out_dtype = h->desc.dtype;
+    ep.act = CADNN_ACT_RELU;
+    if (launch_sconv(h, x, batch, y, ep, st) != CADNN_OK) return -1.0f;   // also raises the kernel's smem limit
+    if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return -1.0f; }
+    cudaGraph_t g = nullptr;
+    cudaGraphExec_t ge = nullptr;
+    float us = -1.0f;
+    if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { cudaGetLastError(); return -1.0f; }
+    bool ok = true;
+    for (int r = 0; r < reps && ok; ++r) ok = launch_sconv(h, x, batch, y, ep, st) == CADNN_OK;
+    if (cudaStreamEndCapture(st, &g) != cudaSuccess) ok = false;
+    if (ok && cudaGraphInstantiate(&ge, g, 0) == cudaSuccess) {
+        cudaEvent_t e0, e1;
+        cudaEventCreate(&e0);
+        cudaEventCreate(&e1);
+        cudaGraphLaunch(ge, st);
+        float best = 1e30f;
+        for (int rep = 0; rep < 2; ++rep) {
+            cudaEventRecord(e0, st);
+            cudaGraphLaunch(ge, st);
+            cudaEventRecord(e1, st);
+            if (cudaStreamSynchronize(st) == cudaSuccess) {
+                float ms = 0.0f;
+                cudaEventElapsedTime(&ms, e0, e1);
+                best = std::min(best, ms);
+            }
+        }
+        if (best < 1e29f) us = best * 1e3f / (float)reps;
+        cudaEventDestroy(e0);
+        cudaEventDestroy(e1);
+    }
+    if (ge) cudaGraphExecDestroy(ge);
+    if (g) cudaGraphDestroy(g);
+    cudaGetLastError();
+    return us;
+}
+
+// Measured parameter selection (Section 4, "Optimization parameters selection": the search
+// space is pruned with knowledge of the layer and the machine - here the time model keeps
+// the best candidate of every structural class - and the survivors are timed).
+cadnn_status autotune_sconv(cadnn_weights *h, const Src &src, const Geometry &g, const std::vector<int64_t> &row_nnz,
+                            const std::vector<Candidate> &cands)
+{
+    const cadnn_layer_desc &d = h->desc;
+    const int batch = std::max(1, d.batch_hint);
+    // best candidate by the model of every (warps, filters per warp, cluster split, bands) class
+    std::vector<Candidate> pick;
+    std::vector<long> seen;
+    for (const Candidate &c : cands) {
+        long key = ((c.s.NW * 8L + c.s.RPW) * 16 + c.s.ksplit) * 16 + c.s.T;
+        if (std::find(seen.begin(), seen.end(), key) != seen.end()) continue;
+        seen.push_back(key);
+        pick.push_back(c);
+    }
+    const size_t kMaxTimed = 56;
+    if (pick.size() > kMaxTimed) pick.resize(kMaxTimed);
+    const size_t esz = src.s8 ? 1 : 4;
+    const size_t xb = (size_t)batch * d.in_h * d.in_w * d.c_in * esz;
+    const size_t yb = (size_t)batch * h->h_out * h->w_out * d.c_out * 4;
+    void *x = nullptr, *y = nullptr;
+    cudaStream_t st = nullptr;
+    if (cudaMalloc(&x, std::max<size_t>(xb, 256)) != cudaSuccess || cudaMalloc(&y, std::max<size_t>(yb, 256)) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking) != cudaSuccess) {
+        if (x) cudaFree(x);
+        if (y) cudaFree(y);
+        cudaGetLastError();
+        return CADNN_E_ALLOC;
+    }
+    cudaMemsetAsync(x, 0, std::max<size_t>(xb, 256), st);
+    float best_us = -1.0f;
+    Schedule best = h->s;
+    for (const Candidate &c : pick) {
+        cadnn_weights tmp;
+        tmp.desc = d;
+        tmp.desc.flags &= ~CADNN_PACK_HOST_ONLY;
+        tmp.h_out = h->h_out;
+        tmp.w_out = h->w_out;
+        tmp.s = c.s;
+        if (build_sconv_image(&tmp, src, g, row_nnz) != CADNN_OK) continue;
+        if (upload(&tmp) != CADNN_OK) { if (tmp.d_blob) cudaFree(tmp.d_blob); continue; }
+        float us = time_schedule(&tmp, batch, x, y, st, 8);
+        if (us > 0.0f && (best_us < 0.0f || us < best_us)) {
+            best_us = us;
+            best = c.s;
+        }
+        cudaFree(tmp.d_blob);
+    }
+    cudaStreamDestroy(st);
+    cudaFree(x);
+    cudaFree(y);
+    h->s = best;
+    Geometry gg = g;
+    bool linear = best.kind == KK_SCONV_LINEAR;
+    finish_candidate(gg, h->s, linear);
+    return CADNN_OK;
+}
+
 cadnn_status pack_sconv(cadnn_weights *h, const Src &src)
 {
     const cadnn_layer_desc &d = h->desc;
@@ -417,6 +523,10 @@ cadnn_status pack_sconv(cadnn_weights *h, const Src &src)
     std::vector<Candidate> cands;
     enumerate_schedules(g, bh, linear, cands);
     h->s = cands[0].s;
+    if ((d.flags & CADNN_PACK_AUTOTUNE) && !(d.flags & CADNN_PACK_HOST_ONLY) && !getenv("CADNN_SCHEDULE")) {
+        cadnn_status st = autotune_sconv(h, src, g, row_nnz, cands);
+        if (st != CADNN_OK) return st;
+    }
     apply_env_override(g, linear, h->s);
     return build_sconv_image(h, src, g, row_nnz);
 }

@@ -28,6 +28,32 @@ namespace cg = cooperative_groups;
 
 namespace {
 
+// Division by a runtime constant as multiply-high and shift (the divisor is fixed per
+// launch; a hardware integer division costs a few dozen dependent instructions).
+// q = umulhi(n, mul) >> shr is exact for 0 <= n < 2^31 when mul = ceil(2^(32 + shr) / d)
+// and 2^shr >= d (shr chosen so that mul fits 32 bits); d == 1 is passed through.
+struct FastDiv {
+    unsigned mul, shr, d;
+};
+FastDiv make_fastdiv(int d)
+{
+    FastDiv f;
+    f.d = (unsigned)d;
+    f.mul = 0;
+    f.shr = 0;
+    if (d <= 1) return f;
+    unsigned l = 0;
+    while ((1u << l) < (unsigned)d) ++l;              // ceil(log2 d)
+    unsigned long long p2 = 1ull << (31 + l);
+    f.mul = (unsigned)((p2 + d - 1) / (unsigned long long)d);
+    f.shr = l - 1;
+    return f;
+}
+__device__ __forceinline__ unsigned fdiv(unsigned n, const FastDiv &f)
+{
+    return f.d == 1 ? n : (__umulhi(n, f.mul) >> f.shr);
+}
+
 struct SconvParams {
     const void *x;
     void *y;
@@ -39,7 +65,7 @@ struct SconvParams {
     int n, h, w, c_in, h_out, w_out, c_out;
     int stride, pad;
     int BW, RB, TBX, TBY, TH, TW, pitch, half, IH_t, IW_t;
-    int CIc, PPb, n_chunks, G, n_groups, stages;
+    int CIc, PPb, n_chunks, G, n_groups, stages, esz;
     int ksplit;   // thread blocks per cluster; each takes a contiguous range of the channel chunks
     int tiles_y, tiles_x;
     long long P;  // total output pixels (linear mode)
@@ -47,6 +73,9 @@ struct SconvParams {
     int tab_off;                  // byte offset of the pixel table / epilogue vectors in shared memory
     int hdr_bytes, block_bytes;   // per (chunk, filter block) record: row-start header + entries, fixed size
     int act, out_dtype, linear;
+    int ks_shift;                 // log2(ksplit)
+    int unit_ok;                  // activations are staged in 4-byte units (always for f32; int8 needs c_in % 4 == 0)
+    FastDiv d_groups, d_tiles_x, d_tiles_y, d_tbx, d_bw, d_cols_full;
 };
 
 // dst: 32-bit shared-window address
@@ -95,8 +124,9 @@ template <> struct Traits<int8_t> {
     static const int kUnitElems = 4;
 };
 
-// Per-block staging table, built once: for every staged input pixel its source pixel index
-// in x (-1 = zero padding / outside) and its byte offset inside a stage.
+// Per-block staging table, built once: for every staged input pixel the offset of its first
+// channel in x, in 4-byte units (the pixel index when activations are staged byte by byte;
+// -1 = zero padding / outside), and its byte offset inside a stage.
 __device__ __forceinline__ void build_pixel_table(const SconvParams &p, int2 *pix, int npx, int img, int oy0, int ox0,
                                                   long long p0)
 {
@@ -115,7 +145,8 @@ __device__ __forceinline__ void build_pixel_table(const SconvParams &p, int2 *pi
                     ip = (b * p.h + (long long)oy * p.stride) * p.w + (long long)ox * p.stride;
                 }
             }
-            pix[q] = make_int2((int)ip, q * p.PPb);
+            const int src = ip < 0 ? -1 : (p.unit_ok ? (int)(unsigned)((ip * p.c_in * (long long)p.esz) >> 2) : (int)ip);
+            pix[q] = make_int2(src, q * p.PPb);
         }
     } else {
         const int iy0 = oy0 * p.stride - p.pad, ix0 = ox0 * p.stride - p.pad;
@@ -123,7 +154,10 @@ __device__ __forceinline__ void build_pixel_table(const SconvParams &p, int2 *pi
             int r = i / p.IW_t, col = i - r * p.IW_t;
             int iy = iy0 + r, ix = ix0 + col;
             int src = -1;
-            if (iy >= 0 && iy < p.h && ix >= 0 && ix < p.w) src = (img * p.h + iy) * p.w + ix;
+            if (iy >= 0 && iy < p.h && ix >= 0 && ix < p.w) {
+                const long long ip = ((long long)img * p.h + iy) * p.w + ix;
+                src = p.unit_ok ? (int)(unsigned)((ip * p.c_in * p.esz) >> 2) : (int)ip;
+            }
             const int pos = p.half ? ((col & 1) * p.half + (col >> 1)) : col;
             pix[i] = make_int2(src, (r * p.pitch + pos) * p.PPb);
         }
@@ -144,36 +178,58 @@ __device__ __forceinline__ void stage_weights(const SconvParams &p, unsigned st3
 // Asynchronous copies that stage the activation tile of chunk c: pixel-major, PPb bytes per
 // pixel, 4 bytes per copy.
 template <typename XT>
-__device__ __forceinline__ void stage_acts(const SconvParams &p, const int2 *pixtab, int npx, unsigned char *smem,
-                                           unsigned smem32, unsigned stage_off, int c)
+__device__ __forceinline__ void stage_acts(const SconvParams &p, const int2 *pixtab, int npx, long long p0,
+                                           unsigned char *smem, unsigned smem32, unsigned stage_off, int c)
 {
     typedef Traits<XT> TR;
     const int tid = threadIdx.x, NT = blockDim.x;
     const int c0 = c * p.CIc;
     const XT *xg = reinterpret_cast<const XT *>(p.x);
     const unsigned st32 = smem32 + stage_off;
-    const bool unit_ok = (TR::kUnitElems == 1) || ((p.c_in & 3) == 0);
-    if (unit_ok) {
+    if (p.unit_ok) {
         const int upp = p.CIc / TR::kUnitElems;   // 4-byte units per staged pixel
-        const int total = npx * upp;
-        if ((upp & (upp - 1)) == 0) {
+        const unsigned char *xb = reinterpret_cast<const unsigned char *>(p.x);
+        if ((upp & (upp - 1)) == 0 && upp <= NT && pixtab == nullptr) {
+            // flat pixel range at stride 1: source and destination follow from the pixel number
             const int sh = 31 - __clz(upp);
+            const int u = tid & (upp - 1);
+            const int ci = c0 + u * TR::kUnitElems;
+            const bool ch_ok = ci < p.c_in;
+            const size_t pix_bytes = (size_t)p.c_in * sizeof(XT);
+            const unsigned char *xcol = xb + (size_t)p0 * pix_bytes + (size_t)ci * sizeof(XT);
+            const unsigned dcol = st32 + u * 4;
+            const int pstep = NT >> sh;
+            const long long left = p.P - p0;   // pixels that exist from p0 on
 #pragma unroll 4
-            for (int idx = tid; idx < total; idx += NT) {
-                const int pix = idx >> sh, u = idx & (upp - 1);
+            for (int pix = tid >> sh; pix < npx; pix += pstep) {
+                const bool ok = ch_ok && pix < left;
+                const unsigned char *src = ok ? xcol + (size_t)pix * pix_bytes : xb;
+                cp_async4(dcol + pix * p.PPb, src, ok);
+            }
+        } else if ((upp & (upp - 1)) == 0 && upp <= NT) {
+            // each thread keeps one unit column and walks the pixels
+            const int sh = 31 - __clz(upp);
+            const int u = tid & (upp - 1);
+            const int ci = c0 + u * TR::kUnitElems;
+            const bool ch_ok = ci < p.c_in;
+            const unsigned char *xcol = xb + (size_t)ci * sizeof(XT);
+            const unsigned dcol = st32 + u * 4;
+            const int pstep = NT >> sh;
+#pragma unroll 4
+            for (int pix = tid >> sh; pix < npx; pix += pstep) {
                 const int2 te = pixtab[pix];
-                const int ci = c0 + u * TR::kUnitElems;
-                const bool ok = te.x >= 0 && ci < p.c_in;
-                const XT *src = ok ? xg + (size_t)te.x * p.c_in + ci : xg;
-                cp_async4(st32 + te.y + u * 4, src, ok);
+                const bool ok = ch_ok && te.x != -1;
+                const unsigned char *src = ok ? xcol + ((size_t)(unsigned)te.x << 2) : xb;
+                cp_async4(dcol + te.y, src, ok);
             }
         } else {
+            const int total = npx * upp;
             for (int idx = tid; idx < total; idx += NT) {
                 const int pix = idx / upp, u = idx - pix * upp;
                 const int2 te = pixtab[pix];
                 const int ci = c0 + u * TR::kUnitElems;
-                const bool ok = te.x >= 0 && ci < p.c_in;
-                const XT *src = ok ? xg + (size_t)te.x * p.c_in + ci : xg;
+                const bool ok = te.x != -1 && ci < p.c_in;
+                const unsigned char *src = ok ? xb + ((size_t)(unsigned)te.x << 2) + (size_t)ci * sizeof(XT) : xb;
                 cp_async4(st32 + te.y + u * 4, src, ok);
             }
         }
@@ -186,7 +242,7 @@ __device__ __forceinline__ void stage_acts(const SconvParams &p, const int2 *pix
             const int2 te = pixtab[pix];
             const int ci = c0 + cl;
             XT v = 0;
-            if (te.x >= 0 && ci < p.c_in) v = xg[(size_t)te.x * p.c_in + ci];
+            if (te.x != -1 && ci < p.c_in) v = xg[(size_t)te.x * p.c_in + ci];
             stage[te.y + cl] = v;
         }
     }
@@ -202,10 +258,10 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int KS = p.ksplit;
-    const int rank = blockIdx.x % KS;
-    const int rest = blockIdx.x / KS;
-    const int grp = rest % p.n_groups;
-    int tile = rest / p.n_groups;
+    const int rank = blockIdx.x & (KS - 1);
+    const unsigned rest = blockIdx.x >> p.ks_shift;
+    unsigned tile = fdiv(rest, p.d_groups);
+    const int grp = (int)(rest - tile * p.n_groups);
     const int G = p.G;
 
     // tile origin
@@ -214,10 +270,11 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
     if (p.linear) {
         p0 = (long long)tile * (32 * T);
     } else {
-        int tx = tile % p.tiles_x;
-        tile /= p.tiles_x;
-        int ty = tile % p.tiles_y;
-        img = tile / p.tiles_y;
+        const unsigned t1 = fdiv(tile, p.d_tiles_x);
+        const int tx = (int)(tile - t1 * p.tiles_x);
+        const unsigned t2 = fdiv(t1, p.d_tiles_y);
+        const int ty = (int)(t1 - t2 * p.tiles_y);
+        img = (int)t2;
         oy0 = ty * p.TH;
         ox0 = tx * p.TW;
     }
@@ -235,11 +292,11 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
 #pragma unroll
         for (int t = 0; t < T; ++t) band[t] = t * 32 * p.PPb;
     } else {
-        const int lr = lane / p.BW, lc = lane - lr * p.BW;
+        const int lr = (int)fdiv(lane, p.d_bw), lc = lane - lr * p.BW;
         lanebase = (lr < p.RB) ? ((lr * p.stride) * p.pitch + lc * xs) * p.PPb : 0;
 #pragma unroll
         for (int t = 0; t < T; ++t) {
-            const int ty = t / p.TBX, tx = t - ty * p.TBX;
+            const int ty = (int)fdiv(t, p.d_tbx), tx = t - ty * p.TBX;
             band[t] = ((ty * p.RB * p.stride) * p.pitch + tx * p.BW * xs) * p.PPb;
         }
     }
@@ -256,11 +313,16 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
     int2 *pixtab = reinterpret_cast<int2 *>(smem + p.tab_off);
     float *sScale = reinterpret_cast<float *>(pixtab + npx_in);
     float *sBias = sScale + G;
-    build_pixel_table(p, pixtab, npx_in, img, oy0, ox0, p0);
-    for (int i = tid; i < G; i += blockDim.x) {
-        const int co = grp * G + i;
-        sScale[i] = (p.scale && co < p.c_out) ? p.scale[co] : 1.0f;
-        sBias[i] = (p.bias && co < p.c_out) ? p.bias[co] : 0.0f;
+    const int upp_chk = p.CIc / TR::kUnitElems;
+    const bool direct = p.linear && p.stride == 1 && p.unit_ok && (upp_chk & (upp_chk - 1)) == 0 &&
+                        upp_chk <= (int)blockDim.x;
+    if (direct) pixtab = nullptr;   // no table needed
+    else build_pixel_table(p, pixtab, npx_in, img, oy0, ox0, p0);
+    if (tid < G) {   // epilogue vectors ride in the first copy group
+        const int co = grp * G + tid;
+        const unsigned ds = smem32 + p.tab_off + npx_in * 8 + tid * 4;
+        if (p.scale && co < p.c_out) cp_async4(ds, p.scale + co, true); else sScale[tid] = 1.0f;
+        if (p.bias && co < p.c_out) cp_async4(ds + G * 4, p.bias + co, true); else sBias[tid] = 0.0f;
     }
     int co_of[RPW];
 #pragma unroll
@@ -274,7 +336,7 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
     grid_dep_wait();          // x (and the residual) are final from here on
     grid_dep_trigger();
     for (int s = 0; s < npre; ++s) {
-        if (c_lo + s < c_hi) stage_acts<XT>(p, pixtab, npx_in, smem, smem32, (unsigned)(s * p.stage_bytes), c_lo + s);
+        if (c_lo + s < c_hi) stage_acts<XT>(p, pixtab, npx_in, p0, smem, smem32, (unsigned)(s * p.stage_bytes), c_lo + s);
         cp_async_commit();
     }
 
@@ -284,7 +346,7 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
             if (c > c_lo) {
                 __syncthreads();   // everyone is done with chunk c - 1
                 stage_weights(p, smem32, c, grp);
-                stage_acts<XT>(p, pixtab, npx_in, smem, smem32, 0u, c);
+                stage_acts<XT>(p, pixtab, npx_in, p0, smem, smem32, 0u, c);
                 cp_async_commit();
             }
             cp_async_wait<0>();
@@ -297,7 +359,7 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
             if (nbuf >= S) nbuf -= S;
             if (nxt < c_hi) {
                 stage_weights(p, smem32 + (unsigned)(nbuf * p.stage_bytes), nxt, grp);
-                stage_acts<XT>(p, pixtab, npx_in, smem, smem32, (unsigned)(nbuf * p.stage_bytes), nxt);
+                stage_acts<XT>(p, pixtab, npx_in, p0, smem, smem32, (unsigned)(nbuf * p.stage_bytes), nxt);
             }
             cp_async_commit();
         }
@@ -375,16 +437,18 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
     const bool has_res = p.residual != nullptr;
     const bool quad = ((gw & 3) == 0) && ((p.c_out & 3) == 0);
     const int cols = quad ? (gw >> 2) : gw;
+    const bool full = quad && gw == G;   // the usual case: a precomputed divisor
     for (int idx = tid + q_lo * cols; idx < q_hi * cols; idx += blockDim.x) {
-        const int q = idx / cols, cq = idx - q * cols;
+        const int q = full ? (int)fdiv(idx, p.d_cols_full) : idx / cols;
+        const int cq = idx - q * cols;
         long long opix;
         if (p.linear) {
             opix = p0 + q;
             if (opix >= p.P) continue;
         } else {
             const int t = q >> 5, l = q & 31;
-            const int ty = t / p.TBX, tx = t - ty * p.TBX;
-            const int lr = l / p.BW, lcx = l - lr * p.BW;
+            const int ty = (int)fdiv(t, p.d_tbx), tx = t - ty * p.TBX;
+            const int lr = (int)fdiv(l, p.d_bw), lcx = l - lr * p.BW;
             const int oy = oy0 + ty * p.RB + lr, ox = ox0 + tx * p.BW + lcx;
             if (lr >= p.RB || oy >= p.h_out || ox >= p.w_out) continue;
             opix = ((long long)img * p.h_out + oy) * p.w_out + ox;
@@ -540,6 +604,9 @@ cadnn_status launch_sconv(const cadnn_weights *w, const void *x, int n, void *y,
     p.block_bytes = p.hdr_bytes + s.max_entries * (s8 ? 4 : 8);
     p.act = ep.act;
     p.out_dtype = ep.out_dtype;
+    p.esz = s8 ? 1 : 4;
+    p.unit_ok = (!s8 || (d.c_in & 3) == 0) ? 1 : 0;
+    p.ks_shift = s.ksplit == 8 ? 3 : s.ksplit == 4 ? 2 : s.ksplit == 2 ? 1 : 0;
     long long tiles;
     if (p.linear) {
         p.tiles_x = p.tiles_y = 1;
@@ -549,8 +616,16 @@ cadnn_status launch_sconv(const cadnn_weights *w, const void *x, int n, void *y,
         p.tiles_x = (w->w_out + s.TW - 1) / s.TW;
         tiles = (long long)n * p.tiles_y * p.tiles_x;
     }
+    p.d_groups = make_fastdiv(s.n_groups);
+    p.d_tiles_x = make_fastdiv(p.tiles_x);
+    p.d_tiles_y = make_fastdiv(p.tiles_y);
+    p.d_tbx = make_fastdiv(s.TBX);
+    p.d_bw = make_fastdiv(s.BW);
+    p.d_cols_full = make_fastdiv(std::max(1, s.G / 4));
     long long blocks = tiles * s.n_groups * s.ksplit;
     if (blocks <= 0) return CADNN_OK;
+    // the staging table addresses x in 4-byte units through 32 bits
+    if ((long long)n * d.in_h * d.in_w * d.c_in * p.esz >= (1LL << 34)) return CADNN_E_UNSUPPORTED;
     if (blocks > 2147483647LL) return CADNN_E_UNSUPPORTED;
     if (s8) return launch_T<int8_t>(p, s.T, s.RPW, (int)blocks, s.NW * 32, s.smem_bytes, ep.pdl, st);
     return launch_T<float>(p, s.T, s.RPW, (int)blocks, s.NW * 32, s.smem_bytes, ep.pdl, st);

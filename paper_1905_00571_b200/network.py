@@ -7,15 +7,15 @@ import torch
 from . import binding as B
 
 
-def desc_for(op, dtype, batch_hint=1):
+def desc_for(op, dtype, batch_hint=1, autotune=False):
     if op.kind == "fc":
-        return B.make_desc(op.c_in, op.c_out, 1, 1, 1, 0, 1, 1, 1, batch_hint, dtype)
+        return B.make_desc(op.c_in, op.c_out, 1, 1, 1, 0, 1, 1, 1, batch_hint, dtype, autotune=autotune)
     return B.make_desc(op.c_in, op.c_out, op.k, op.k, op.stride, op.pad, op.groups,
-                       op.in_hw[0], op.in_hw[1], batch_hint, dtype)
+                       op.in_hw[0], op.in_hw[1], batch_hint, dtype, autotune=autotune)
 
 
-def pack_op(op, dtype, batch_hint=1):
-    d = desc_for(op, dtype, batch_hint)
+def pack_op(op, dtype, batch_hint=1, autotune=False):
+    d = desc_for(op, dtype, batch_hint, autotune)
     if op.w.dtype == np.int8:
         return B.cadnn_pack_q8(d, op.w, op.mask)
     return B.cadnn_pack(d, op.w, op.mask)
@@ -24,7 +24,7 @@ def pack_op(op, dtype, batch_hint=1):
 class PackedModel:
     """Packed weights + device epilogue vectors + cadnn_net for one batch size."""
 
-    def __init__(self, model, batch=1, device="cuda:0"):
+    def __init__(self, model, batch=1, device="cuda:0", autotune=False):
         self.model = model
         self.batch = batch
         self.device = torch.device(device)
@@ -34,7 +34,7 @@ class PackedModel:
         with torch.cuda.device(self.device):
             for i, op in enumerate(model.ops):
                 if op.kind in ("conv", "fc"):
-                    w = pack_op(op, model.dtype, batch)
+                    w = pack_op(op, model.dtype, batch, autotune)
                     self.weights[i] = w
                     sc = None if op.scale is None else torch.from_numpy(op.scale).to(self.device)
                     bi = None if op.bias is None else torch.from_numpy(op.bias).to(self.device)
