@@ -212,9 +212,9 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
  * cadnn_forward - run the network: x device input, y device output of the last op.
  * use_graph != 0 replays a CUDA graph captured on the first call with this (x, y)
  * pair (re-captured when either pointer changes); 0 launches the layers one by one.
- * Layers after the first are launched as programmatic dependents of their predecessor
- * (their weight fetch overlaps its tail); set CADNN_NO_PDL in the environment before
- * cadnn_net_create to use plain stream order instead.
+ * Without a graph, layers after the first are launched as programmatic dependents of
+ * their predecessor (their weight fetch overlaps its stores); set CADNN_NO_PDL in the
+ * environment before cadnn_net_create to use plain stream order instead.
  * Asynchronous on stream.
  */
 cadnn_status cadnn_forward(cadnn_net *net, const void *x, void *y, int use_graph, void *stream);

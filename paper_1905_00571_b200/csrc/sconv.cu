@@ -334,7 +334,6 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
         if (c_lo + s < c_hi) stage_weights(p, smem32 + (unsigned)(s * p.stage_bytes), c_lo + s, grp);
     __syncthreads();          // the pixel table is complete
     grid_dep_wait();          // x (and the residual) are final from here on
-    grid_dep_trigger();
     for (int s = 0; s < npre; ++s) {
         if (c_lo + s < c_hi) stage_acts<XT>(p, pixtab, npx_in, p0, smem, smem32, (unsigned)(s * p.stage_bytes), c_lo + s);
         cp_async_commit();
@@ -430,6 +429,9 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
         }
     }
     __syncthreads();
+    // The next layer may start its prologue now: it overlaps this block's stores and the
+    // tail of the grid without competing with the multiply-add loop.
+    grid_dep_trigger();
 
     // ---- epilogue and contiguous NHWC stores ----
     const int co_base = grp * G;
