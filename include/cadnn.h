@@ -227,6 +227,42 @@ cadnn_status cadnn_forward(cadnn_net *net, const void *x, void *y, int use_graph
  */
 cadnn_status cadnn_forward_host(cadnn_net *net, const void *x_host, void *y_host, int use_graph, void *stream);
 
+/*
+ * cadnn_forward_static - run an op list WITHOUT allocating anything.  (The paper has no
+ * counterpart of this call; it exists for deployment.)
+ *
+ * cadnn_net_create gives every intermediate tensor a cudaMalloc'ed buffer, and doing
+ * that again for each new batch size allocates again.  Some callers must not allocate
+ * while they run a network: a serving thread on its latency path (cudaMalloc and
+ * cudaFree synchronize the whole device and stall every other stream), a process whose
+ * device memory has already been handed in full to a framework's caching allocator, or
+ * code that meets a batch size it built no cadnn_net for.  This call takes the same op
+ * list as cadnn_net_create (weights packed earlier, scale / bias vectors on the device)
+ * plus the input shape, and places the intermediate tensors in a fixed device array of
+ * CADNN_STATIC_WORKSPACE_BYTES that is part of the library image: every GPU that loads
+ * the library holds that much memory until the process exits.  Regions are reused as
+ * soon as the last op reading them has been issued.  It calls no cudaMalloc, cudaFree or
+ * other allocating routine, on the device or on the host heap; at most 512 ops.
+ *
+ *   x  device input [n][h][w][c] of in_dtype; y device output of the last op; both the
+ *      caller's.  Asynchronous on stream; the layers run in stream order, one by one.
+ * Errors: E_ARG / E_SHAPE / E_DTYPE as cadnn_net_create; E_UNSUPPORTED when the
+ * intermediate tensors of this input shape do not fit the fixed workspace (or the list
+ * has more than 512 ops) - nothing has been launched in that case.
+ *
+ * The first call on a device looks up the array's device address (with that device
+ * current); make that first call before any stream capture.  All calls on a device
+ * share the one array, which keeps whatever the previous call left there: nothing in it
+ * needs clearing, because every tensor is written in full before it is read, but two
+ * calls that overlap on the GPU (different streams, or the same stream from two threads
+ * without ordering) race on it, as does a call that overlaps a kernel still reading the
+ * previous call's intermediates.  The output y is safe to read once stream has reached
+ * the end of the call's work.
+ */
+#define CADNN_STATIC_WORKSPACE_BYTES (32 << 20)
+cadnn_status cadnn_forward_static(const cadnn_op *ops, int n_ops, int n, int h, int wd, int c, int in_dtype,
+                                  const void *x, void *y, void *stream);
+
 /* Number of kernel launches one forward issues; bytes of slot memory the net owns. */
 cadnn_status cadnn_net_info(const cadnn_net *net, int *n_launches, int64_t *workspace_bytes);
 

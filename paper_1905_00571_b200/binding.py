@@ -62,6 +62,7 @@ _SIGS = {
     "cadnn_net_create": (_i, [ctypes.POINTER(Op), _i, _i, _i, _i, _i, _i, ctypes.POINTER(_vp)]),
     "cadnn_forward": (_i, [_vp, _vp, _vp, _i, _vp]),
     "cadnn_forward_host": (_i, [_vp, _vp, _vp, _i, _vp]),
+    "cadnn_forward_static": (_i, [ctypes.POINTER(Op), _i, _i, _i, _i, _i, _i, _vp, _vp, _vp]),
     "cadnn_net_info": (_i, [_vp, ctypes.POINTER(_i), _i64p]),
     "cadnn_net_layer_times": (_i, [_vp, _vp, _vp, _i, _i, ctypes.POINTER(ctypes.c_float), _vp]),
     "cadnn_net_slot": (_i, [_vp, _i, ctypes.POINTER(_vp), _i64p]),
@@ -267,6 +268,19 @@ def cadnn_forward_host(net, x_host, y_host, use_graph=True, stream=None):
     _check(_lib.cadnn_forward_host(net.handle, ctypes.c_void_p(xp), ctypes.c_void_p(yp), 1 if use_graph else 0,
                                    _stream(stream)), "cadnn_forward_host")
     return y_host
+
+
+STATIC_WORKSPACE_BYTES = 32 << 20
+
+
+def cadnn_forward_static(ops, x, y, in_dtype, stream=None):
+    """Run the op list on x (NHWC torch CUDA tensor) into y without allocating: intermediates live
+    in the library's fixed device workspace (STATIC_WORKSPACE_BYTES); see include/cadnn.h."""
+    arr = (Op * len(ops))(*ops)
+    n, h, w, c = (int(v) for v in x.shape)
+    _check(_lib.cadnn_forward_static(arr, len(ops), n, h, w, c, DTYPE[in_dtype] if not isinstance(in_dtype, int) else in_dtype,
+                                     _dev_ptr(x), _dev_ptr(y), _stream(stream)), "cadnn_forward_static")
+    return y
 
 
 def cadnn_net_info(net):

@@ -50,6 +50,7 @@ class PackedModel:
                 else:
                     raise ValueError(op.kind)
             h, w_, c = model.in_shape
+            self.ops = ops
             self.net = B.cadnn_net_create(ops, batch, h, w_, c, model.dtype, keep=(self.weights, self.vecs))
         last = model.ops[-1]
         self.out_shape = (batch, last.c_out) if last.kind in ("fc", "gavgpool") else (batch, last.out_hw[0], last.out_hw[1], last.c_out)
@@ -62,6 +63,10 @@ class PackedModel:
         if y is None:
             y = self.new_output()
         return B.cadnn_forward(self.net, x, y, use_graph, stream)
+
+    def forward_static(self, x, y, stream=None):
+        """Same layers through cadnn_forward_static (no allocation; any batch that fits the fixed workspace)."""
+        return B.cadnn_forward_static(self.ops, x, y, self.model.dtype, stream)
 
     def forward_host(self, x_host, y_host, use_graph=True, stream=None):
         return B.cadnn_forward_host(self.net, x_host, y_host, use_graph, stream)
