@@ -383,7 +383,7 @@ cadnn_status build_sconv_image(cadnn_weights *h, const Src &src, const Geometry 
                 s.max_entries = std::max(s.max_entries, running);
             }
         }
-        s.max_entries = round_up(std::max(s.max_entries, 2), 4);
+        s.max_entries = round_up(std::max(s.max_entries, 2) + 2, 4);   // + one pair of slack for the kernel's look-ahead
         finish_smem(s, s8);
         // A dense or skewed layer can overflow the stage budget: halve the chunk and repack.
         if ((s.stage_bytes > kMaxStageBytes || s.smem_bytes > kSmemPerSm) && s.CIc > (s8 ? 4 : 1) && attempt < 8) {

@@ -370,25 +370,36 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
         for (int j = 0; j < RPW; ++j) {
             const int row = warp * RPW + j;
             const int beg = sP[row], end = sP[row + 1];
+            // software pipeline: the next pair of nonzeros is fetched while this pair is used
+            // (reading one pair past the row stays inside the record: the packer leaves slack)
+            if (TR::kEntryBytes == 8) {
+                uint4 nx = *reinterpret_cast<const uint4 *>(smem + sW + beg * 8);
 #pragma unroll 2
-            for (int e = beg; e < end; e += 2) {
-                AT w0, w1;
-                unsigned o0, o1;
-                if (TR::kEntryBytes == 8) {
-                    const uint4 v = *reinterpret_cast<const uint4 *>(smem + sW + e * 8);
-                    w0 = (AT)__uint_as_float(v.x); o0 = v.y;
-                    w1 = (AT)__uint_as_float(v.z); o1 = v.w;
-                } else {
-                    const uint2 v = *reinterpret_cast<const uint2 *>(smem + sW + e * 4);
-                    w0 = (AT)(int)(int8_t)(v.x & 0xffu); o0 = v.x >> 8;
-                    w1 = (AT)(int)(int8_t)(v.y & 0xffu); o1 = v.y >> 8;
+                for (int e = beg; e < end; e += 2) {
+                    const uint4 v = nx;
+                    nx = *reinterpret_cast<const uint4 *>(smem + sW + (e + 2) * 8);
+                    const AT w0 = (AT)__uint_as_float(v.x), w1 = (AT)__uint_as_float(v.z);
+                    const unsigned a0 = lanep + v.y;
+                    const unsigned a1 = lanep + v.w;
+#pragma unroll
+                    for (int t = 0; t < T; ++t) acc[j][t] += w0 * (AT)(*reinterpret_cast<const XT *>(smem + a0 + band[t]));
+#pragma unroll
+                    for (int t = 0; t < T; ++t) acc[j][t] += w1 * (AT)(*reinterpret_cast<const XT *>(smem + a1 + band[t]));
                 }
-                const unsigned a0 = lanep + o0;
-                const unsigned a1 = lanep + o1;
+            } else {
+                uint2 nx = *reinterpret_cast<const uint2 *>(smem + sW + beg * 4);
+#pragma unroll 2
+                for (int e = beg; e < end; e += 2) {
+                    const uint2 v = nx;
+                    nx = *reinterpret_cast<const uint2 *>(smem + sW + (e + 2) * 4);
+                    const AT w0 = (AT)(int)(int8_t)(v.x & 0xffu), w1 = (AT)(int)(int8_t)(v.y & 0xffu);
+                    const unsigned a0 = lanep + (v.x >> 8);
+                    const unsigned a1 = lanep + (v.y >> 8);
 #pragma unroll
-                for (int t = 0; t < T; ++t) acc[j][t] += w0 * (AT)(*reinterpret_cast<const XT *>(smem + a0 + band[t]));
+                    for (int t = 0; t < T; ++t) acc[j][t] += w0 * (AT)(*reinterpret_cast<const XT *>(smem + a0 + band[t]));
 #pragma unroll
-                for (int t = 0; t < T; ++t) acc[j][t] += w1 * (AT)(*reinterpret_cast<const XT *>(smem + a1 + band[t]));
+                    for (int t = 0; t < T; ++t) acc[j][t] += w1 * (AT)(*reinterpret_cast<const XT *>(smem + a1 + band[t]));
+                }
             }
         }
         if (++buf == S) buf = 0;
