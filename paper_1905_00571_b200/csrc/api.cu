@@ -60,6 +60,7 @@ cadnn_status conv2d_impl(const cadnn_weights *w, const void *x, int n, int h, in
         case KK_SCONV_LINEAR: return launch_sconv(w, x, n, y, le, s);
         case KK_FC_SPMV: return launch_fc_spmv(w, x, n, y, le, s);
         case KK_DW: return launch_dw(w, x, n, y, le, s);
+        case KK_DENSE_SMALLC: return launch_dense_smallc(w, x, n, y, le, s);
     }
     return CADNN_E_UNSUPPORTED;
 }

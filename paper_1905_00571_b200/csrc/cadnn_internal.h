@@ -59,6 +59,7 @@ struct cadnn_weights {
     std::vector<int32_t> ptr;        // fc: [c_pad + 1]
     std::vector<int32_t> perm;       // packed row -> original output channel, -1 = padding row
     std::vector<float> dense_f;      // dense kinds: tap-major weights
+    std::vector<uint8_t> dense_kept; // dense kinds: which positions the mask kept (host only, for unpack)
     int c_pad = 0;
 
     // device image (one allocation)
@@ -95,6 +96,8 @@ cadnn_status launch_fc_spmv(const cadnn_weights *w, const void *x, int n, void *
                             cudaStream_t st);
 cadnn_status launch_dw(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
                        cudaStream_t st);
+cadnn_status launch_dense_smallc(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
+                                 cudaStream_t st);
 cadnn_status launch_maxpool(const void *x, int n, int h, int wd, int c, int k, int stride, int pad, int dtype,
                             void *y, bool pdl, cudaStream_t st);
 cadnn_status launch_gavgpool(const float *x, int n, int h, int wd, int c, float *y, bool pdl, cudaStream_t st);

@@ -78,6 +78,108 @@ __global__ void __launch_bounds__(256) dw_kernel(const DwParams p)
     }
 }
 
+
+// Dense convolution with very few input channels (the network stem: 7x7 or 3x3, stride 2,
+// 3 -> 32/64 channels).  Genuinely dense, so it is register-tiled like a small GEMM: a warp
+// owns 32 output columns x 2 output rows and 16 output channels; per tap it reads 2
+// activations per lane and 16 weights as four broadcast 16-byte loads, and issues 32 FMAs.
+struct StemParams {
+    const float *x;
+    float *y;
+    const float *wt;   // [taps][c_out], taps = (ky*kw + kx)*c_in + ci
+    const float *scale;
+    const float *bias;
+    const float *residual;
+    int n, h, w, c_in, c_out, h_out, w_out, kh, kw, stride, pad, act;
+    int tiles_x, tiles_y, in_rows, in_cols, taps, co_blocks;
+};
+
+const int kStemCo = 16;      // output channels per warp
+const int kStemRows = 4;     // output rows per block (2 warps down x 2 rows per lane)
+const int kStemCoBlock = 64; // output channels per block (4 warps across channels)
+
+__global__ void __launch_bounds__(256) stem_kernel(const StemParams p)
+{
+    extern __shared__ __align__(16) float sm[];
+    float *sW = sm;                                   // [taps][64]
+    float *sIn = sm + (size_t)p.taps * kStemCoBlock;  // [in_rows][in_cols][c_in]
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int b = blockIdx.x;
+    const int cb = b % p.co_blocks; b /= p.co_blocks;
+    const int tx = b % p.tiles_x; b /= p.tiles_x;
+    const int ty = b % p.tiles_y;
+    const int img = b / p.tiles_y;
+    const int ox0 = tx * 32, oy0 = ty * kStemRows, co0 = cb * kStemCoBlock;
+
+    // weights of this block's 64 channels (static data: before the grid-dependency wait)
+    for (int i = tid; i < p.taps * kStemCoBlock; i += blockDim.x) {
+        const int t = i / kStemCoBlock, c = i - t * kStemCoBlock;
+        sW[i] = (co0 + c < p.c_out) ? p.wt[(size_t)t * p.c_out + co0 + c] : 0.0f;
+    }
+    grid_dep_wait();
+    grid_dep_trigger();
+    const int iy0 = oy0 * p.stride - p.pad, ix0 = ox0 * p.stride - p.pad;
+    const int row_words = p.in_cols * p.c_in;
+    for (int i = tid; i < p.in_rows * row_words; i += blockDim.x) {
+        const int r = i / row_words, rem = i - r * row_words;
+        const int col = rem / p.c_in, ci = rem - col * p.c_in;
+        const int iy = iy0 + r, ix = ix0 + col;
+        float v = 0.0f;
+        if (iy >= 0 && iy < p.h && ix >= 0 && ix < p.w) v = p.x[(((size_t)img * p.h + iy) * p.w + ix) * p.c_in + ci];
+        sIn[i] = v;
+    }
+    __syncthreads();
+
+    const int wc = warp & 3, wr = warp >> 2;          // channel group, row pair
+    const int ly = wr * 2;                            // first of this lane's two output rows
+    float acc0[kStemCo], acc1[kStemCo];
+#pragma unroll
+    for (int c = 0; c < kStemCo; ++c) acc0[c] = acc1[c] = 0.0f;
+    const float *w_base = sW + wc * kStemCo;
+    const float *in0 = sIn + ((ly * p.stride) * p.in_cols + lane * p.stride) * p.c_in;
+    const float *in1 = in0 + p.stride * row_words;
+    int t = 0;
+    for (int ky = 0; ky < p.kh; ++ky) {
+        const float *r0 = in0 + ky * row_words, *r1 = in1 + ky * row_words;
+        for (int k = 0; k < p.kw * p.c_in; ++k, ++t) {
+            const float a0 = r0[k], a1 = r1[k];
+            const float4 *wq = reinterpret_cast<const float4 *>(w_base + t * kStemCoBlock);
+#pragma unroll
+            for (int q = 0; q < kStemCo / 4; ++q) {
+                const float4 wv = wq[q];
+                acc0[4 * q + 0] = fmaf(a0, wv.x, acc0[4 * q + 0]);
+                acc0[4 * q + 1] = fmaf(a0, wv.y, acc0[4 * q + 1]);
+                acc0[4 * q + 2] = fmaf(a0, wv.z, acc0[4 * q + 2]);
+                acc0[4 * q + 3] = fmaf(a0, wv.w, acc0[4 * q + 3]);
+                acc1[4 * q + 0] = fmaf(a1, wv.x, acc1[4 * q + 0]);
+                acc1[4 * q + 1] = fmaf(a1, wv.y, acc1[4 * q + 1]);
+                acc1[4 * q + 2] = fmaf(a1, wv.z, acc1[4 * q + 2]);
+                acc1[4 * q + 3] = fmaf(a1, wv.w, acc1[4 * q + 3]);
+            }
+        }
+    }
+
+    const int ox = ox0 + lane;
+    const int cbase = co0 + wc * kStemCo;
+    if (ox < p.w_out) {
+#pragma unroll
+        for (int rr = 0; rr < 2; ++rr) {
+            const int oy = oy0 + ly + rr;
+            if (oy >= p.h_out) continue;
+            const float *acc = rr ? acc1 : acc0;
+            const size_t o = (((size_t)img * p.h_out + oy) * p.w_out + ox) * p.c_out + cbase;
+#pragma unroll
+            for (int c = 0; c < kStemCo; ++c) {
+                const int co = cbase + c;
+                if (co >= p.c_out) break;
+                float z = fmaf(acc[c], p.scale ? p.scale[co] : 1.0f, p.bias ? p.bias[co] : 0.0f);
+                if (p.residual) z += p.residual[o + c];
+                p.y[o + c] = dw_act(z, p.act);
+            }
+        }
+    }
+}
+
 }  // namespace
 
 cadnn_status launch_dw(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
@@ -96,4 +198,33 @@ cadnn_status launch_dw(const cadnn_weights *w, const void *x, int n, void *y, co
     if (blocks > 148LL * 64) blocks = 148LL * 64;
     if (v4) return launch_kernel(dw_kernel<4>, (int)blocks, 256, 0, ep.pdl, st, p);
     return launch_kernel(dw_kernel<1>, (int)blocks, 256, 0, ep.pdl, st, p);
+}
+
+cadnn_status launch_dense_smallc(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
+                                 cudaStream_t st)
+{
+    const cadnn_layer_desc &d = w->desc;
+    StemParams p;
+    p.x = (const float *)x; p.y = (float *)y; p.wt = w->d_dense;
+    p.scale = ep.scale; p.bias = ep.bias; p.residual = (const float *)ep.residual;
+    p.n = n; p.h = d.in_h; p.w = d.in_w; p.c_in = d.c_in; p.c_out = d.c_out;
+    p.h_out = w->h_out; p.w_out = w->w_out; p.kh = d.kh; p.kw = d.kw; p.stride = d.stride; p.pad = d.pad;
+    p.act = ep.act;
+    p.tiles_x = (w->w_out + 31) / 32;
+    p.tiles_y = (w->h_out + kStemRows - 1) / kStemRows;
+    p.in_rows = (kStemRows - 1) * d.stride + d.kh;
+    p.in_cols = 31 * d.stride + d.kw;
+    p.taps = d.kh * d.kw * d.c_in;
+    p.co_blocks = (d.c_out + kStemCoBlock - 1) / kStemCoBlock;
+    long long blocks = (long long)n * p.tiles_y * p.tiles_x * p.co_blocks;
+    if (blocks <= 0) return CADNN_OK;
+    if (blocks > 2147483647LL) return CADNN_E_UNSUPPORTED;
+    size_t smem = ((size_t)p.taps * kStemCoBlock + (size_t)p.in_rows * p.in_cols * d.c_in) * 4;
+    static size_t smem_allowed = 48 * 1024;
+    if (smem > smem_allowed) {
+        if (smem > 200 * 1024) return CADNN_E_UNSUPPORTED;
+        CADNN_CUDA_TRY(cudaFuncSetAttribute(stem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        smem_allowed = smem;
+    }
+    return launch_kernel(stem_kernel, (int)blocks, 256, smem, ep.pdl, st, p);
 }

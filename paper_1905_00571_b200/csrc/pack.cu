@@ -259,7 +259,7 @@ void enumerate_schedules(const Geometry &g, int batch, bool linear, std::vector<
     }
     const int tbx_full = std::min(8, nbx_total);
     for (int nw : {16, 8, 4})
-        for (int rpw : {4, 2, 1})
+        for (int rpw : {16, 8, 4, 2, 1})
             for (int cic : cics)
                 for (int ks : {1, 2, 4, 8})
                     for (int tbx = 1; tbx <= (linear ? 8 : tbx_full); ++tbx)
@@ -267,6 +267,8 @@ void enumerate_schedules(const Geometry &g, int batch, bool linear, std::vector<
                             if (linear && tby > 1) break;
                             if (!linear && tbx != tbx_full && tbx != 1 && tbx * 2 != tbx_full) continue;
                             if (!linear && (tby - 1) * RB >= g.h_out) break;
+                            if (rpw * tbx * tby > 32) continue;            // accumulator registers per lane
+                            if (nw * rpw > std::max(8, round_up(g.c_out, 8))) continue;   // more filter slots than filters
                             Schedule s;
                             s.kind = linear ? KK_SCONV_LINEAR : KK_SCONV_SPATIAL;
                             s.NW = nw; s.RPW = rpw; s.CIc = cic; s.ksplit = ks;
@@ -298,7 +300,7 @@ void apply_env_override(const Geometry &g, bool linear, Schedule &best)
     int v;
     const char *q;
     if ((q = strstr(env, "nw=")) && sscanf(q + 3, "%d", &v) == 1 && (v == 4 || v == 8 || v == 16)) s.NW = v;
-    if ((q = strstr(env, "rpw=")) && sscanf(q + 4, "%d", &v) == 1 && (v == 1 || v == 2 || v == 4)) s.RPW = v;
+    if ((q = strstr(env, "rpw=")) && sscanf(q + 4, "%d", &v) == 1 && (v == 1 || v == 2 || v == 4 || v == 8 || v == 16)) s.RPW = v;
     if ((q = strstr(env, "tbx=")) && sscanf(q + 4, "%d", &v) == 1 && v >= 1 && v <= 8) s.TBX = v;
     if ((q = strstr(env, "tby=")) && sscanf(q + 4, "%d", &v) == 1 && v >= 1 && v <= 8) s.TBY = v;
     if ((q = strstr(env, "cic=")) && sscanf(q + 4, "%d", &v) == 1 && v >= 1 && v <= 512 && (!g.s8 || v % 4 == 0))
@@ -463,7 +465,7 @@ cadnn_status autotune_sconv(cadnn_weights *h, const Src &src, const Geometry &g,
         seen.push_back(key);
         pick.push_back(c);
     }
-    const size_t kMaxTimed = 56;
+    const size_t kMaxTimed = 80;
     if (pick.size() > kMaxTimed) pick.resize(kMaxTimed);
     const size_t esz = src.s8 ? 1 : 4;
     const size_t xb = (size_t)batch * d.in_h * d.in_w * d.c_in * esz;
@@ -583,11 +585,13 @@ cadnn_status pack_dense(cadnn_weights *h, const Src &src, int kind)
     const int taps = d.kh * d.kw * cg;
     // tap-major: [kh][kw][cg][c_out], so that lanes over output channels read contiguously
     h->dense_f.assign((size_t)taps * d.c_out, 0.0f);
+    h->dense_kept.assign((size_t)taps * d.c_out, 0);
     for (int co = 0; co < d.c_out; ++co)
         for (int t = 0; t < taps; ++t) {
             size_t wi = (size_t)co * taps + t;
             if (src.kept(wi)) {
                 h->dense_f[(size_t)t * d.c_out + co] = src.fval(wi);
+                h->dense_kept[wi] = 1;
                 h->nnz++;
             }
         }
@@ -621,7 +625,16 @@ cadnn_status pack_common(const cadnn_layer_desc *desc, const Src &src, cadnn_wei
     cadnn_status st;
     try {
         const bool is_fc = d.kh == 1 && d.kw == 1 && d.in_h == 1 && d.in_w == 1 && d.pad == 0;
+        // a float layer with <= 4 input channels whose mask keeps (nearly) everything is a dense stem
+        bool dense_stem = false;
+        if (!depthwise && d.dtype == CADNN_F32 && d.c_in <= 4 && (d.kh > 1 || d.kw > 1) &&
+            (size_t)d.kh * d.kw * d.c_in * 64 * 4 <= 160 * 1024) {
+            size_t numel = (size_t)d.c_out * d.kh * d.kw * d.c_in, kept = 0;
+            for (size_t i = 0; i < numel; ++i) kept += src.kept(i);
+            dense_stem = kept * 2 >= numel;
+        }
         if (depthwise) st = pack_dense(h, src, KK_DW);
+        else if (dense_stem) st = pack_dense(h, src, KK_DENSE_SMALLC);
         else if (is_fc && std::max(1, d.batch_hint) <= 8 && d.c_in <= 65536) st = pack_fc_spmv(h, src);
         else st = pack_sconv(h, src);
         if (st == CADNN_OK) st = upload(h);
@@ -721,7 +734,7 @@ cadnn_status cadnn_weights_unpack(const cadnn_weights *w, float *dense, uint8_t 
         for (int co = 0; co < d.c_out; ++co)
             for (size_t t = 0; t < K; ++t) {
                 if (dense) dense[co * K + t] = w->dense_f[t * d.c_out + co];
-                if (mask) mask[co * K + t] = 1;
+                if (mask) mask[co * K + t] = w->dense_kept[co * K + t];
             }
         return CADNN_OK;
     }

@@ -1,6 +1,7 @@
 // Glue layers of the evaluated networks: max pooling (float and int8) and global
 // average pooling.  The paper (arXiv 1905.00571) does not discuss them; they are
 // bound by one read and one write of the feature map, so lanes map to channels.
+#include <algorithm>
 #include <cfloat>
 #include "cadnn_internal.h"
 
@@ -38,6 +39,49 @@ __global__ void __launch_bounds__(256) maxpool_kernel(const XT *x, XT *y, int n,
     }
 }
 
+// 16 bytes per thread: four floats, or sixteen int8 channels (per-byte signed max).
+template <bool S8>
+__global__ void __launch_bounds__(256) maxpool_vec_kernel(const uint4 *x, uint4 *y, int n, int h, int w, int cv,
+                                                          int h_out, int w_out, int k, int stride, int pad)
+{
+    const long long total = (long long)n * h_out * w_out * cv;
+    grid_dep_wait();
+    grid_dep_trigger();
+    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int ch = (int)(idx % cv);
+        long long pix = idx / cv;
+        const int ox = (int)(pix % w_out);
+        long long r = pix / w_out;
+        const int oy = (int)(r % h_out);
+        const int b = (int)(r / h_out);
+        bool any = false;
+        uint4 best = make_uint4(0, 0, 0, 0);
+        for (int ky = 0; ky < k; ++ky) {
+            const int iy = oy * stride + ky - pad;
+            if (iy < 0 || iy >= h) continue;
+            for (int kx = 0; kx < k; ++kx) {
+                const int ix = ox * stride + kx - pad;
+                if (ix < 0 || ix >= w) continue;
+                const uint4 v = x[(((size_t)b * h + iy) * w + ix) * cv + ch];
+                if (!any) {
+                    best = v;
+                    any = true;
+                } else if (S8) {
+                    best.x = __vmaxs4(best.x, v.x); best.y = __vmaxs4(best.y, v.y);
+                    best.z = __vmaxs4(best.z, v.z); best.w = __vmaxs4(best.w, v.w);
+                } else {
+                    best.x = __float_as_uint(fmaxf(__uint_as_float(best.x), __uint_as_float(v.x)));
+                    best.y = __float_as_uint(fmaxf(__uint_as_float(best.y), __uint_as_float(v.y)));
+                    best.z = __float_as_uint(fmaxf(__uint_as_float(best.z), __uint_as_float(v.z)));
+                    best.w = __float_as_uint(fmaxf(__uint_as_float(best.w), __uint_as_float(v.w)));
+                }
+            }
+        }
+        y[idx] = best;
+    }
+}
+
 __global__ void __launch_bounds__(256) gavgpool_kernel(const float *x, float *y, int n, int hw, int c, float inv)
 {
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
@@ -59,6 +103,16 @@ cadnn_status launch_maxpool(const void *x, int n, int h, int wd, int c, int k, i
     const int h_out = (h + 2 * pad - k) / stride + 1, w_out = (wd + 2 * pad - k) / stride + 1;
     long long total = (long long)n * h_out * w_out * c;
     if (total <= 0) return CADNN_OK;
+    const int per = dtype == CADNN_S8 ? 16 : 4;   // channels per 16-byte vector
+    if (c % per == 0 && ((uintptr_t)x & 15) == 0 && ((uintptr_t)y & 15) == 0) {
+        long long tv = total / per;
+        long long bv = std::min((tv + 255) / 256, 148LL * 32);
+        if (dtype == CADNN_S8)
+            return launch_kernel(maxpool_vec_kernel<true>, (int)bv, 256, 0, pdl, st, (const uint4 *)x, (uint4 *)y, n, h, wd,
+                                 c / per, h_out, w_out, k, stride, pad);
+        return launch_kernel(maxpool_vec_kernel<false>, (int)bv, 256, 0, pdl, st, (const uint4 *)x, (uint4 *)y, n, h, wd,
+                             c / per, h_out, w_out, k, stride, pad);
+    }
     long long blocks = (total + 255) / 256;
     if (blocks > 148LL * 64) blocks = 148LL * 64;
     if (dtype == CADNN_S8)

@@ -564,6 +564,9 @@ cadnn_status launch_rpw(const SconvParams &p, int rpw, int blocks, int threads, 
         case 1: return launch_one<XT, T, 1>(p, blocks, threads, smem, pdl, st);
         case 2: return launch_one<XT, T, 2>(p, blocks, threads, smem, pdl, st);
         case 4: return launch_one<XT, T, 4>(p, blocks, threads, smem, pdl, st);
+        // many filters per warp only with few pixel bands per lane (accumulators = RPW * T registers)
+        case 8: if (T <= 4) return launch_one<XT, (T <= 4 ? T : 1), 8>(p, blocks, threads, smem, pdl, st); break;
+        case 16: if (T <= 2) return launch_one<XT, (T <= 2 ? T : 1), 16>(p, blocks, threads, smem, pdl, st); break;
     }
     return CADNN_E_UNSUPPORTED;
 }
