@@ -1,0 +1,146 @@
+"""Measurement report: whole-network and per-layer times of the synthetic pruned networks, the
+fraction of the sparse roofline they reach, and the same layers run dense.
+
+    python -m paper_1905_00571_b200.report --workload resnet50 --batch 1 8 --density 0.125 1.0 [--layers]
+
+Everything timed here runs through the C ABI (argument marshalling only in Python).  The dense
+comparison is (i) this library at density 1.0 and (ii), as labelled context, torch's cuDNN
+convolutions on the same shapes (fp32 with TF32 off, and TF32 on) - library calls only.
+Prints markdown.
+"""
+import argparse
+import sys
+
+import numpy as np
+import torch
+
+from workloads import models
+from . import binding as B
+from . import roofline
+from .network import PackedModel
+
+
+def build(workload, density):
+    if workload == "resnet50":
+        fc = 0.10 if density < 1.0 else 1.0
+        return models.resnet50(density=density, fc_density=fc)
+    if workload == "mobilenet_v2":
+        return models.mobilenet_v2(density=density)
+    if workload == "vgg16":
+        return models.vgg16(density=density, fc_density=min(1.0, density / 2))
+    raise SystemExit("unknown workload " + workload)
+
+
+def time_forward(pm, x, y, reps=50):
+    pm.forward(x, y)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        pm.forward(x, y)
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps
+
+
+def torch_dense_ms(model, batch, tf32, reps=20):
+    """cuDNN convolutions / matmuls on the same layer shapes (dense weights), layer by layer."""
+    if model.dtype != "f32":
+        return None
+    torch.backends.cudnn.allow_tf32 = tf32
+    torch.backends.cuda.matmul.allow_tf32 = tf32
+    layers = []
+    for op in model.ops:
+        if op.kind == "conv":
+            w = torch.randn(op.c_out, op.c_in // op.groups, op.k, op.k, device="cuda").contiguous(memory_format=torch.channels_last)
+            xin = torch.randn(batch, op.c_in, op.in_hw[0], op.in_hw[1], device="cuda").contiguous(memory_format=torch.channels_last)
+            layers.append((lambda xin=xin, w=w, op=op: torch.nn.functional.conv2d(xin, w, None, op.stride, op.pad, 1, op.groups)))
+        elif op.kind == "fc":
+            w = torch.randn(op.c_out, op.c_in, device="cuda")
+            xin = torch.randn(batch, op.c_in, device="cuda")
+            layers.append((lambda xin=xin, w=w: xin @ w.t()))
+    for f in layers:
+        f()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for f in layers:
+            f()
+    g.replay()
+    torch.cuda.synchronize()
+    a.record()
+    for _ in range(reps):
+        g.replay()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="resnet50")
+    ap.add_argument("--batch", type=int, nargs="+", default=[1])
+    ap.add_argument("--density", type=float, nargs="+", default=[0.125])
+    ap.add_argument("--layers", action="store_true", help="also print the per-layer table")
+    ap.add_argument("--no-autotune", action="store_true")
+    ap.add_argument("--torch-dense", action="store_true", help="add cuDNN dense timings (context)")
+    args = ap.parse_args()
+    peaks = roofline.measured_peaks()
+    r_alu = roofline.alu_peak_tflops(peaks["sm_max_mhz"])
+    print("# %s: sparse-roofline report (ALU peak %.1f TFLOP/s, HBM %.0f GB/s nominal / %.0f measured)\n"
+          % (args.workload, r_alu, roofline.HBM_NOMINAL_GBS, peaks["hbm_gbs"]))
+    print("| batch | density | latency ms | images/s | roofline µs | fraction | k×k frac | 1×1 frac | nnz stored |")
+    print("|---|---|---|---|---|---|---|---|---|")
+    layer_tables = []
+    for dens in args.density:
+        model = build(args.workload, dens)
+        for batch in args.batch:
+            pm = PackedModel(model, batch, "cuda:0", autotune=not args.no_autotune)
+            x = torch.from_numpy(models.make_input(model, batch)).cuda()
+            y = pm.new_output()
+            ms = time_forward(pm, x, y)
+            rows = roofline.network_roofline(model, batch, r_alu, roofline.HBM_NOMINAL_GBS)
+            per = np.zeros(len(model.ops))
+            for _ in range(2):
+                per += np.array(pm.layer_times(x, y, reps=10)) / 2
+            t_roof = sum(r["t_roof_us"] for r in rows)
+            fam = {}
+            for r, t in zip(rows, per):
+                f = fam.setdefault(r["family"], [0.0, 0.0])
+                f[0] += r["t_roof_us"]
+                f[1] += t * 1e3
+            frac = lambda k: ("%.3f" % (fam[k][0] / fam[k][1])) if k in fam and fam[k][1] > 0 else "-"
+            print("| %d | %.3g | %.4f | %.0f | %.1f | %.4f | %s | %s | %d |" % (
+                batch, dens, ms, batch / ms * 1e3, t_roof, t_roof / (ms * 1e3), frac("sconv_kxk"), frac("sconv_1x1"),
+                sum(o.nnz for o in model.weight_ops())))
+            sys.stdout.flush()
+            if args.layers:
+                lines = ["\n## per layer: batch %d, density %.3g\n" % (batch, dens),
+                         "| layer | kernel | in | c_in→c_out | k/s | nnz | µs | roofline µs | fraction | schedule |", "|---|---|---|---|---|---|---|---|---|---|"]
+                for i, (op, r, t) in enumerate(zip(model.ops, rows, per)):
+                    s = B.cadnn_weights_schedule(pm.weights[i]) if i in pm.weights else None
+                    ss = ("T%d rpw%d nw%d cic%d ks%d" % (s["T"], s["RPW"], s["NW"], s["CIc"], s["ksplit"])) if s and s["kind"] in (1, 2) else ""
+                    lines.append("| %s | %s | %dx%d | %d→%d | %d/%d | %d | %.1f | %.2f | %.3f | %s |" % (
+                        op.name, r["family"], op.in_hw[0], op.in_hw[1], op.c_in, op.c_out, op.k, op.stride, r["nnz"],
+                        t * 1e3, r["t_roof_us"], r["t_roof_us"] / (t * 1e3), ss))
+                layer_tables.append("\n".join(lines))
+            del pm
+            torch.cuda.empty_cache()
+    for t in layer_tables:
+        print(t)
+    if args.torch_dense:
+        print("\n## dense context: torch / cuDNN on the same layer shapes (library calls, channels-last)\n")
+        print("| batch | fp32 (TF32 off) ms | TF32 on ms |")
+        print("|---|---|---|")
+        model = build(args.workload, 1.0) if args.workload != "vgg16" else None
+        for batch in args.batch:
+            if model is None:
+                break
+            a = torch_dense_ms(model, batch, False)
+            b = torch_dense_ms(model, batch, True)
+            print("| %d | %.4f | %.4f |" % (batch, a, b))
+
+
+if __name__ == "__main__":
+    main()
