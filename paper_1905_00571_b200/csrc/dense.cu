@@ -18,6 +18,7 @@ struct DwParams {
     const float *bias;
     const float *residual;
     int n, h, w, c, h_out, w_out, kh, kw, stride, pad, act;
+    FastDiv d_cv, d_wout, d_hout;
 };
 
 __device__ __forceinline__ float dw_act(float z, int act)
@@ -34,14 +35,14 @@ __global__ void __launch_bounds__(256) dw_kernel(const DwParams p)
     const long long total = (long long)p.n * p.h_out * p.w_out * cv;
     grid_dep_wait();
     grid_dep_trigger();
-    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
-         idx += (long long)gridDim.x * blockDim.x) {
-        const int c0 = (int)(idx % cv) * VEC;
-        long long pix = idx / cv;
-        const int ox = (int)(pix % p.w_out);
-        long long r = pix / p.w_out;
-        const int oy = (int)(r % p.h_out);
-        const int b = (int)(r / p.h_out);
+    // the host refuses tensors with 2^31 or more vectors, so 32-bit index arithmetic is exact
+    for (unsigned idx = blockIdx.x * blockDim.x + threadIdx.x; idx < (unsigned)total; idx += gridDim.x * blockDim.x) {
+        const unsigned pix = fdiv(idx, p.d_cv);
+        const int c0 = (int)(idx - pix * cv) * VEC;
+        const unsigned r = fdiv(pix, p.d_wout);
+        const int ox = (int)(pix - r * p.w_out);
+        const unsigned b = fdiv(r, p.d_hout);
+        const int oy = (int)(r - b * p.h_out);
         float acc[VEC];
 #pragma unroll
         for (int v = 0; v < VEC; ++v) acc[v] = 0.0f;
@@ -194,6 +195,10 @@ cadnn_status launch_dw(const cadnn_weights *w, const void *x, int n, void *y, co
     const bool v4 = d.c_out % 4 == 0;
     long long total = (long long)n * w->h_out * w->w_out * (v4 ? d.c_out / 4 : d.c_out);
     if (total <= 0) return CADNN_OK;
+    if (total >= (1LL << 31)) return CADNN_E_UNSUPPORTED;
+    p.d_cv = make_fastdiv(v4 ? d.c_out / 4 : d.c_out);
+    p.d_wout = make_fastdiv(w->w_out);
+    p.d_hout = make_fastdiv(w->h_out);
     long long blocks = (total + 255) / 256;
     if (blocks > 148LL * 64) blocks = 148LL * 64;
     if (v4) return launch_kernel(dw_kernel<4>, (int)blocks, 256, 0, ep.pdl, st, p);

@@ -42,19 +42,19 @@ __global__ void __launch_bounds__(256) maxpool_kernel(const XT *x, XT *y, int n,
 // 16 bytes per thread: four floats, or sixteen int8 channels (per-byte signed max).
 template <bool S8>
 __global__ void __launch_bounds__(256) maxpool_vec_kernel(const uint4 *x, uint4 *y, int n, int h, int w, int cv,
-                                                          int h_out, int w_out, int k, int stride, int pad)
+                                                          int h_out, int w_out, int k, int stride, int pad,
+                                                          FastDiv d_cv, FastDiv d_wout, FastDiv d_hout)
 {
-    const long long total = (long long)n * h_out * w_out * cv;
+    const unsigned total = (unsigned)n * h_out * w_out * cv;   // < 2^31, checked by the host
     grid_dep_wait();
     grid_dep_trigger();
-    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
-         idx += (long long)gridDim.x * blockDim.x) {
-        const int ch = (int)(idx % cv);
-        long long pix = idx / cv;
-        const int ox = (int)(pix % w_out);
-        long long r = pix / w_out;
-        const int oy = (int)(r % h_out);
-        const int b = (int)(r / h_out);
+    for (unsigned idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        const unsigned pix = fdiv(idx, d_cv);
+        const int ch = (int)(idx - pix * cv);
+        const unsigned r = fdiv(pix, d_wout);
+        const int ox = (int)(pix - r * w_out);
+        const unsigned b = fdiv(r, d_hout);
+        const int oy = (int)(r - b * h_out);
         bool any = false;
         uint4 best = make_uint4(0, 0, 0, 0);
         for (int ky = 0; ky < k; ++ky) {
@@ -104,14 +104,15 @@ cadnn_status launch_maxpool(const void *x, int n, int h, int wd, int c, int k, i
     long long total = (long long)n * h_out * w_out * c;
     if (total <= 0) return CADNN_OK;
     const int per = dtype == CADNN_S8 ? 16 : 4;   // channels per 16-byte vector
-    if (c % per == 0 && ((uintptr_t)x & 15) == 0 && ((uintptr_t)y & 15) == 0) {
+    if (c % per == 0 && ((uintptr_t)x & 15) == 0 && ((uintptr_t)y & 15) == 0 && total / per < (1LL << 31)) {
+        const FastDiv d_cv = make_fastdiv(c / per), d_wout = make_fastdiv(w_out), d_hout = make_fastdiv(h_out);
         long long tv = total / per;
         long long bv = std::min((tv + 255) / 256, 148LL * 32);
         if (dtype == CADNN_S8)
             return launch_kernel(maxpool_vec_kernel<true>, (int)bv, 256, 0, pdl, st, (const uint4 *)x, (uint4 *)y, n, h, wd,
-                                 c / per, h_out, w_out, k, stride, pad);
+                                 c / per, h_out, w_out, k, stride, pad, d_cv, d_wout, d_hout);
         return launch_kernel(maxpool_vec_kernel<false>, (int)bv, 256, 0, pdl, st, (const uint4 *)x, (uint4 *)y, n, h, wd,
-                             c / per, h_out, w_out, k, stride, pad);
+                             c / per, h_out, w_out, k, stride, pad, d_cv, d_wout, d_hout);
     }
     long long blocks = (total + 255) / 256;
     if (blocks > 148LL * 64) blocks = 148LL * 64;

@@ -28,32 +28,6 @@ namespace cg = cooperative_groups;
 
 namespace {
 
-// Division by a runtime constant as multiply-high and shift (the divisor is fixed per
-// launch; a hardware integer division costs a few dozen dependent instructions).
-// q = umulhi(n, mul) >> shr is exact for 0 <= n < 2^31 when mul = ceil(2^(32 + shr) / d)
-// and 2^shr >= d (shr chosen so that mul fits 32 bits); d == 1 is passed through.
-struct FastDiv {
-    unsigned mul, shr, d;
-};
-FastDiv make_fastdiv(int d)
-{
-    FastDiv f;
-    f.d = (unsigned)d;
-    f.mul = 0;
-    f.shr = 0;
-    if (d <= 1) return f;
-    unsigned l = 0;
-    while ((1u << l) < (unsigned)d) ++l;              // ceil(log2 d)
-    unsigned long long p2 = 1ull << (31 + l);
-    f.mul = (unsigned)((p2 + d - 1) / (unsigned long long)d);
-    f.shr = l - 1;
-    return f;
-}
-__device__ __forceinline__ unsigned fdiv(unsigned n, const FastDiv &f)
-{
-    return f.d == 1 ? n : (__umulhi(n, f.mul) >> f.shr);
-}
-
 struct SconvParams {
     const void *x;
     void *y;
