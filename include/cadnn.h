@@ -171,6 +171,20 @@ cadnn_status cadnn_conv2d(const cadnn_weights *w, const void *x, int n, int h, i
                           const cadnn_epilogue *ep, void *stream);
 
 /*
+ * cadnn_conv2d_planar - the same layer on channel-planar activations (Section 4, "Memory
+ * layout transformation": data laid out to fit the processor).  This is the layout
+ * cadnn_forward uses between the layers of a float network; the call exists so that it can
+ * be checked on its own.
+ *   x device float [n][c_in][in_h + 2][in_w + 2], y device float [n][c_out][h_out + 2][w_out + 2]:
+ *   every plane carries a one-pixel border that MUST be zero in x and that the call never
+ *   writes in y (so a y buffer zeroed once stays a valid input for the next layer).
+ *   residual (optional) has y's layout.  Float layers with pad <= 1 and k - 1 - pad <= 1 only:
+ *   E_UNSUPPORTED otherwise.  Same epilogue, same errors as cadnn_conv2d.
+ */
+cadnn_status cadnn_conv2d_planar(const cadnn_weights *w, const void *x, int n, void *y, const cadnn_epilogue *ep,
+                                 void *stream);
+
+/*
  * cadnn_fc - one sparse fully connected layer: y[b][co] = sum_k W[co][k] x[b][k],
  * same epilogue.  x device [n][k], y device [n][c_out].
  */
@@ -212,6 +226,10 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
  * cadnn_forward - run the network: x device input, y device output of the last op.
  * use_graph != 0 replays a CUDA graph captured on the first call with this (x, y)
  * pair (re-captured when either pointer changes); 0 launches the layers one by one.
+ * Float networks made of a dense stem, sparse convs, max pools, a global average pool and fc
+ * layers keep their intermediate feature maps channel-planar with a zero halo (see
+ * cadnn_conv2d_planar); others (depthwise, int8) keep NHWC.  CADNN_NO_PLANAR in the
+ * environment at cadnn_net_create forces NHWC.
  * Without a graph, layers after the first are launched as programmatic dependents of
  * their predecessor (their weight fetch overlaps its stores); set CADNN_NO_PDL in the
  * environment before cadnn_net_create to use plain stream order instead.

@@ -56,6 +56,7 @@ _SIGS = {
     "cadnn_weights_unpack": (_i, [_vp, _vp, _vp]),
     "cadnn_weights_free": (None, [_vp]),
     "cadnn_conv2d": (_i, [_vp, _vp, _i, _i, _i, _vp, ctypes.POINTER(Epilogue), _vp]),
+    "cadnn_conv2d_planar": (_i, [_vp, _vp, _i, _vp, ctypes.POINTER(Epilogue), _vp]),
     "cadnn_fc": (_i, [_vp, _vp, _i, _vp, ctypes.POINTER(Epilogue), _vp]),
     "cadnn_maxpool2d": (_i, [_vp, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _vp]),
     "cadnn_global_avgpool": (_i, [_vp, _i, _i, _i, _i, _vp, _vp]),
@@ -202,6 +203,14 @@ def cadnn_conv2d(w, x, y, scale=None, bias=None, residual=None, act="none", out_
     ep = _epilogue(scale, bias, residual, act, out_dtype)
     _check(_lib.cadnn_conv2d(w.handle, _dev_ptr(x), n, h, wd, _dev_ptr(y), ctypes.byref(ep), _stream(stream)),
            "cadnn_conv2d")
+    return y
+
+
+def cadnn_conv2d_planar(w, x, y, scale=None, bias=None, residual=None, act="none", stream=None):
+    """x [n, c_in, h+2, w+2], y [n, c_out, ho+2, wo+2]: float CUDA tensors with a zero one-pixel border."""
+    ep = _epilogue(scale, bias, residual, act, F32)
+    _check(_lib.cadnn_conv2d_planar(w.handle, _dev_ptr(x), int(x.shape[0]), _dev_ptr(y), ctypes.byref(ep), _stream(stream)),
+           "cadnn_conv2d_planar")
     return y
 
 

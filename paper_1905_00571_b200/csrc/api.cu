@@ -73,6 +73,18 @@ cadnn_status cadnn_conv2d(const cadnn_weights *w, const void *x, int n, int h, i
     return conv2d_impl(w, x, n, h, wd, y, ep, false, (cudaStream_t)stream);
 }
 
+cadnn_status cadnn_conv2d_planar(const cadnn_weights *w, const void *x, int n, void *y, const cadnn_epilogue *ep,
+                                 void *stream)
+{
+    if (!w || !x || !y || n < 0) return CADNN_E_ARG;
+    if (!w->on_device || !w->has_planar) return CADNN_E_UNSUPPORTED;
+    if (!aligned16(x) || !aligned16(y) || x == y) return CADNN_E_ARG;
+    LaunchEpilogue le;
+    cadnn_status st = check_epilogue(w, ep, le);
+    if (st != CADNN_OK) return st;
+    return launch_sconv_planar(w, x, n, y, le, (cudaStream_t)stream);
+}
+
 cadnn_status cadnn_fc(const cadnn_weights *w, const void *x, int n, void *y, const cadnn_epilogue *ep, void *stream)
 {
     if (!w) return CADNN_E_ARG;

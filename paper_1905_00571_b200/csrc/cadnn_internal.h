@@ -13,6 +13,7 @@ enum KernelKind {
     KK_DENSE_SMALLC = 5    // dense conv with <= 4 input channels
 };
 
+static const int kPlanarHalo = 1;     // zero border of the channel-planar activation layout
 static const int kWarpsPerBlock = 8;  // fc kernel; the conv kernels take it from the schedule
 
 // Per-layer schedule chosen by the packer (Section 4, "Optimization parameters selection").
@@ -62,6 +63,18 @@ struct cadnn_weights {
     std::vector<uint8_t> dense_kept; // dense kinds: which positions the mask kept (host only, for unpack)
     int c_pad = 0;
 
+    // channel-planar variant of a float conv layer (see planar.cu): CSR by output channel,
+    // entries {value bits, element offset into the padded planar input}, rows padded to even counts
+    bool has_planar = false;
+    std::vector<uint32_t> pl_ent;
+    std::vector<int32_t> pl_ptr;     // [c_out + 1], in entries
+    std::vector<int32_t> pl_order;   // warp slot -> output channel (filters dealt to warps by load)
+    std::vector<int64_t> row_nnz;    // stored nonzeros per output channel
+    int pl_T = 2, pl_NW = 8, pl_RPW = 1, pl_KSW = 1;   // bands per lane, warps per block, filters per warp slot, warps per filter
+    const uint32_t *d_pl_ent = nullptr;
+    const int32_t *d_pl_ptr = nullptr;
+    const int32_t *d_pl_order = nullptr;
+
     // device image (one allocation)
     void *d_blob = nullptr;
     const uint32_t *d_ent = nullptr;
@@ -79,6 +92,7 @@ struct LaunchEpilogue {
     int act = 0;
     int out_dtype = 0;
     bool pdl = false;   // launch as a programmatic dependent of the previous kernel (inside cadnn_forward)
+    bool planar_out = false;   // dense stem: write the channel-planar layout instead of NHWC
 };
 
 // status helpers
@@ -98,6 +112,11 @@ cadnn_status launch_dw(const cadnn_weights *w, const void *x, int n, void *y, co
                        cudaStream_t st);
 cadnn_status launch_dense_smallc(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
                                  cudaStream_t st);
+cadnn_status launch_sconv_planar(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
+                                 cudaStream_t st);
+cadnn_status launch_maxpool_planar(const float *x, int n, int h, int wd, int c, int k, int stride, int pad, float *y,
+                                   bool pdl, cudaStream_t st);
+cadnn_status launch_gavgpool_planar(const float *x, int n, int h, int wd, int c, float *y, bool pdl, cudaStream_t st);
 cadnn_status launch_maxpool(const void *x, int n, int h, int wd, int c, int k, int stride, int pad, int dtype,
                             void *y, bool pdl, cudaStream_t st);
 cadnn_status launch_gavgpool(const float *x, int n, int h, int wd, int c, float *y, bool pdl, cudaStream_t st);

@@ -93,6 +93,7 @@ struct StemParams {
     const float *residual;
     int n, h, w, c_in, c_out, h_out, w_out, kh, kw, stride, pad, act;
     int tiles_x, tiles_y, in_rows, in_cols, taps, co_blocks;
+    int planar_out, halo;   // write [n][c][h_out + 2 halo][w_out + 2 halo] instead of NHWC
 };
 
 const int kStemCo = 16;      // output channels per warp
@@ -169,13 +170,20 @@ __global__ void __launch_bounds__(256) stem_kernel(const StemParams p)
             if (oy >= p.h_out) continue;
             const float *acc = rr ? acc1 : acc0;
             const size_t o = (((size_t)img * p.h_out + oy) * p.w_out + ox) * p.c_out + cbase;
+            const int wp = p.w_out + 2 * p.halo;
+            const size_t plane = (size_t)(p.h_out + 2 * p.halo) * wp;
+            const size_t opl = (size_t)img * p.c_out * plane + (size_t)(oy + p.halo) * wp + ox + p.halo;
 #pragma unroll
             for (int c = 0; c < kStemCo; ++c) {
                 const int co = cbase + c;
                 if (co >= p.c_out) break;
                 float z = fmaf(acc[c], p.scale ? p.scale[co] : 1.0f, p.bias ? p.bias[co] : 0.0f);
-                if (p.residual) z += p.residual[o + c];
-                p.y[o + c] = dw_act(z, p.act);
+                if (p.planar_out) {
+                    p.y[opl + (size_t)co * plane] = dw_act(z, p.act);   // lanes are consecutive columns: contiguous
+                } else {
+                    if (p.residual) z += p.residual[o + c];
+                    p.y[o + c] = dw_act(z, p.act);
+                }
             }
         }
     }
@@ -215,6 +223,9 @@ cadnn_status launch_dense_smallc(const cadnn_weights *w, const void *x, int n, v
     p.n = n; p.h = d.in_h; p.w = d.in_w; p.c_in = d.c_in; p.c_out = d.c_out;
     p.h_out = w->h_out; p.w_out = w->w_out; p.kh = d.kh; p.kw = d.kw; p.stride = d.stride; p.pad = d.pad;
     p.act = ep.act;
+    p.planar_out = ep.planar_out ? 1 : 0;
+    p.halo = kPlanarHalo;
+    if (ep.planar_out && ep.residual) return CADNN_E_UNSUPPORTED;
     p.tiles_x = (w->w_out + 31) / 32;
     p.tiles_y = (w->h_out + kStemRows - 1) / kStemRows;
     p.in_rows = (kStemRows - 1) * d.stride + d.kh;

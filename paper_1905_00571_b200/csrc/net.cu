@@ -21,6 +21,7 @@ struct cadnn_net {
     std::vector<SlotInfo> slots;
     int out_slot = -1;
     bool use_pdl = true;   // layers after the first launch as programmatic dependents
+    bool planar = false;   // intermediate feature maps are channel-planar with a zero halo (planar.cu)
     int64_t workspace = 0;
     // graph cache: [0] caller's device pointers, [1] the net's own staging buffers
     struct GraphCache {
@@ -51,6 +52,26 @@ cadnn_status run_op(cadnn_net *net, const cadnn_op &op, const void *x, void *y, 
     const SlotInfo &si = net->slots[op.src];
     const void *src = slot_ptr(net, op.src, x, y);
     void *dst = slot_ptr(net, op.dst, x, y);
+    if (net->planar && op.kind != CADNN_OP_FC) {
+        if (op.kind == CADNN_OP_CONV) {
+            LaunchEpilogue le;
+            le.scale = op.scale;
+            le.bias = op.bias;
+            le.residual = op.res >= 0 ? slot_ptr(net, op.res, x, y) : nullptr;
+            le.act = op.act;
+            le.out_dtype = CADNN_F32;
+            le.pdl = pdl;
+            if (op.w->s.kind == KK_DENSE_SMALLC) {   // the stem reads the NHWC image and writes planes
+                le.planar_out = true;
+                return launch_dense_smallc(op.w, src, si.n, dst, le, st);
+            }
+            return launch_sconv_planar(op.w, src, si.n, dst, le, st);
+        }
+        if (op.kind == CADNN_OP_MAXPOOL)
+            return launch_maxpool_planar((const float *)src, si.n, si.h, si.w, si.c, op.pool_k, op.pool_stride,
+                                         op.pool_pad, (float *)dst, pdl, st);
+        return launch_gavgpool_planar((const float *)src, si.n, si.h, si.w, si.c, (float *)dst, pdl, st);
+    }
     if (op.kind == CADNN_OP_CONV || op.kind == CADNN_OP_FC) {
         cadnn_epilogue ep;
         ep.scale = op.scale;
@@ -155,6 +176,29 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
         in.n = n; in.h = h; in.w = wd; in.c = c; in.dtype = in_dtype; in.defined = true;
         net->out_slot = ops[n_ops - 1].dst;
         net->in_bytes = (int64_t)n * h * wd * c * dtype_size(in_dtype);
+        // Channel-planar intermediates are used when every op has a planar kernel: a dense stem on
+        // the NHWC input, then sparse float convs, max pools, a global average pool, and fc layers
+        // fed by it.  (Depthwise and int8 layers keep NHWC.)
+        bool planar = in_dtype == CADNN_F32 && getenv("CADNN_NO_PLANAR") == nullptr && n_ops >= 2 &&
+                      ops[n_ops - 1].kind == CADNN_OP_FC;
+        std::vector<char> flat(max_slot + 1, 0);   // slot holds a dense [n][c] vector
+        for (int i = 0; i < n_ops && planar; ++i) {
+            const cadnn_op &op = ops[i];
+            if (op.kind == CADNN_OP_CONV) {
+                if (!op.w) { planar = false; break; }
+                const bool stem = op.w->s.kind == KK_DENSE_SMALLC && op.src == 0 && op.res < 0;
+                if (!stem && (!op.w->has_planar || op.src == 0 || flat[op.src])) planar = false;
+            } else if (op.kind == CADNN_OP_FC) {
+                if (!flat[op.src]) planar = false;
+                flat[op.dst] = 1;
+            } else if (op.kind == CADNN_OP_GAVGPOOL) {
+                if (op.src == 0 || flat[op.src]) planar = false;
+                flat[op.dst] = 1;
+            } else if (op.kind == CADNN_OP_MAXPOOL) {
+                if (op.src == 0 || flat[op.src]) planar = false;
+            }
+        }
+        net->planar = planar;
     }
     for (int i = 0; i < n_ops && st == CADNN_OK; ++i) {
         const cadnn_op &op = ops[i];
@@ -189,9 +233,13 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
         } else { st = CADNN_E_ARG; break; }
         so.defined = true;
         so.bytes = (int64_t)so.n * so.h * so.w * so.c * dtype_size(so.dtype);
+        const bool padded = net->planar && (op.kind == CADNN_OP_CONV || op.kind == CADNN_OP_MAXPOOL);
+        if (padded) so.bytes = (int64_t)so.n * so.c * (so.h + 2 * kPlanarHalo) * (so.w + 2 * kPlanarHalo) * 4;
         if (op.dst != net->out_slot) {
             size_t alloc = (size_t)((so.bytes + 255) / 256 * 256);
             cudaError_t e = cudaMalloc(&so.ptr, alloc ? alloc : 256);
+            // the halo of a planar tensor must read as zero and is never written afterwards
+            if (e == cudaSuccess && padded) e = cudaMemset(so.ptr, 0, alloc);
             if (e != cudaSuccess) {
                 cadnn_note_cuda(e);
                 st = e == cudaErrorMemoryAllocation ? CADNN_E_ALLOC : CADNN_E_CUDA;

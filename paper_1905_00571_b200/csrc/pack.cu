@@ -173,8 +173,10 @@ cadnn_status upload(cadnn_weights *h)
     size_t b_vals = h->desc.dtype == CADNN_S8 ? h->vals_q.size() : h->vals_f.size() * 4;
     size_t b_offs = h->offs.size() * 2, b_ptr = h->ptr.size() * 4, b_perm = h->perm.size() * 4;
     size_t b_dense = h->dense_f.size() * 4, b_ent = h->ent.size() * 4;
+    size_t b_ple = h->pl_ent.size() * 4, b_plp = h->pl_ptr.size() * 4, b_plo = h->pl_order.size() * 4;
     size_t o_vals = 0, o_offs = o_vals + al(b_vals), o_ptr = o_offs + al(b_offs), o_perm = o_ptr + al(b_ptr);
-    size_t o_dense = o_perm + al(b_perm), o_ent = o_dense + al(b_dense), total = o_ent + al(b_ent);
+    size_t o_dense = o_perm + al(b_perm), o_ent = o_dense + al(b_dense);
+    size_t o_ple = o_ent + al(b_ent), o_plp = o_ple + al(b_ple), o_plo = o_plp + al(b_plp), total = o_plo + al(b_plo);
     h->packed_bytes = (int64_t)(b_vals + b_offs + b_ptr + b_perm + b_dense + b_ent);
     if (h->desc.flags & CADNN_PACK_HOST_ONLY) return CADNN_OK;
     if (total == 0) total = 256;
@@ -193,6 +195,12 @@ cadnn_status upload(cadnn_weights *h)
     if (b_dense) CADNN_CUDA_TRY(cudaMemcpy(base + o_dense, h->dense_f.data(), b_dense, cudaMemcpyHostToDevice));
     if (b_ent) CADNN_CUDA_TRY(cudaMemcpy(base + o_ent, h->ent.data(), b_ent, cudaMemcpyHostToDevice));
     h->d_ent = (const uint32_t *)(base + o_ent);
+    if (b_ple) CADNN_CUDA_TRY(cudaMemcpy(base + o_ple, h->pl_ent.data(), b_ple, cudaMemcpyHostToDevice));
+    if (b_plp) CADNN_CUDA_TRY(cudaMemcpy(base + o_plp, h->pl_ptr.data(), b_plp, cudaMemcpyHostToDevice));
+    if (b_plo) CADNN_CUDA_TRY(cudaMemcpy(base + o_plo, h->pl_order.data(), b_plo, cudaMemcpyHostToDevice));
+    h->d_pl_ent = (const uint32_t *)(base + o_ple);
+    h->d_pl_ptr = (const int32_t *)(base + o_plp);
+    h->d_pl_order = (const int32_t *)(base + o_plo);
     // A copy from pageable host memory may return before its DMA has landed; kernels on
     // non-blocking streams are not ordered behind it, so wait for it here.
     CADNN_CUDA_TRY(cudaStreamSynchronize(cudaStreamLegacy));
@@ -508,6 +516,146 @@ cadnn_status autotune_sconv(cadnn_weights *h, const Src &src, const Geometry &g,
     return CADNN_OK;
 }
 
+// Filters dealt to the warp slots of the planar kernel: blocks of G consecutive output
+// channels, longest-processing-time inside a block so that a block's warps finish together.
+void planar_order(cadnn_weights *h, const std::vector<int64_t> &row_nnz)
+{
+    const int c_out = h->desc.c_out;
+    const int G = std::max(1, h->pl_NW / std::max(1, h->pl_KSW)) * h->pl_RPW;
+    const int n_groups = ceil_div(c_out, G);
+    // constant capacity whatever the grouping, so that the device copy can be rewritten in place
+    h->pl_order.assign(std::max((size_t)n_groups * G, (size_t)round_up(c_out, 128) + 128), -1);
+    for (int gi = 0; gi < n_groups; ++gi) {
+        int lo = gi * G, hi = std::min(c_out, lo + G);
+        std::vector<int64_t> load(row_nnz.begin() + lo, row_nnz.begin() + hi);
+        std::vector<int> slot;
+        balance_block(load, G, h->pl_RPW, slot);
+        for (int sl = 0; sl < G; ++sl)
+            if (slot[sl] >= 0) h->pl_order[lo + sl] = lo + slot[sl];
+    }
+}
+
+// Channel-planar image of a float conv layer: offsets address [c_in][in_h + 2][in_w + 2].
+void build_planar_image(cadnn_weights *h, const Src &src, const std::vector<int64_t> &row_nnz)
+{
+    const cadnn_layer_desc &d = h->desc;
+    const int halo = kPlanarHalo;
+    if (src.s8 || d.groups != 1 || d.pad > halo || d.kh - 1 - d.pad > halo || d.kw - 1 - d.pad > halo) return;
+    const long long plane = (long long)(d.in_h + 2 * halo) * (d.in_w + 2 * halo);
+    if (plane * d.c_in >= (1LL << 31)) return;
+    const int wp = d.in_w + 2 * halo;
+    h->pl_ptr.assign(d.c_out + 1, 0);
+    h->pl_ent.clear();
+    int32_t running = 0;
+    for (int co = 0; co < d.c_out; ++co) {
+        h->pl_ptr[co] = running;
+        int real = 0;
+        for (int ci = 0; ci < d.c_in; ++ci)
+            for (int ky = 0; ky < d.kh; ++ky)
+                for (int kx = 0; kx < d.kw; ++kx) {
+                    size_t wi = (((size_t)co * d.kh + ky) * d.kw + kx) * d.c_in + ci;
+                    if (!src.kept(wi)) continue;
+                    float v = src.fval(wi);
+                    uint32_t bits;
+                    memcpy(&bits, &v, 4);
+                    h->pl_ent.push_back(bits);
+                    h->pl_ent.push_back((uint32_t)(ci * plane + (long long)(ky + halo - d.pad) * wp + kx + halo - d.pad));
+                    ++real;
+                }
+        if (real & 1) {   // padding entry: weight 0 at offset 0
+            h->pl_ent.push_back(0u);
+            h->pl_ent.push_back(0u);
+        }
+        running += real + (real & 1);
+    }
+    h->pl_ptr[d.c_out] = running;
+    // schedule: pixel bands per lane from the plane size, one or two filters per warp
+    const long long qtot = (long long)h->h_out * (h->w_out + 2 * halo) * std::max(1, d.batch_hint);
+    h->pl_NW = 8;
+    h->pl_T = qtot >= 8L * 32 * kSmCount ? 8 : qtot >= 2L * 32 * kSmCount ? 4 : qtot >= 512 ? 2 : 1;
+    long long warps = ((qtot + 32 * h->pl_T - 1) / (32 * h->pl_T)) * d.c_out;
+    h->pl_RPW = warps >= 64L * kSmCount * 8 ? 4 : warps >= 32L * kSmCount * 4 ? 2 : 1;
+    // few warps in the whole layer: let several warps share a filter's nonzeros
+    h->pl_KSW = 1;
+    const long long mean_pairs = std::max<long long>(1, running / 2 / std::max(1, d.c_out));
+    while (h->pl_KSW < 8 && warps * h->pl_KSW < 24L * kSmCount && mean_pairs / (h->pl_KSW * 2) >= 8) h->pl_KSW *= 2;
+    planar_order(h, row_nnz);
+    h->has_planar = true;
+}
+
+// Time the planar kernel's launch shapes on the device and keep the fastest (the stored image does
+// not depend on them; only the dealing of filters to warps does).
+void autotune_planar(cadnn_weights *h, const std::vector<int64_t> &row_nnz)
+{
+    const cadnn_layer_desc &d = h->desc;
+    const int halo = kPlanarHalo, batch = std::max(1, d.batch_hint);
+    const size_t xb = (size_t)batch * d.c_in * (d.in_h + 2 * halo) * (d.in_w + 2 * halo) * 4;
+    const size_t yb = (size_t)batch * d.c_out * (h->h_out + 2 * halo) * (h->w_out + 2 * halo) * 4;
+    void *x = nullptr, *y = nullptr;
+    cudaStream_t st = nullptr;
+    if (cudaMalloc(&x, xb) != cudaSuccess || cudaMalloc(&y, yb) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking) != cudaSuccess) {
+        if (x) cudaFree(x);
+        if (y) cudaFree(y);
+        cudaGetLastError();
+        return;
+    }
+    cudaMemsetAsync(x, 0, xb, st);
+    cudaMemsetAsync(y, 0, yb, st);
+    int32_t *d_order = const_cast<int32_t *>(h->d_pl_order);
+    const size_t order_cap = h->pl_order.size();   // device room reserved for the order array
+    float best_us = -1.0f;
+    int bT = h->pl_T, bNW = h->pl_NW, bRPW = h->pl_RPW, bKSW = h->pl_KSW;
+    LaunchEpilogue ep;
+    ep.out_dtype = CADNN_F32;
+    ep.act = CADNN_ACT_RELU;
+    for (int T : {1, 2, 4, 8})
+        for (int nw : {4, 8, 16, 32})
+            for (int ksw : {1, 2, 4, 8})
+                for (int rpw : {1, 2, 4}) {
+                    if (ksw > nw || nw > (T <= 2 ? 32 : T <= 4 ? 16 : 8)) continue;
+                    h->pl_T = T; h->pl_NW = nw; h->pl_KSW = ksw; h->pl_RPW = rpw;
+                    planar_order(h, row_nnz);
+                    if (h->pl_order.size() > order_cap) continue;
+                    if (cudaMemcpyAsync(d_order, h->pl_order.data(), h->pl_order.size() * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+                        cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); continue; }
+                    cudaGraph_t g = nullptr;
+                    cudaGraphExec_t ge = nullptr;
+                    if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { cudaGetLastError(); continue; }
+                    bool ok = true;
+                    for (int r = 0; r < 8 && ok; ++r) ok = launch_sconv_planar(h, x, batch, y, ep, st) == CADNN_OK;
+                    if (cudaStreamEndCapture(st, &g) != cudaSuccess) ok = false;
+                    if (ok && cudaGraphInstantiate(&ge, g, 0) == cudaSuccess) {
+                        cudaEvent_t e0, e1;
+                        cudaEventCreate(&e0);
+                        cudaEventCreate(&e1);
+                        cudaGraphLaunch(ge, st);
+                        cudaEventRecord(e0, st);
+                        cudaGraphLaunch(ge, st);
+                        cudaEventRecord(e1, st);
+                        if (cudaStreamSynchronize(st) == cudaSuccess) {
+                            float ms = 0.0f;
+                            cudaEventElapsedTime(&ms, e0, e1);
+                            float us = ms * 1e3f / 8.0f;
+                            if (best_us < 0.0f || us < best_us) { best_us = us; bT = T; bNW = nw; bRPW = rpw; bKSW = ksw; }
+                        }
+                        cudaEventDestroy(e0);
+                        cudaEventDestroy(e1);
+                    }
+                    if (ge) cudaGraphExecDestroy(ge);
+                    if (g) cudaGraphDestroy(g);
+                    cudaGetLastError();
+                }
+    h->pl_T = bT; h->pl_NW = bNW; h->pl_RPW = bRPW; h->pl_KSW = bKSW;
+    planar_order(h, row_nnz);
+    cudaMemcpyAsync(d_order, h->pl_order.data(), h->pl_order.size() * 4, cudaMemcpyHostToDevice, st);
+    cudaStreamSynchronize(st);
+    cudaStreamDestroy(st);
+    cudaFree(x);
+    cudaFree(y);
+    cudaGetLastError();
+}
+
 cadnn_status pack_sconv(cadnn_weights *h, const Src &src)
 {
     const cadnn_layer_desc &d = h->desc;
@@ -530,6 +678,8 @@ cadnn_status pack_sconv(cadnn_weights *h, const Src &src)
         if (st != CADNN_OK) return st;
     }
     apply_env_override(g, linear, h->s);
+    h->row_nnz = row_nnz;
+    build_planar_image(h, src, row_nnz);
     return build_sconv_image(h, src, g, row_nnz);
 }
 
@@ -638,6 +788,8 @@ cadnn_status pack_common(const cadnn_layer_desc *desc, const Src &src, cadnn_wei
         else if (is_fc && std::max(1, d.batch_hint) <= 8 && d.c_in <= 65536) st = pack_fc_spmv(h, src);
         else st = pack_sconv(h, src);
         if (st == CADNN_OK) st = upload(h);
+        if (st == CADNN_OK && h->has_planar && h->on_device && (d.flags & CADNN_PACK_AUTOTUNE))
+            autotune_planar(h, h->row_nnz);
     } catch (const std::bad_alloc &) {
         st = CADNN_E_ALLOC;
     }

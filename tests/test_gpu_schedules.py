@@ -185,3 +185,70 @@ def test_resnet50_full_batch1_with_timed_schedules():
     got = y.cpu().numpy()
     assert_close_f32(got, want, "logits", floor=NET_FLOOR)
     assert set(np.argsort(-got[0])[:5]) == set(np.argsort(-want[0])[:5])
+
+
+def _to_planar(a):
+    """NHWC numpy -> [n, c, h+2, w+2] torch CUDA tensor with a zero border."""
+    n, h, w, c = a.shape
+    t = torch.zeros((n, c, h + 2, w + 2), dtype=torch.float32, device=DEV)
+    t[:, :, 1:h + 1, 1:w + 1] = torch.from_numpy(np.ascontiguousarray(a.transpose(0, 3, 1, 2))).to(DEV)
+    return t
+
+
+PLANAR_CASES = [
+    # n, h, w, c_in, c_out, k, stride, density
+    (1, 56, 56, 64, 64, 3, 1, 0.125), (2, 28, 28, 128, 128, 3, 2, 0.125), (1, 14, 14, 256, 200, 3, 1, 0.125),
+    (3, 7, 7, 512, 96, 3, 1, 0.125), (1, 56, 56, 64, 256, 1, 1, 0.125), (2, 28, 28, 512, 130, 1, 2, 0.125),
+    (1, 13, 17, 10, 7, 3, 1, 0.5), (1, 13, 17, 10, 7, 3, 2, 0.5), (1, 9, 9, 16, 16, 1, 1, 1.0), (1, 9, 9, 16, 16, 3, 1, 0.0),
+]
+
+
+@pytest.mark.parametrize("case", PLANAR_CASES)
+def test_planar_sparse_conv(case):
+    B = _B()
+    n, h, w, c_in, c_out, k, stride, density = case
+    pad = k // 2
+    g = gen.rng(sum(case[:7]))
+    x = gen.relu_normal_input(g, (n, h, w, c_in))
+    wt = gen.he_weights(g, c_out, k, k, c_in)
+    mask = None if density >= 1.0 else gen.magnitude_mask(wt, density)
+    scale, bias = gen.folded_bn(g, c_out)
+    ho, wo = ref.out_hw(h, w, k, stride, pad)
+    res = gen.normal_input(g, (n, ho, wo, c_out))
+    want = ref.conv2d_f32(x, wt, mask, stride, pad, 1, scale, bias, res, "relu")
+    d = B.make_desc(c_in, c_out, k, k, stride, pad, 1, h, w, n, "f32", autotune=(c_in >= 256))
+    wh = B.cadnn_pack(d, wt, mask)
+    y = torch.zeros((n, c_out, ho + 2, wo + 2), device=DEV)
+    dev = lambda a: torch.from_numpy(a).to(DEV)
+    B.cadnn_conv2d_planar(wh, _to_planar(x), y, dev(scale), dev(bias), _to_planar(res), "relu")
+    torch.cuda.synchronize()
+    yc = y.cpu().numpy()
+    got = yc[:, :, 1:ho + 1, 1:wo + 1].transpose(0, 2, 3, 1)
+    # the residual (|res| up to ~4) cancels against the conv result: a few ulps of the operands is the floor
+    assert_close_f32(got, want, str(case), floor=NET_FLOOR)
+    # the border is never written
+    border = yc.copy()
+    border[:, :, 1:ho + 1, 1:wo + 1] = 0
+    assert not border.any()
+
+
+def test_planar_and_nhwc_networks_agree_with_the_oracle():
+    from oracle import forward as oracle_forward
+    from paper_1905_00571_b200.network import PackedModel
+    m = models.resnet50(width=0.25, image=64, classes=100)
+    x = models.make_input(m, 2)
+    want, _ = oracle_forward.forward(m, x)
+    outs = []
+    for no_planar in (False, True):
+        if no_planar:
+            os.environ["CADNN_NO_PLANAR"] = "1"
+        try:
+            pm = PackedModel(m, 2, DEV)
+        finally:
+            os.environ.pop("CADNN_NO_PLANAR", None)
+        y = pm.new_output()
+        pm.forward(torch.from_numpy(x).to(DEV), y)
+        pm.forward(torch.from_numpy(x).to(DEV), y)
+        torch.cuda.synchronize()
+        outs.append(y.cpu().numpy())
+        assert_close_f32(outs[-1], want, "planar off" if no_planar else "planar on", floor=NET_FLOOR)
