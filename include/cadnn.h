@@ -125,6 +125,17 @@ cadnn_status cadnn_weights_info(const cadnn_weights *w, int64_t *nnz, int64_t *p
 cadnn_status cadnn_weights_schedule(const cadnn_weights *w, int sched[16]);
 
 /*
+ * Schedule of the layer's channel-planar variant (the one cadnn_forward and
+ * cadnn_conv2d_planar run): sched[0..13] = variant (0 none, 1 direct loads, 2 tile staged in
+ * shared memory), position bands per lane, filters per warp, warps per block, warps sharing
+ * a filter, filters per block, channel chunk, pipeline stages, channel chunks, tiles per
+ * image, shared-memory bytes per block, entries per weight record, and the times measured
+ * by CADNN_PACK_AUTOTUNE for the staged and the direct variant in hundredths of a
+ * microsecond (negative = not measured); sched[14..15] = 0.  Host ints.
+ */
+cadnn_status cadnn_weights_planar_schedule(const cadnn_weights *w, int sched[16]);
+
+/*
  * Per-warp load of the packed image: for every (filter block, warp) the number of
  * stored nonzeros that warp walks.  n_out receives the count; loads (host, may be
  * NULL) receives up to cap entries.
@@ -175,9 +186,11 @@ cadnn_status cadnn_conv2d(const cadnn_weights *w, const void *x, int n, int h, i
  * layout transformation": data laid out to fit the processor).  This is the layout
  * cadnn_forward uses between the layers of a float network; the call exists so that it can
  * be checked on its own.
- *   x device float [n][c_in][in_h + 2][in_w + 2], y device float [n][c_out][h_out + 2][w_out + 2]:
- *   every plane carries a one-pixel border that MUST be zero in x and that the call never
- *   writes in y (so a y buffer zeroed once stays a valid input for the next layer).
+ *   x device float [n][c_in][pitch(in_h, in_w)], y device float [n][c_out][pitch(h_out, w_out)]:
+ *   a plane is (h + 2) x (w + 2) values, row-major, and consecutive planes are
+ *   pitch(h, w) = (h + 2) * (w + 2) rounded up to a multiple of 4 floats apart.  The one-pixel
+ *   border and the padding behind a plane MUST be zero in x; the call never writes them in y
+ *   (so a y buffer zeroed once stays a valid input for the next layer).
  *   residual (optional) has y's layout.  Float layers with pad <= 1 and k - 1 - pad <= 1 only:
  *   E_UNSUPPORTED otherwise.  Same epilogue, same errors as cadnn_conv2d.
  */

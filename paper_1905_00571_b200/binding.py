@@ -52,6 +52,7 @@ _SIGS = {
     "cadnn_pack_q8": (_i, [ctypes.POINTER(LayerDesc), _vp, _vp, ctypes.POINTER(_vp)]),
     "cadnn_weights_info": (_i, [_vp, _i64p, _i64p, ctypes.POINTER(_i)]),
     "cadnn_weights_schedule": (_i, [_vp, ctypes.POINTER(_i)]),
+    "cadnn_weights_planar_schedule": (_i, [_vp, ctypes.POINTER(_i)]),
     "cadnn_weights_warp_loads": (_i, [_vp, _i64p, _i, ctypes.POINTER(_i)]),
     "cadnn_weights_unpack": (_i, [_vp, _vp, _vp]),
     "cadnn_weights_free": (None, [_vp]),
@@ -172,6 +173,14 @@ def cadnn_weights_schedule(w):
     return dict(zip(keys, list(arr)))
 
 
+def cadnn_weights_planar_schedule(w):
+    arr = (ctypes.c_int * 16)()
+    _check(_lib.cadnn_weights_planar_schedule(w.handle, arr), "cadnn_weights_planar_schedule")
+    keys = ("variant", "T", "RPW", "NW", "KS", "G", "CIc", "stages", "chunks", "tiles", "smem", "max_entries",
+            "staged_us_x100", "direct_us_x100")
+    return dict(zip(keys, list(arr)))
+
+
 def cadnn_weights_warp_loads(w):
     n = ctypes.c_int()
     _check(_lib.cadnn_weights_warp_loads(w.handle, None, 0, ctypes.byref(n)), "cadnn_weights_warp_loads")
@@ -207,7 +216,8 @@ def cadnn_conv2d(w, x, y, scale=None, bias=None, residual=None, act="none", out_
 
 
 def cadnn_conv2d_planar(w, x, y, scale=None, bias=None, residual=None, act="none", stream=None):
-    """x [n, c_in, h+2, w+2], y [n, c_out, ho+2, wo+2]: float CUDA tensors with a zero one-pixel border."""
+    """x [n, c_in, pitch(h, w)], y [n, c_out, pitch(ho, wo)]: float CUDA tensors of channel planes, each
+    (h+2) x (w+2) with a zero one-pixel border, followed by padding to pitch = a multiple of 4 floats."""
     ep = _epilogue(scale, bias, residual, act, F32)
     _check(_lib.cadnn_conv2d_planar(w.handle, _dev_ptr(x), int(x.shape[0]), _dev_ptr(y), ctypes.byref(ep), _stream(stream)),
            "cadnn_conv2d_planar")

@@ -82,6 +82,7 @@ cadnn_status cadnn_conv2d_planar(const cadnn_weights *w, const void *x, int n, v
     LaunchEpilogue le;
     cadnn_status st = check_epilogue(w, ep, le);
     if (st != CADNN_OK) return st;
+    if (w->has_ps && w->use_ps) return launch_sconv_planar_staged(w, x, n, y, le, (cudaStream_t)stream);
     return launch_sconv_planar(w, x, n, y, le, (cudaStream_t)stream);
 }
 

@@ -14,6 +14,12 @@ enum KernelKind {
 };
 
 static const int kPlanarHalo = 1;     // zero border of the channel-planar activation layout
+// floats from one channel plane of a planar tensor to the next: the padded plane rounded up to a
+// multiple of 4, so that 16-byte copies that start at a multiple of 4 inside a plane are aligned
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+static inline int planar_pitch(int h, int w) { return ((h + 2 * kPlanarHalo) * (w + 2 * kPlanarHalo) + 3) & ~3; }
 static const int kWarpsPerBlock = 8;  // fc kernel; the conv kernels take it from the schedule
 
 // Per-layer schedule chosen by the packer (Section 4, "Optimization parameters selection").
@@ -37,6 +43,22 @@ struct Schedule {
     int ksplit = 1;          // thread blocks per cluster splitting the channel chunks (partial sums meet in DSMEM)
     int max_entries = 0;     // (padded) entries of the fullest (chunk, filter block) record
     int tile_bytes = 0, stage_bytes = 0, smem_bytes = 0;
+};
+
+// Schedule of the shared-memory-staged planar kernel (planar_staged.cu).
+struct PsSchedule {
+    int T = 1;        // position bands per lane (a band = 32 consecutive positions of the padded plane)
+    int RPW = 1;      // filters per warp slot
+    int NW = 8;       // warps per block = filter slots x KS
+    int KS = 1;       // warps sharing a filter (each takes a share of its nonzeros in every chunk)
+    int G = 8;        // filters per block = (NW / KS) * RPW
+    int CIc = 0;      // input channels staged per chunk
+    int stages = 1;
+    int n_chunks = 1, n_groups = 1;
+    int A = 0, L = 32;           // staged margin / floats per channel
+    int q_start = 0, tiles = 1;  // first computed position, tiles per image
+    int max_entries = 0;
+    int hdr_bytes = 0, block_bytes = 0, tile_bytes = 0, stage_bytes = 0, smem_bytes = 0;
 };
 
 struct cadnn_weights {
@@ -74,6 +96,16 @@ struct cadnn_weights {
     const uint32_t *d_pl_ent = nullptr;
     const int32_t *d_pl_ptr = nullptr;
     const int32_t *d_pl_order = nullptr;
+
+    // shared-memory-staged planar variant (stride-1 "same" float conv): records per (chunk, filter block)
+    bool has_ps = false;
+    bool use_ps = false;             // the network runner prefers it over the direct planar kernel
+    PsSchedule ps;
+    float ps_us = -1.0f, pl_us = -1.0f;   // measured time of the staged / direct planar kernel (autotune), microseconds
+    std::vector<uint32_t> ps_ent;
+    std::vector<int32_t> ps_perm;    // packed row -> output channel, -1 = padding row
+    const uint32_t *d_ps_ent = nullptr;
+    const int32_t *d_ps_perm = nullptr;
 
     // device image (one allocation)
     void *d_blob = nullptr;
@@ -114,6 +146,8 @@ cadnn_status launch_dense_smallc(const cadnn_weights *w, const void *x, int n, v
                                  cudaStream_t st);
 cadnn_status launch_sconv_planar(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
                                  cudaStream_t st);
+cadnn_status launch_sconv_planar_staged(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
+                                        cudaStream_t st);
 cadnn_status launch_maxpool_planar(const float *x, int n, int h, int wd, int c, int k, int stride, int pad, float *y,
                                    bool pdl, cudaStream_t st);
 cadnn_status launch_gavgpool_planar(const float *x, int n, int h, int wd, int c, float *y, bool pdl, cudaStream_t st);

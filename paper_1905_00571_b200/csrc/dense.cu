@@ -171,7 +171,7 @@ __global__ void __launch_bounds__(256) stem_kernel(const StemParams p)
             const float *acc = rr ? acc1 : acc0;
             const size_t o = (((size_t)img * p.h_out + oy) * p.w_out + ox) * p.c_out + cbase;
             const int wp = p.w_out + 2 * p.halo;
-            const size_t plane = (size_t)(p.h_out + 2 * p.halo) * wp;
+            const size_t plane = (size_t)planar_pitch(p.h_out, p.w_out);
             const size_t opl = (size_t)img * p.c_out * plane + (size_t)(oy + p.halo) * wp + ox + p.halo;
 #pragma unroll
             for (int c = 0; c < kStemCo; ++c) {

@@ -65,6 +65,7 @@ cadnn_status run_op(cadnn_net *net, const cadnn_op &op, const void *x, void *y, 
                 le.planar_out = true;
                 return launch_dense_smallc(op.w, src, si.n, dst, le, st);
             }
+            if (op.w->has_ps && op.w->use_ps) return launch_sconv_planar_staged(op.w, src, si.n, dst, le, st);
             return launch_sconv_planar(op.w, src, si.n, dst, le, st);
         }
         if (op.kind == CADNN_OP_MAXPOOL)
@@ -234,7 +235,7 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
         so.defined = true;
         so.bytes = (int64_t)so.n * so.h * so.w * so.c * dtype_size(so.dtype);
         const bool padded = net->planar && (op.kind == CADNN_OP_CONV || op.kind == CADNN_OP_MAXPOOL);
-        if (padded) so.bytes = (int64_t)so.n * so.c * (so.h + 2 * kPlanarHalo) * (so.w + 2 * kPlanarHalo) * 4;
+        if (padded) so.bytes = (int64_t)so.n * so.c * planar_pitch(so.h, so.w) * 4;
         if (op.dst != net->out_slot) {
             size_t alloc = (size_t)((so.bytes + 255) / 256 * 256);
             cudaError_t e = cudaMalloc(&so.ptr, alloc ? alloc : 256);

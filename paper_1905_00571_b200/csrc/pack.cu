@@ -176,7 +176,9 @@ cadnn_status upload(cadnn_weights *h)
     size_t b_ple = h->pl_ent.size() * 4, b_plp = h->pl_ptr.size() * 4, b_plo = h->pl_order.size() * 4;
     size_t o_vals = 0, o_offs = o_vals + al(b_vals), o_ptr = o_offs + al(b_offs), o_perm = o_ptr + al(b_ptr);
     size_t o_dense = o_perm + al(b_perm), o_ent = o_dense + al(b_dense);
-    size_t o_ple = o_ent + al(b_ent), o_plp = o_ple + al(b_ple), o_plo = o_plp + al(b_plp), total = o_plo + al(b_plo);
+    size_t b_pse = h->ps_ent.size() * 4, b_psp = h->ps_perm.size() * 4;
+    size_t o_ple = o_ent + al(b_ent), o_plp = o_ple + al(b_ple), o_plo = o_plp + al(b_plp), o_pse = o_plo + al(b_plo);
+    size_t o_psp = o_pse + al(b_pse), total = o_psp + al(b_psp);
     h->packed_bytes = (int64_t)(b_vals + b_offs + b_ptr + b_perm + b_dense + b_ent);
     if (h->desc.flags & CADNN_PACK_HOST_ONLY) return CADNN_OK;
     if (total == 0) total = 256;
@@ -198,6 +200,10 @@ cadnn_status upload(cadnn_weights *h)
     if (b_ple) CADNN_CUDA_TRY(cudaMemcpy(base + o_ple, h->pl_ent.data(), b_ple, cudaMemcpyHostToDevice));
     if (b_plp) CADNN_CUDA_TRY(cudaMemcpy(base + o_plp, h->pl_ptr.data(), b_plp, cudaMemcpyHostToDevice));
     if (b_plo) CADNN_CUDA_TRY(cudaMemcpy(base + o_plo, h->pl_order.data(), b_plo, cudaMemcpyHostToDevice));
+    if (b_pse) CADNN_CUDA_TRY(cudaMemcpy(base + o_pse, h->ps_ent.data(), b_pse, cudaMemcpyHostToDevice));
+    if (b_psp) CADNN_CUDA_TRY(cudaMemcpy(base + o_psp, h->ps_perm.data(), b_psp, cudaMemcpyHostToDevice));
+    h->d_ps_ent = (const uint32_t *)(base + o_pse);
+    h->d_ps_perm = (const int32_t *)(base + o_psp);
     h->d_pl_ent = (const uint32_t *)(base + o_ple);
     h->d_pl_ptr = (const int32_t *)(base + o_plp);
     h->d_pl_order = (const int32_t *)(base + o_plo);
@@ -541,7 +547,7 @@ void build_planar_image(cadnn_weights *h, const Src &src, const std::vector<int6
     const cadnn_layer_desc &d = h->desc;
     const int halo = kPlanarHalo;
     if (src.s8 || d.groups != 1 || d.pad > halo || d.kh - 1 - d.pad > halo || d.kw - 1 - d.pad > halo) return;
-    const long long plane = (long long)(d.in_h + 2 * halo) * (d.in_w + 2 * halo);
+    const long long plane = planar_pitch(d.in_h, d.in_w);
     if (plane * d.c_in >= (1LL << 31)) return;
     const int wp = d.in_w + 2 * halo;
     h->pl_ptr.assign(d.c_out + 1, 0);
@@ -589,8 +595,8 @@ void autotune_planar(cadnn_weights *h, const std::vector<int64_t> &row_nnz)
 {
     const cadnn_layer_desc &d = h->desc;
     const int halo = kPlanarHalo, batch = std::max(1, d.batch_hint);
-    const size_t xb = (size_t)batch * d.c_in * (d.in_h + 2 * halo) * (d.in_w + 2 * halo) * 4;
-    const size_t yb = (size_t)batch * d.c_out * (h->h_out + 2 * halo) * (h->w_out + 2 * halo) * 4;
+    const size_t xb = (size_t)batch * d.c_in * planar_pitch(d.in_h, d.in_w) * 4;
+    const size_t yb = (size_t)batch * d.c_out * planar_pitch(h->h_out, h->w_out) * 4;
     void *x = nullptr, *y = nullptr;
     cudaStream_t st = nullptr;
     if (cudaMalloc(&x, xb) != cudaSuccess || cudaMalloc(&y, yb) != cudaSuccess ||
@@ -610,10 +616,10 @@ void autotune_planar(cadnn_weights *h, const std::vector<int64_t> &row_nnz)
     ep.out_dtype = CADNN_F32;
     ep.act = CADNN_ACT_RELU;
     for (int T : {1, 2, 4, 8})
-        for (int nw : {4, 8, 16, 32})
+        for (int nw : {4, 8, 16})
             for (int ksw : {1, 2, 4, 8})
                 for (int rpw : {1, 2, 4}) {
-                    if (ksw > nw || nw > (T <= 2 ? 32 : T <= 4 ? 16 : 8)) continue;
+                    if (ksw > nw || nw > (T <= 4 ? 16 : 8)) continue;
                     h->pl_T = T; h->pl_NW = nw; h->pl_KSW = ksw; h->pl_RPW = rpw;
                     planar_order(h, row_nnz);
                     if (h->pl_order.size() > order_cap) continue;
@@ -647,6 +653,8 @@ void autotune_planar(cadnn_weights *h, const std::vector<int64_t> &row_nnz)
                     cudaGetLastError();
                 }
     h->pl_T = bT; h->pl_NW = bNW; h->pl_RPW = bRPW; h->pl_KSW = bKSW;
+    h->pl_us = best_us;
+    if (h->has_ps && h->ps_us > 0.0f && best_us > 0.0f) h->use_ps = h->ps_us <= best_us || getenv("CADNN_FORCE_STAGED") != nullptr;
     planar_order(h, row_nnz);
     cudaMemcpyAsync(d_order, h->pl_order.data(), h->pl_order.size() * 4, cudaMemcpyHostToDevice, st);
     cudaStreamSynchronize(st);
@@ -654,6 +662,296 @@ void autotune_planar(cadnn_weights *h, const std::vector<int64_t> &row_nnz)
     cudaFree(x);
     cudaFree(y);
     cudaGetLastError();
+}
+
+// ---- shared-memory-staged planar kernel (planar_staged.cu): schedule, image, timing ----
+
+// kept weights of every filter as (input channel, tap shift inside the padded plane, value), channel-major
+struct PsRows {
+    std::vector<int32_t> ptr;   // [c_out + 1]
+    std::vector<int32_t> ci, tap;
+    std::vector<float> v;
+};
+
+bool ps_eligible(const cadnn_layer_desc &d, bool s8)
+{
+    if (s8 || d.groups != 1 || d.stride != 1 || d.kh != d.kw || 2 * d.pad != d.kh - 1 || d.pad > kPlanarHalo) return false;
+    return (long long)planar_pitch(d.in_h, d.in_w) * d.c_in < (1LL << 31);
+}
+
+void ps_collect_rows(const cadnn_layer_desc &d, const Src &src, PsRows &r)
+{
+    const int wp = d.in_w + 2 * kPlanarHalo;
+    r.ptr.assign(d.c_out + 1, 0);
+    for (int co = 0; co < d.c_out; ++co) {
+        r.ptr[co] = (int32_t)r.ci.size();
+        for (int ci = 0; ci < d.c_in; ++ci)
+            for (int ky = 0; ky < d.kh; ++ky)
+                for (int kx = 0; kx < d.kw; ++kx) {
+                    const size_t wi = (((size_t)co * d.kh + ky) * d.kw + kx) * d.c_in + ci;
+                    if (!src.kept(wi)) continue;
+                    r.ci.push_back(ci);
+                    r.tap.push_back((ky - d.pad) * wp + (kx - d.pad));
+                    r.v.push_back(src.fval(wi));
+                }
+    }
+    r.ptr[d.c_out] = (int32_t)r.ci.size();
+}
+
+// derived fields of a staged-planar schedule from (T, RPW, NW, KS, CIc, stages); false if it cannot run
+bool ps_finish(const cadnn_layer_desc &d, PsSchedule &s)
+{
+    const int wp = d.in_w + 2 * kPlanarHalo;
+    if (s.KS < 1 || s.KS > s.NW || s.NW % s.KS || s.RPW * s.T > 32) return false;
+    s.G = (s.NW / s.KS) * s.RPW;
+    s.n_groups = ceil_div(d.c_out, s.G);
+    s.CIc = std::max(1, std::min(s.CIc, d.c_in));
+    s.n_chunks = ceil_div(d.c_in, s.CIc);
+    s.stages = std::max(1, std::min(std::min(s.stages, 3), s.n_chunks));
+    s.A = round_up(d.pad * (wp + 1), 4);
+    s.L = 32 * s.T + 2 * s.A;
+    s.q_start = (kPlanarHalo * (wp + 1)) & ~3;                         // first interior position, rounded down
+    const int q_end = (d.in_h + kPlanarHalo - 1) * wp + d.in_w + kPlanarHalo;   // one past the last interior position
+    s.tiles = ceil_div(q_end - s.q_start, 32 * s.T);
+    s.tile_bytes = s.CIc * s.L * 4;
+    s.hdr_bytes = round_up(s.G * s.KS + 1, 4) * 4;
+    return true;
+}
+
+void ps_finish_smem(PsSchedule &s)
+{
+    s.block_bytes = s.hdr_bytes + s.max_entries * 8;
+    s.stage_bytes = s.tile_bytes + s.block_bytes;
+    const int red = (s.NW / s.KS) * (s.KS - 1) * s.RPW * s.T * 128;   // partial sums of the warps that share filters
+    s.smem_bytes = std::max(s.stages * s.stage_bytes, red);
+}
+
+// Image for schedule h->ps (through ps_finish): one fixed-size record per (chunk, filter block): a header
+// of G * KS + 1 segment starts, then the entries {value bits, byte offset into the staged tile}; the
+// nonzeros a filter has in the chunk are cut into KS equal segments, each padded to an even count.
+bool build_ps_image(cadnn_weights *h, const PsRows &rows, const std::vector<int64_t> &row_nnz)
+{
+    const cadnn_layer_desc &d = h->desc;
+    PsSchedule &s = h->ps;
+    const int c_pad = s.n_groups * s.G;
+    h->ps_perm.assign(c_pad, -1);
+    for (int gi = 0; gi < s.n_groups; ++gi) {
+        int lo = gi * s.G, hi = std::min(d.c_out, lo + s.G);
+        std::vector<int64_t> load(row_nnz.begin() + lo, row_nnz.begin() + hi);
+        std::vector<int> slot;
+        balance_block(load, s.G, s.RPW, slot);
+        for (int sl = 0; sl < s.G; ++sl)
+            if (slot[sl] >= 0) h->ps_perm[lo + sl] = lo + slot[sl];
+    }
+    const int hdr_words = s.hdr_bytes / 4;
+    std::vector<std::vector<uint32_t>> blocks((size_t)s.n_chunks * s.n_groups);
+    std::vector<int32_t> cur(rows.ptr.begin(), rows.ptr.end() - 1);   // next unread nonzero of every filter
+    s.max_entries = 0;
+    for (int c = 0; c < s.n_chunks; ++c) {
+        const int c0 = c * s.CIc, c1 = std::min(d.c_in, c0 + s.CIc);
+        for (int gi = 0; gi < s.n_groups; ++gi) {
+            std::vector<uint32_t> &blk = blocks[(size_t)c * s.n_groups + gi];
+            blk.assign(hdr_words, 0u);
+            int running = 0;
+            for (int sl = 0; sl < s.G; ++sl) {
+                const int co = h->ps_perm[gi * s.G + sl];
+                int lo = 0, cnt = 0;
+                if (co >= 0) {
+                    lo = cur[co];
+                    int e = lo;
+                    while (e < rows.ptr[co + 1] && rows.ci[e] < c1) ++e;
+                    cnt = e - lo;
+                    cur[co] = e;
+                }
+                for (int k = 0; k < s.KS; ++k) {
+                    blk[sl * s.KS + k] = (uint32_t)running;
+                    const int a = (int)((long long)cnt * k / s.KS), b = (int)((long long)cnt * (k + 1) / s.KS);
+                    for (int e = lo + a; e < lo + b; ++e) {
+                        uint32_t bits;
+                        memcpy(&bits, &rows.v[e], 4);
+                        blk.push_back(bits);
+                        blk.push_back((uint32_t)(((rows.ci[e] - c0) * s.L + s.A + rows.tap[e]) * 4));
+                    }
+                    if ((b - a) & 1) {   // padding entry: weight 0 at offset 0
+                        blk.push_back(0u);
+                        blk.push_back(0u);
+                    }
+                    running += (b - a) + ((b - a) & 1);
+                }
+            }
+            blk[s.G * s.KS] = (uint32_t)running;
+            s.max_entries = std::max(s.max_entries, running);
+        }
+    }
+    s.max_entries = std::max(s.max_entries, 2) + 16;   // + two batches of slack for the kernel's look-ahead (stays even)
+    ps_finish_smem(s);
+    if (s.smem_bytes > 220 * 1024) return false;
+    const size_t block_words = (size_t)s.block_bytes / 4;
+    h->ps_ent.assign(block_words * blocks.size(), 0u);
+    for (size_t b = 0; b < blocks.size(); ++b) std::copy(blocks[b].begin(), blocks[b].end(), h->ps_ent.begin() + b * block_words);
+    return true;
+}
+
+// default staged-planar schedule from the layer's shape
+void ps_default(const cadnn_layer_desc &d, int64_t nnz, PsSchedule &s)
+{
+    const int wp = d.in_w + 2 * kPlanarHalo;
+    const int range = d.in_h * wp;
+    const int batch = std::max(1, d.batch_hint);
+    s.T = (long long)range * batch >= 16L * 32 * kSmCount ? 8 : (long long)range * batch >= 2L * 32 * kSmCount ? 4 : range >= 512 ? 2 : 1;
+    s.NW = 8;
+    s.RPW = 2;
+    s.KS = 1;
+    const long long tiles = (long long)ceil_div(range, 32 * s.T) * batch;
+    while (s.KS < 8 && tiles * ceil_div(d.c_out, (s.NW / s.KS) * s.RPW) < 2L * kSmCount && nnz / std::max(1, d.c_out) / (2 * s.KS) >= 8) s.KS *= 2;
+    // the largest chunk whose two stages (tile + about its share of the nonzeros) fit 96 KB
+    const int A = round_up(d.pad * (wp + 1), 4), L = 32 * s.T + 2 * A;
+    s.CIc = d.c_in;
+    s.stages = 1;
+    const double per_ci = (double)L * 4 + 8.0 * 1.3 * (double)nnz / std::max(1, d.c_in) / std::max(1, ceil_div(d.c_out, (s.NW / s.KS) * s.RPW));
+    if (per_ci * d.c_in > 64.0 * 1024) {
+        s.stages = 2;
+        s.CIc = std::max(4, (int)(48.0 * 1024 / per_ci) & ~3);
+    }
+}
+
+template <class F>
+float time_launches(F launch, cudaStream_t st, int reps)
+{
+    if (launch() != CADNN_OK) return -1.0f;   // also raises the kernel's shared-memory limit outside the capture
+    if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return -1.0f; }
+    cudaGraph_t g = nullptr;
+    cudaGraphExec_t ge = nullptr;
+    float us = -1.0f;
+    if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { cudaGetLastError(); return -1.0f; }
+    bool ok = true;
+    for (int r = 0; r < reps && ok; ++r) ok = launch() == CADNN_OK;
+    if (cudaStreamEndCapture(st, &g) != cudaSuccess) ok = false;
+    if (ok && cudaGraphInstantiate(&ge, g, 0) == cudaSuccess) {
+        cudaEvent_t e0, e1;
+        cudaEventCreate(&e0);
+        cudaEventCreate(&e1);
+        cudaGraphLaunch(ge, st);
+        float best = 1e30f;
+        for (int rep = 0; rep < 2; ++rep) {
+            cudaEventRecord(e0, st);
+            cudaGraphLaunch(ge, st);
+            cudaEventRecord(e1, st);
+            if (cudaStreamSynchronize(st) == cudaSuccess) {
+                float ms = 0.0f;
+                cudaEventElapsedTime(&ms, e0, e1);
+                best = std::min(best, ms);
+            }
+        }
+        if (best < 1e29f) us = best * 1e3f / (float)reps;
+        cudaEventDestroy(e0);
+        cudaEventDestroy(e1);
+    }
+    if (ge) cudaGraphExecDestroy(ge);
+    if (g) cudaGraphDestroy(g);
+    cudaGetLastError();
+    return us;
+}
+
+// Time staged-planar schedules on the device and keep the fastest in h->ps (image not built here).
+void autotune_ps(cadnn_weights *h, const PsRows &rows, const std::vector<int64_t> &row_nnz)
+{
+    const cadnn_layer_desc &d = h->desc;
+    const int batch = std::max(1, d.batch_hint);
+    std::vector<PsSchedule> cands;
+    long long max_warps = 0;
+    const int range = d.in_h * (d.in_w + 2 * kPlanarHalo);   // computed positions of a plane, about
+    for (int T : {1, 2, 4, 8})
+        for (int nw : {4, 8, 16})
+            for (int ks : {1, 2, 4, 8})
+                for (int rpw : {1, 2, 4, 8})
+                    for (int div : {1, 2, 4, 8}) {
+                        PsSchedule s;
+                        s.T = T; s.NW = nw; s.KS = ks; s.RPW = rpw;
+                        s.CIc = round_up(ceil_div(d.c_in, div), 4);
+                        s.stages = div == 1 ? 1 : div >= 8 ? 3 : 2;
+                        if (ks > nw || rpw * T > 16 || (rpw == 8 && T > 1)) continue;
+                        if (div > 1 && ceil_div(d.c_in, s.CIc) < 2) continue;
+                        if (!ps_finish(d, s)) continue;
+                        if (T > 1 && 32 * (T / 2) >= range) continue;   // bands nobody needs
+                        if (s.G > d.c_out && rpw > 1) continue;
+                        // nonzeros spread evenly is the optimistic guess for the record size
+                        const double rec = s.hdr_bytes + 8.0 * (double)h->nnz / s.n_chunks / s.n_groups;
+                        if (s.stages * (s.tile_bytes + rec) > 220.0 * 1024) continue;
+                        cands.push_back(s);
+                        max_warps = std::max(max_warps, (long long)batch * s.tiles * s.n_groups * nw);
+                    }
+    const long long want = std::min<long long>(8L * kSmCount, max_warps) / 2;
+    const size_t xb = (size_t)batch * d.c_in * planar_pitch(d.in_h, d.in_w) * 4;
+    const size_t yb = (size_t)batch * d.c_out * planar_pitch(h->h_out, h->w_out) * 4;
+    void *x = nullptr, *y = nullptr;
+    cudaStream_t st = nullptr;
+    if (cudaMalloc(&x, xb) != cudaSuccess || cudaMalloc(&y, yb) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking) != cudaSuccess) {
+        if (x) cudaFree(x);
+        if (y) cudaFree(y);
+        cudaGetLastError();
+        return;
+    }
+    cudaMemsetAsync(x, 0, xb, st);
+    cudaMemsetAsync(y, 0, yb, st);
+    LaunchEpilogue ep;
+    ep.out_dtype = CADNN_F32;
+    ep.act = CADNN_ACT_RELU;
+    float best_us = -1.0f;
+    PsSchedule best = h->ps;
+    for (const PsSchedule &c : cands) {
+        const long long warps = (long long)batch * c.tiles * c.n_groups * c.NW;
+        if (warps < want || warps > 64L * kSmCount * 6) continue;
+        cadnn_weights tmp;
+        tmp.desc = d;
+        tmp.desc.flags &= ~CADNN_PACK_HOST_ONLY;
+        tmp.h_out = h->h_out;
+        tmp.w_out = h->w_out;
+        tmp.ps = c;
+        if (!build_ps_image(&tmp, rows, row_nnz)) continue;
+        if (upload(&tmp) != CADNN_OK) { if (tmp.d_blob) cudaFree(tmp.d_blob); continue; }
+        const float us = time_launches([&]() { return launch_sconv_planar_staged(&tmp, x, batch, y, ep, st); }, st, 8);
+        if (us > 0.0f && (best_us < 0.0f || us < best_us)) {
+            best_us = us;
+            best = tmp.ps;
+        }
+        cudaFree(tmp.d_blob);
+    }
+    cudaStreamDestroy(st);
+    cudaFree(x);
+    cudaFree(y);
+    cudaGetLastError();
+    if (best_us > 0.0f) {
+        h->ps = best;
+        h->ps_us = best_us;
+    }
+}
+
+void pack_ps(cadnn_weights *h, const Src &src, const std::vector<int64_t> &row_nnz)
+{
+    const cadnn_layer_desc &d = h->desc;
+    if (!ps_eligible(d, src.s8) || getenv("CADNN_NO_STAGED")) return;
+    PsRows rows;
+    ps_collect_rows(d, src, rows);
+    ps_default(d, h->nnz, h->ps);
+    if (!ps_finish(d, h->ps)) return;
+    if ((d.flags & CADNN_PACK_AUTOTUNE) && !(d.flags & CADNN_PACK_HOST_ONLY)) autotune_ps(h, rows, row_nnz);
+    ps_finish(d, h->ps);
+    for (int attempt = 0; attempt < 8; ++attempt) {
+        if (build_ps_image(h, rows, row_nnz)) {
+            h->has_ps = true;
+            h->use_ps = true;
+            return;
+        }
+        // a dense or skewed layer can overflow shared memory: halve the chunk and repack
+        if (h->ps.CIc <= 1) break;
+        h->ps.CIc = std::max(1, (h->ps.CIc / 2 + 3) & ~3);
+        h->ps.stages = 2;
+        if (!ps_finish(d, h->ps)) break;
+    }
+    h->ps_ent.clear();
+    h->ps_perm.clear();
 }
 
 cadnn_status pack_sconv(cadnn_weights *h, const Src &src)
@@ -680,6 +978,7 @@ cadnn_status pack_sconv(cadnn_weights *h, const Src &src)
     apply_env_override(g, linear, h->s);
     h->row_nnz = row_nnz;
     build_planar_image(h, src, row_nnz);
+    if (h->has_planar) pack_ps(h, src, row_nnz);
     return build_sconv_image(h, src, g, row_nnz);
 }
 
@@ -842,6 +1141,25 @@ cadnn_status cadnn_weights_schedule(const cadnn_weights *w, int sched[16])
     const Schedule &s = w->s;
     int v[16] = {s.kind, s.T, s.RPW, s.G, s.CIc, s.TH, s.TW, s.pitch, s.NW, s.stages, s.ksplit, s.n_chunks,
                  s.smem_bytes, s.TBX, s.TBY, s.max_entries};
+    memcpy(sched, v, sizeof(v));
+    return CADNN_OK;
+}
+
+cadnn_status cadnn_weights_planar_schedule(const cadnn_weights *w, int sched[16])
+{
+    if (!w || !sched) return CADNN_E_ARG;
+    int v[16] = {0};
+    if (w->has_ps && w->use_ps) {
+        const PsSchedule &s = w->ps;
+        int t[16] = {2, s.T, s.RPW, s.NW, s.KS, s.G, s.CIc, s.stages, s.n_chunks, s.tiles, s.smem_bytes, s.max_entries,
+                     (int)lrintf(w->ps_us * 100.0f), (int)lrintf(w->pl_us * 100.0f), 0, 0};
+        memcpy(v, t, sizeof(v));
+    } else if (w->has_planar) {
+        const int slots = std::max(1, w->pl_NW / std::max(1, w->pl_KSW));
+        int t[16] = {1, w->pl_T, w->pl_RPW, w->pl_NW, w->pl_KSW, slots * w->pl_RPW, w->desc.c_in, 0, 1, 0, 0, 0,
+                     (int)lrintf(w->ps_us * 100.0f), (int)lrintf(w->pl_us * 100.0f), 0, 0};
+        memcpy(v, t, sizeof(v));
+    }
     memcpy(sched, v, sizeof(v));
     return CADNN_OK;
 }

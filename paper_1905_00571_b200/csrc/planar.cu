@@ -45,7 +45,7 @@ __device__ __forceinline__ float pl_act(float z, int act)
 }
 
 template <int T>
-__global__ void __launch_bounds__(1024) sconv_planar_kernel(const PlanarParams p)
+__global__ void __launch_bounds__(512) sconv_planar_kernel(const PlanarParams p)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // block -> (image, pixel tile, filter group); groups vary fastest so that blocks running
@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(1024) sconv_planar_kernel(const PlanarParams p
 
     // KSW warps share a filter: each walks a slice of its nonzeros, slice 0 adds the partial sums
     // (through shared memory) and stores.  Few-pixel layers get their parallelism this way.
-    __shared__ float sRed[(T <= 2 ? 32 : T <= 4 ? 16 : 8)][T][32];   // as many warps as a block of this T may have
+    __shared__ float sRed[(T <= 4 ? 16 : 8)][T][32];   // as many warps as a block of this T may have
     const int KSW = 1 << p.ksw_shift;
     const int rslot = warp >> p.ksw_shift, slice = warp & (KSW - 1);
     for (int j = 0; j < p.RPW; ++j) {
@@ -89,19 +89,36 @@ __global__ void __launch_bounds__(1024) sconv_planar_kernel(const PlanarParams p
             const int rbeg = p.ptr[co] >> 1, rend = p.ptr[co + 1] >> 1;   // in pairs
             const int per = (rend - rbeg + KSW - 1) >> p.ksw_shift;
             const int beg = min(rend, rbeg + slice * per), end = min(rend, beg + per);
-            // every lane reads the same pair of nonzeros (one broadcast transaction), one pair ahead
-            uint4 nx = (beg < end) ? __ldg(p.ent + beg) : make_uint4(0, 0, 0, 0);
-#pragma unroll 2
-            for (int e = beg; e < end; ++e) {
-                const uint4 v = nx;
-                if (e + 1 < end) nx = __ldg(p.ent + e + 1);
-                const float w0 = __uint_as_float(v.x), w1 = __uint_as_float(v.z);
-                const float *a0 = ximg + v.y;
-                const float *a1 = ximg + v.w;
+            // Every lane reads the same pairs of nonzeros (broadcast transactions), one batch ahead.
+            // A batch issues all its activation loads before the first multiply-add: the loads are
+            // independent L1/L2 round trips and only their number in flight hides that latency.
+            // Slots past the end of the slice hold {0, offset 0}: they add nothing.
+            constexpr int P = T == 1 ? 8 : T == 2 ? 4 : T == 4 ? 2 : 1;   // pairs per batch
+            const uint4 zero4 = make_uint4(0, 0, 0, 0);
+            uint4 nx[P];
 #pragma unroll
-                for (int t = 0; t < T; ++t) acc[t] = fmaf(w0, __ldg(a0 + inb[t]), acc[t]);
+            for (int i = 0; i < P; ++i) nx[i] = (beg + i < end) ? __ldg(p.ent + beg + i) : zero4;
+            for (int e = beg; e < end; e += P) {
+                uint4 v[P];
 #pragma unroll
-                for (int t = 0; t < T; ++t) acc[t] = fmaf(w1, __ldg(a1 + inb[t]), acc[t]);
+                for (int i = 0; i < P; ++i) v[i] = nx[i];
+#pragma unroll
+                for (int i = 0; i < P; ++i) nx[i] = (e + P + i < end) ? __ldg(p.ent + e + P + i) : zero4;
+                float a[P][2][T];
+#pragma unroll
+                for (int i = 0; i < P; ++i)
+#pragma unroll
+                    for (int t = 0; t < T; ++t) {
+                        a[i][0][t] = __ldg(ximg + v[i].y + inb[t]);
+                        a[i][1][t] = __ldg(ximg + v[i].w + inb[t]);
+                    }
+#pragma unroll
+                for (int i = 0; i < P; ++i) {
+#pragma unroll
+                    for (int t = 0; t < T; ++t) acc[t] = fmaf(__uint_as_float(v[i].x), a[i][0][t], acc[t]);
+#pragma unroll
+                    for (int t = 0; t < T; ++t) acc[t] = fmaf(__uint_as_float(v[i].z), a[i][1][t], acc[t]);
+                }
             }
         }
         if (KSW > 1) {
@@ -196,12 +213,12 @@ cadnn_status launch_sconv_planar(const cadnn_weights *w, const void *x, int n, v
     p.ent = (const uint4 *)w->d_pl_ent; p.ptr = w->d_pl_ptr; p.order = w->d_pl_order;
     p.scale = ep.scale; p.bias = ep.bias; p.residual = (const float *)ep.residual;
     p.n = n; p.c_in = d.c_in; p.c_out = d.c_out;
-    p.wp_in = d.in_w + 2 * halo; p.plane_in = (d.in_h + 2 * halo) * p.wp_in;
+    p.wp_in = d.in_w + 2 * halo; p.plane_in = planar_pitch(d.in_h, d.in_w);
     p.h_out = w->h_out; p.w_out = w->w_out;
-    p.wp_out = w->w_out + 2 * halo; p.plane_out = (w->h_out + 2 * halo) * p.wp_out;
+    p.wp_out = w->w_out + 2 * halo; p.plane_out = planar_pitch(w->h_out, w->w_out);
     p.stride = d.stride; p.halo = halo; p.qtot = w->h_out * p.wp_out;
     const int T = w->pl_T;
-    if (w->pl_NW > (T <= 2 ? 32 : T <= 4 ? 16 : 8)) return CADNN_E_UNSUPPORTED;
+    if (w->pl_NW > (T <= 4 ? 16 : 8)) return CADNN_E_UNSUPPORTED;
     const int ksw = std::max(1, std::min(w->pl_KSW, w->pl_NW));
     p.ksw_shift = ksw >= 8 ? 3 : ksw >= 4 ? 2 : ksw >= 2 ? 1 : 0;
     p.G = (w->pl_NW >> p.ksw_shift) * w->pl_RPW; p.RPW = w->pl_RPW;
@@ -234,8 +251,7 @@ cadnn_status launch_maxpool_planar(const float *x, int n, int h, int wd, int c, 
     if (total >= (1LL << 31)) return CADNN_E_UNSUPPORTED;
     long long blocks = std::min((total + 255) / 256, 148LL * 32);
     return launch_kernel(maxpool_planar_kernel, (int)blocks, 256, 0, pdl, st, x, y, n * c, h, wd, wd + 2 * halo,
-                         (h + 2 * halo) * (wd + 2 * halo), h_out, w_out, w_out + 2 * halo,
-                         (h_out + 2 * halo) * (w_out + 2 * halo), halo, k, stride, pad, make_fastdiv(w_out),
+                         planar_pitch(h, wd), h_out, w_out, w_out + 2 * halo, planar_pitch(h_out, w_out), halo, k, stride, pad, make_fastdiv(w_out),
                          make_fastdiv(h_out));
 }
 
@@ -244,5 +260,5 @@ cadnn_status launch_gavgpool_planar(const float *x, int n, int h, int wd, int c,
     const int halo = kPlanarHalo;
     if (n * c <= 0) return CADNN_OK;
     return launch_kernel(gavgpool_planar_kernel, (n * c + 7) / 8, 256, 0, pdl, st, x, y, n * c, h, wd, wd + 2 * halo,
-                         (h + 2 * halo) * (wd + 2 * halo), halo, 1.0f / (float)(h * wd));
+                         planar_pitch(h, wd), halo, 1.0f / (float)(h * wd));
 }

@@ -187,11 +187,16 @@ def test_resnet50_full_batch1_with_timed_schedules():
     assert set(np.argsort(-got[0])[:5]) == set(np.argsort(-want[0])[:5])
 
 
+def _pitch(h, w):
+    return ((h + 2) * (w + 2) + 3) // 4 * 4
+
+
 def _to_planar(a):
-    """NHWC numpy -> [n, c, h+2, w+2] torch CUDA tensor with a zero border."""
+    """NHWC numpy -> [n, c, pitch] torch CUDA tensor: planes of (h+2) x (w+2) with a zero border, padded to a multiple of 4."""
     n, h, w, c = a.shape
-    t = torch.zeros((n, c, h + 2, w + 2), dtype=torch.float32, device=DEV)
-    t[:, :, 1:h + 1, 1:w + 1] = torch.from_numpy(np.ascontiguousarray(a.transpose(0, 3, 1, 2))).to(DEV)
+    t = torch.zeros((n, c, _pitch(h, w)), dtype=torch.float32, device=DEV)
+    t[:, :, :(h + 2) * (w + 2)].view(n, c, h + 2, w + 2)[:, :, 1:h + 1, 1:w + 1] = \
+        torch.from_numpy(np.ascontiguousarray(a.transpose(0, 3, 1, 2))).to(DEV)
     return t
 
 
@@ -200,13 +205,18 @@ PLANAR_CASES = [
     (1, 56, 56, 64, 64, 3, 1, 0.125), (2, 28, 28, 128, 128, 3, 2, 0.125), (1, 14, 14, 256, 200, 3, 1, 0.125),
     (3, 7, 7, 512, 96, 3, 1, 0.125), (1, 56, 56, 64, 256, 1, 1, 0.125), (2, 28, 28, 512, 130, 1, 2, 0.125),
     (1, 13, 17, 10, 7, 3, 1, 0.5), (1, 13, 17, 10, 7, 3, 2, 0.5), (1, 9, 9, 16, 16, 1, 1, 1.0), (1, 9, 9, 16, 16, 3, 1, 0.0),
+    (2, 7, 7, 2048, 512, 1, 1, 0.125), (1, 14, 14, 1024, 256, 1, 1, 0.05), (2, 5, 3, 6, 5, 3, 1, 1.0), (1, 28, 28, 130, 66, 3, 1, 0.3),
 ]
 
 
+@pytest.mark.parametrize("staged", [True, False])
 @pytest.mark.parametrize("case", PLANAR_CASES)
-def test_planar_sparse_conv(case):
+def test_planar_sparse_conv(case, staged):
+    """Both planar kernels: the shared-memory-staged one (stride 1) and the direct one (any stride)."""
     B = _B()
     n, h, w, c_in, c_out, k, stride, density = case
+    if staged and stride != 1:
+        pytest.skip("the staged kernel is stride 1 only; the direct kernel covers this case")
     pad = k // 2
     g = gen.rng(sum(case[:7]))
     x = gen.relu_normal_input(g, (n, h, w, c_in))
@@ -217,19 +227,25 @@ def test_planar_sparse_conv(case):
     res = gen.normal_input(g, (n, ho, wo, c_out))
     want = ref.conv2d_f32(x, wt, mask, stride, pad, 1, scale, bias, res, "relu")
     d = B.make_desc(c_in, c_out, k, k, stride, pad, 1, h, w, n, "f32", autotune=(c_in >= 256))
-    wh = B.cadnn_pack(d, wt, mask)
-    y = torch.zeros((n, c_out, ho + 2, wo + 2), device=DEV)
+    if not staged:
+        os.environ["CADNN_NO_STAGED"] = "1"
+    try:
+        wh = B.cadnn_pack(d, wt, mask)
+    finally:
+        os.environ.pop("CADNN_NO_STAGED", None)
+    y = torch.zeros((n, c_out, _pitch(ho, wo)), device=DEV)
     dev = lambda a: torch.from_numpy(a).to(DEV)
     B.cadnn_conv2d_planar(wh, _to_planar(x), y, dev(scale), dev(bias), _to_planar(res), "relu")
     torch.cuda.synchronize()
     yc = y.cpu().numpy()
-    got = yc[:, :, 1:ho + 1, 1:wo + 1].transpose(0, 2, 3, 1)
+    planes = yc[:, :, :(ho + 2) * (wo + 2)].reshape(n, c_out, ho + 2, wo + 2)
+    got = planes[:, :, 1:ho + 1, 1:wo + 1].transpose(0, 2, 3, 1)
     # the residual (|res| up to ~4) cancels against the conv result: a few ulps of the operands is the floor
     assert_close_f32(got, want, str(case), floor=NET_FLOOR)
-    # the border is never written
-    border = yc.copy()
+    # the border (and the padding behind a plane) is never written
+    border = planes.copy()
     border[:, :, 1:ho + 1, 1:wo + 1] = 0
-    assert not border.any()
+    assert not border.any() and not yc[:, :, (ho + 2) * (wo + 2):].any()
 
 
 def test_planar_and_nhwc_networks_agree_with_the_oracle():
