@@ -131,7 +131,8 @@ cadnn_status cadnn_weights_schedule(const cadnn_weights *w, int sched[16]);
  * a filter, filters per block, channel chunk, pipeline stages, channel chunks, tiles per
  * image, shared-memory bytes per block, entries per weight record, and the times measured
  * by CADNN_PACK_AUTOTUNE for the staged and the direct variant in hundredths of a
- * microsecond (negative = not measured); sched[14..15] = 0.  Host ints.
+ * microsecond (negative = not measured), 1 if the tile is staged by TMA copies (0: cp.async);
+ * sched[15] = 0.  Host ints.
  */
 cadnn_status cadnn_weights_planar_schedule(const cadnn_weights *w, int sched[16]);
 
@@ -306,6 +307,15 @@ cadnn_status cadnn_net_info(const cadnn_net *net, int *n_launches, int64_t *work
  */
 cadnn_status cadnn_net_layer_times(cadnn_net *net, const void *x, void *y, int flush_l2, int reps, float *ms,
                                    void *stream);
+
+/*
+ * cadnn_device_status - health flags the kernels leave on the current device (the paper has no
+ * counterpart: it exists because every wait inside a kernel is bounded).  *copy_timeouts
+ * receives how many thread-block waits on an asynchronous copy barrier ran out since the
+ * library was loaded; anything but 0 means results of that launch are invalid.  Synchronizes
+ * the device.  Errors: E_ARG, E_CUDA.
+ */
+cadnn_status cadnn_device_status(int *copy_timeouts);
 
 /* Device pointer and byte size of slot `slot` (for per-layer inspection). */
 cadnn_status cadnn_net_slot(const cadnn_net *net, int slot, void **ptr, int64_t *bytes);

@@ -69,6 +69,7 @@ _SIGS = {
     "cadnn_net_layer_times": (_i, [_vp, _vp, _vp, _i, _i, ctypes.POINTER(ctypes.c_float), _vp]),
     "cadnn_net_slot": (_i, [_vp, _i, ctypes.POINTER(_vp), _i64p]),
     "cadnn_net_free": (None, [_vp]),
+    "cadnn_device_status": (_i, [ctypes.POINTER(_i)]),
     "cadnn_status_str": (ctypes.c_char_p, [_i]),
     "cadnn_last_cuda_error": (ctypes.c_char_p, []),
 }
@@ -177,8 +178,14 @@ def cadnn_weights_planar_schedule(w):
     arr = (ctypes.c_int * 16)()
     _check(_lib.cadnn_weights_planar_schedule(w.handle, arr), "cadnn_weights_planar_schedule")
     keys = ("variant", "T", "RPW", "NW", "KS", "G", "CIc", "stages", "chunks", "tiles", "smem", "max_entries",
-            "staged_us_x100", "direct_us_x100")
+            "staged_us_x100", "direct_us_x100", "tma")
     return dict(zip(keys, list(arr)))
+
+
+def cadnn_device_status():
+    n = ctypes.c_int()
+    _check(_lib.cadnn_device_status(ctypes.byref(n)), "cadnn_device_status")
+    return {"copy_timeouts": n.value}
 
 
 def cadnn_weights_warp_loads(w):

@@ -109,6 +109,13 @@ cadnn_status cadnn_global_avgpool(const float *x, int n, int h, int wd, int c, f
     return launch_gavgpool(x, n, h, wd, c, y, false, (cudaStream_t)stream);
 }
 
+cadnn_status cadnn_device_status(int *copy_timeouts)
+{
+    if (!copy_timeouts) return CADNN_E_ARG;
+    CADNN_CUDA_TRY(cudaDeviceSynchronize());
+    return read_copy_timeouts(copy_timeouts);
+}
+
 const char *cadnn_status_str(cadnn_status s)
 {
     switch (s) {

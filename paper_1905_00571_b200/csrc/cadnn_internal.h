@@ -54,6 +54,8 @@ struct PsSchedule {
     int G = 8;        // filters per block = (NW / KS) * RPW
     int CIc = 0;      // input channels staged per chunk
     int stages = 1;
+    int tma = 0;      // 1: staged by TMA copies on mbarriers (stages may then cover all chunks), 0: cp.async by all threads
+    int RB = 0, nb = 0;          // TMA: channel rows per box (<= 256), boxes per chunk
     int n_chunks = 1, n_groups = 1;
     int A = 0, L = 32;           // staged margin / floats per channel
     int q_start = 0, tiles = 1;  // first computed position, tiles per image
@@ -148,6 +150,7 @@ cadnn_status launch_sconv_planar(const cadnn_weights *w, const void *x, int n, v
                                  cudaStream_t st);
 cadnn_status launch_sconv_planar_staged(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
                                         cudaStream_t st);
+cadnn_status read_copy_timeouts(int *count);
 cadnn_status launch_maxpool_planar(const float *x, int n, int h, int wd, int c, int k, int stride, int pad, float *y,
                                    bool pdl, cudaStream_t st);
 cadnn_status launch_gavgpool_planar(const float *x, int n, int h, int wd, int c, float *y, bool pdl, cudaStream_t st);

@@ -707,13 +707,19 @@ bool ps_finish(const cadnn_layer_desc &d, PsSchedule &s)
     s.n_groups = ceil_div(d.c_out, s.G);
     s.CIc = std::max(1, std::min(s.CIc, d.c_in));
     s.n_chunks = ceil_div(d.c_in, s.CIc);
-    s.stages = std::max(1, std::min(std::min(s.stages, 3), s.n_chunks));
+    s.stages = std::max(1, std::min(std::min(s.stages, s.tma ? 8 : 3), s.n_chunks));
     s.A = round_up(d.pad * (wp + 1), 4);
     s.L = 32 * s.T + 2 * s.A;
+    if (s.tma && s.L > 256) return false;   // a box is at most 256 elements wide
     s.q_start = (kPlanarHalo * (wp + 1)) & ~3;                         // first interior position, rounded down
     const int q_end = (d.in_h + kPlanarHalo - 1) * wp + d.in_w + kPlanarHalo;   // one past the last interior position
     s.tiles = ceil_div(q_end - s.q_start, 32 * s.T);
     s.tile_bytes = s.CIc * s.L * 4;
+    if (s.tma) {   // boxes of equal height (a multiple of 4 rows keeps every box 128-byte aligned in shared memory)
+        s.nb = ceil_div(s.CIc, 256);
+        s.RB = round_up(ceil_div(s.CIc, s.nb), 4);
+        s.tile_bytes = s.nb * s.RB * s.L * 4;
+    }
     s.hdr_bytes = round_up(s.G * s.KS + 1, 4) * 4;
     return true;
 }
@@ -722,8 +728,9 @@ void ps_finish_smem(PsSchedule &s)
 {
     s.block_bytes = s.hdr_bytes + s.max_entries * 8;
     s.stage_bytes = s.tile_bytes + s.block_bytes;
+    if (s.tma) s.stage_bytes = round_up(s.stage_bytes, 128);
     const int red = (s.NW / s.KS) * (s.KS - 1) * s.RPW * s.T * 128;   // partial sums of the warps that share filters
-    s.smem_bytes = std::max(s.stages * s.stage_bytes, red);
+    s.smem_bytes = std::max(s.stages * s.stage_bytes + (s.tma ? 8 * s.stages : 0), red);
 }
 
 // Image for schedule h->ps (through ps_finish): one fixed-size record per (chunk, filter block): a header
@@ -860,16 +867,25 @@ void autotune_ps(cadnn_weights *h, const PsRows &rows, const std::vector<int64_t
     const int batch = std::max(1, d.batch_hint);
     std::vector<PsSchedule> cands;
     long long max_warps = 0;
+    // ways of cutting the input channels into chunks: cp.async staging with 1-3 stages, TMA staging
+    // with every chunk in flight at once or a ring of half as many stages
+    static const int kStagingTab[][3] = {{1, 1, 0}, {2, 2, 0}, {4, 2, 0}, {8, 3, 0}, {1, 1, 1}, {2, 2, 1},
+                                         {4, 4, 1}, {8, 8, 1}, {4, 2, 1}, {8, 4, 1}, {16, 4, 1}};
+    std::vector<const int *> kStaging;
+    for (const auto &row : kStagingTab) kStaging.push_back(row);
     const int range = d.in_h * (d.in_w + 2 * kPlanarHalo);   // computed positions of a plane, about
     for (int T : {1, 2, 4, 8})
         for (int nw : {4, 8, 16})
             for (int ks : {1, 2, 4, 8})
                 for (int rpw : {1, 2, 4, 8})
-                    for (int div : {1, 2, 4, 8}) {
+                    for (const int *o : kStaging) {   // {chunks, stages, tma}
                         PsSchedule s;
                         s.T = T; s.NW = nw; s.KS = ks; s.RPW = rpw;
+                        const int div = o[0];
+                        s.tma = o[2];
                         s.CIc = round_up(ceil_div(d.c_in, div), 4);
-                        s.stages = div == 1 ? 1 : div >= 8 ? 3 : 2;
+                        s.stages = o[1];
+                        if (s.tma && getenv("CADNN_NO_TMA")) continue;
                         if (ks > nw || rpw * T > 16 || (rpw == 8 && T > 1)) continue;
                         if (div > 1 && ceil_div(d.c_in, s.CIc) < 2) continue;
                         if (!ps_finish(d, s)) continue;
@@ -1152,7 +1168,7 @@ cadnn_status cadnn_weights_planar_schedule(const cadnn_weights *w, int sched[16]
     if (w->has_ps && w->use_ps) {
         const PsSchedule &s = w->ps;
         int t[16] = {2, s.T, s.RPW, s.NW, s.KS, s.G, s.CIc, s.stages, s.n_chunks, s.tiles, s.smem_bytes, s.max_entries,
-                     (int)lrintf(w->ps_us * 100.0f), (int)lrintf(w->pl_us * 100.0f), 0, 0};
+                     (int)lrintf(w->ps_us * 100.0f), (int)lrintf(w->pl_us * 100.0f), s.tma, 0};
         memcpy(v, t, sizeof(v));
     } else if (w->has_planar) {
         const int slots = std::max(1, w->pl_NW / std::max(1, w->pl_KSW));

@@ -20,8 +20,27 @@
 //     inside the block, without a cluster;
 //   * lanes store their own positions (contiguous in the output plane) with the epilogue
 //     applied; border positions are computed but never stored, so the border stays zero.
+//
+// Two ways of staging: 16-byte cp.async copies issued by all threads, or (schedule flag tma) one
+// thread issuing TMA copies - a 2-D tensor copy per box of up to 256 channels x L floats of the
+// [n * c_in][pitch] view of x (out-of-range columns and rows are zero-filled by the unit) and a
+// bulk copy of the weight record - that complete on one mbarrier per stage, so the other
+// warps spend no issue slots on staging and several chunks are in flight from the first cycles.
 #include <algorithm>
+#include <cuda.h>
 #include "cadnn_internal.h"
+
+// set when a wait on a copy barrier ran out (never expected; the kernel then finishes with
+// whatever it has, and cadnn_device_status reports it)
+__device__ int g_copy_timeout;
+
+cadnn_status read_copy_timeouts(int *count)
+{
+    int v = 0;
+    CADNN_CUDA_TRY(cudaMemcpyFromSymbol(&v, g_copy_timeout, sizeof(int)));
+    *count = v;
+    return CADNN_OK;
+}
 
 namespace {
 
@@ -41,6 +60,7 @@ struct PsParams {
     int ks_shift;
     int tile_bytes, stage_bytes, hdr_bytes, block_bytes;
     int act;
+    int RB, nb, bar_off;   // TMA staging: rows per box, boxes per chunk, byte offset of the stage barriers
     FastDiv d_groups, d_tiles, d_wp, d_l4;
 };
 
@@ -84,6 +104,105 @@ __device__ __forceinline__ void ps_stage_acts(const PsParams &p, const float *xi
         const bool ok = ci < p.c_in && qa >= 0 && qa + 4 <= p.pitch;
         const float *src = ok ? ximg + (size_t)ci * p.pitch + qa : ximg;
         cp16(st32 + (unsigned)idx * 16u, src, ok);
+    }
+}
+
+// multiply-adds of one staged chunk for the filters of this warp
+template <int T, int RPW>
+__device__ __forceinline__ void ps_compute_chunk(const PsParams &p, const unsigned char *smem, unsigned stage_off, int lane,
+                                                 int rslot, int slice, float (&acc)[RPW][T])
+{
+    const int *sP = reinterpret_cast<const int *>(smem + stage_off + p.tile_bytes);
+    const unsigned sW = stage_off + p.tile_bytes + p.hdr_bytes;
+    const unsigned lanep = stage_off + lane * 4;
+#pragma unroll
+    for (int j = 0; j < RPW; ++j) {
+        const int seg = ((rslot * RPW + j) << p.ks_shift) + slice;
+        const int beg = sP[seg], end = sP[seg + 1];
+        // A batch of P pairs of nonzeros is read with broadcast loads one batch ahead; the batch's
+        // activation loads are all issued before its first multiply-add, so that a warp keeps
+        // 2 * P * T shared-memory loads in flight (with few warps per SM nothing else hides
+        // their latency).  Slots past the end of the segment get weight 0 (their offsets
+        // point inside the tile; the packer leaves two batches of slack behind a record).
+        constexpr int P = T == 1 ? 4 : T <= 4 ? 2 : 1;
+        uint4 nx[P];
+#pragma unroll
+        for (int i = 0; i < P; ++i) nx[i] = *reinterpret_cast<const uint4 *>(smem + sW + (beg + 2 * i) * 8);
+        for (int e = beg; e < end; e += 2 * P) {
+            uint4 v[P];
+#pragma unroll
+            for (int i = 0; i < P; ++i) {
+                v[i] = nx[i];
+                if (P > 1 && e + 2 * i >= end) v[i].x = v[i].z = 0u;
+            }
+#pragma unroll
+            for (int i = 0; i < P; ++i) nx[i] = *reinterpret_cast<const uint4 *>(smem + sW + (e + 2 * P + 2 * i) * 8);
+            float a[P][2][T];
+#pragma unroll
+            for (int i = 0; i < P; ++i)
+#pragma unroll
+                for (int t = 0; t < T; ++t) {
+                    a[i][0][t] = *reinterpret_cast<const float *>(smem + lanep + v[i].y + t * 128);
+                    a[i][1][t] = *reinterpret_cast<const float *>(smem + lanep + v[i].w + t * 128);
+                }
+#pragma unroll
+            for (int i = 0; i < P; ++i) {
+#pragma unroll
+                for (int t = 0; t < T; ++t) acc[j][t] = fmaf(__uint_as_float(v[i].x), a[i][0][t], acc[j][t]);
+#pragma unroll
+                for (int t = 0; t < T; ++t) acc[j][t] = fmaf(__uint_as_float(v[i].z), a[i][1][t], acc[j][t]);
+            }
+        }
+    }
+}
+
+// partial sums of the warps that share a filter, epilogue, stores
+template <int T, int RPW>
+__device__ __forceinline__ void ps_block_tail(const PsParams &p, unsigned char *smem, int lane, int rslot, int slice, int KS,
+                                              unsigned img, int q0, unsigned okmask, const int (&co_of)[RPW],
+                                              const float (&sc)[RPW], const float (&bi)[RPW], float (&acc)[RPW][T])
+{
+    // ---- warps that share a filter: partial sums meet in shared memory (the stages are free now) ----
+    if (KS > 1) {
+        __syncthreads();
+        float *sRed = reinterpret_cast<float *>(smem);
+        if (slice > 0) {
+            float *dst = sRed + (size_t)((rslot * (KS - 1) + slice - 1) * RPW) * T * 32 + lane;
+#pragma unroll
+            for (int j = 0; j < RPW; ++j)
+#pragma unroll
+                for (int t = 0; t < T; ++t) dst[(j * T + t) * 32] = acc[j][t];
+        }
+        __syncthreads();
+        if (slice == 0) {
+            for (int s2 = 1; s2 < KS; ++s2) {
+                const float *srcp = sRed + (size_t)((rslot * (KS - 1) + s2 - 1) * RPW) * T * 32 + lane;
+#pragma unroll
+                for (int j = 0; j < RPW; ++j)
+#pragma unroll
+                    for (int t = 0; t < T; ++t) acc[j][t] += srcp[(j * T + t) * 32];
+            }
+        }
+    }
+    grid_dep_trigger();
+
+    // ---- epilogue: every lane stores its own positions, contiguous in the output plane ----
+    if (slice == 0) {
+#pragma unroll
+        for (int j = 0; j < RPW; ++j) {
+            const int co = co_of[j];
+            if (co < 0) continue;
+            const size_t obase = ((size_t)img * p.c_out + co) * p.pitch + q0 + lane;
+#pragma unroll
+            for (int t = 0; t < T; ++t) {
+                if (okmask & (1u << t)) {
+                    const size_t oi = obase + 32 * t;
+                    float z = fmaf(acc[j][t], sc[j], bi[j]);
+                    if (p.residual) z += p.residual[oi];
+                    p.y[oi] = ps_act(z, p.act);
+                }
+            }
+        }
     }
 }
 
@@ -167,102 +286,150 @@ __global__ void __launch_bounds__(512) sconv_planar_staged_kernel(const PsParams
             }
             cp_commit();
         }
-        const unsigned stage_off = (unsigned)(buf * p.stage_bytes);
-        const int *sP = reinterpret_cast<const int *>(smem + stage_off + p.tile_bytes);
-        const unsigned sW = stage_off + p.tile_bytes + p.hdr_bytes;
-        const unsigned lanep = stage_off + lane * 4;
-#pragma unroll
-        for (int j = 0; j < RPW; ++j) {
-            const int seg = ((rslot * RPW + j) << p.ks_shift) + slice;
-            const int beg = sP[seg], end = sP[seg + 1];
-            // A batch of P pairs of nonzeros is read with broadcast loads one batch ahead; the batch's
-            // activation loads are all issued before its first multiply-add, so that a warp keeps
-            // 2 * P * T shared-memory loads in flight (with few warps per SM nothing else hides
-            // their latency).  Slots past the end of the segment get weight 0 (their offsets
-            // point inside the tile; the packer leaves two batches of slack behind a record).
-            constexpr int P = T == 1 ? 4 : T <= 4 ? 2 : 1;
-            uint4 nx[P];
-#pragma unroll
-            for (int i = 0; i < P; ++i) nx[i] = *reinterpret_cast<const uint4 *>(smem + sW + (beg + 2 * i) * 8);
-            for (int e = beg; e < end; e += 2 * P) {
-                uint4 v[P];
-#pragma unroll
-                for (int i = 0; i < P; ++i) {
-                    v[i] = nx[i];
-                    if (P > 1 && e + 2 * i >= end) v[i].x = v[i].z = 0u;
-                }
-#pragma unroll
-                for (int i = 0; i < P; ++i) nx[i] = *reinterpret_cast<const uint4 *>(smem + sW + (e + 2 * P + 2 * i) * 8);
-                float a[P][2][T];
-#pragma unroll
-                for (int i = 0; i < P; ++i)
-#pragma unroll
-                    for (int t = 0; t < T; ++t) {
-                        a[i][0][t] = *reinterpret_cast<const float *>(smem + lanep + v[i].y + t * 128);
-                        a[i][1][t] = *reinterpret_cast<const float *>(smem + lanep + v[i].w + t * 128);
-                    }
-#pragma unroll
-                for (int i = 0; i < P; ++i) {
-#pragma unroll
-                    for (int t = 0; t < T; ++t) acc[j][t] = fmaf(__uint_as_float(v[i].x), a[i][0][t], acc[j][t]);
-#pragma unroll
-                    for (int t = 0; t < T; ++t) acc[j][t] = fmaf(__uint_as_float(v[i].z), a[i][1][t], acc[j][t]);
-                }
-            }
-        }
+        ps_compute_chunk<T, RPW>(p, smem, (unsigned)(buf * p.stage_bytes), lane, rslot, slice, acc);
         if (++buf == S) buf = 0;
     }
     cp_wait<0>();
 
-    // ---- warps that share a filter: partial sums meet in shared memory (the stages are free now) ----
-    if (KS > 1) {
-        __syncthreads();
-        float *sRed = reinterpret_cast<float *>(smem);
-        if (slice > 0) {
-            float *dst = sRed + (size_t)((rslot * (KS - 1) + slice - 1) * RPW) * T * 32 + lane;
-#pragma unroll
-            for (int j = 0; j < RPW; ++j)
-#pragma unroll
-                for (int t = 0; t < T; ++t) dst[(j * T + t) * 32] = acc[j][t];
-        }
-        __syncthreads();
-        if (slice == 0) {
-            for (int s2 = 1; s2 < KS; ++s2) {
-                const float *srcp = sRed + (size_t)((rslot * (KS - 1) + s2 - 1) * RPW) * T * 32 + lane;
-#pragma unroll
-                for (int j = 0; j < RPW; ++j)
-#pragma unroll
-                    for (int t = 0; t < T; ++t) acc[j][t] += srcp[(j * T + t) * 32];
-            }
-        }
-    }
-    grid_dep_trigger();
+    ps_block_tail<T, RPW>(p, smem, lane, rslot, slice, KS, img, q0, okmask, co_of, sc, bi, acc);
+}
 
-    // ---- epilogue: every lane stores its own positions, contiguous in the output plane ----
-    if (slice == 0) {
-#pragma unroll
-        for (int j = 0; j < RPW; ++j) {
-            const int co = co_of[j];
-            if (co < 0) continue;
-            const size_t obase = ((size_t)img * p.c_out + co) * p.pitch + q0 + lane;
-#pragma unroll
-            for (int t = 0; t < T; ++t) {
-                if (okmask & (1u << t)) {
-                    const size_t oi = obase + 32 * t;
-                    float z = fmaf(acc[j][t], sc[j], bi[j]);
-                    if (p.residual) z += p.residual[oi];
-                    p.y[oi] = ps_act(z, p.act);
-                }
-            }
-        }
-    }
+
+// ---- TMA staging ----
+
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile("{\n.reg .pred q;\nmbarrier.try_wait.parity.shared::cta.b64 q, [%1], %2;\nselp.u32 %0, 1, 0, q;\n}\n"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Wait for a stage's copies.  The wait is bounded: if the barrier has not completed after
+// about a second the block records it and goes on (its results are then wrong, and the host
+// learns of it through the flag), after a second bounded wait that lets copies in flight land.
+__device__ __forceinline__ void mbar_wait(unsigned bar, unsigned parity)
+{
+    for (int it = 0; it < (1 << 22); ++it)
+        if (mbar_try_wait(bar, parity)) return;
+    atomicAdd(&g_copy_timeout, 1);
+    for (int it = 0; it < (1 << 22); ++it)
+        if (mbar_try_wait(bar, parity)) return;
+}
+__device__ __forceinline__ void bulk_copy(unsigned dst, const void *src, unsigned bytes, unsigned bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tensor_copy_2d(unsigned dst, const CUtensorMap *map, int x, int y, unsigned bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+// one thread: start the copies of chunk c into stage `buf`
+__device__ __forceinline__ void ps_tma_issue(const PsParams &p, const CUtensorMap *map, unsigned smem32, int buf, int c, int grp,
+                                             int row0, int xq)
+{
+    const unsigned bar = smem32 + p.bar_off + buf * 8;
+    const unsigned st32 = smem32 + (unsigned)(buf * p.stage_bytes);
+    mbar_expect_tx(bar, (unsigned)(p.tile_bytes + p.block_bytes));
+    const unsigned char *rec = reinterpret_cast<const unsigned char *>(p.ent) + ((size_t)c * p.n_groups + grp) * p.block_bytes;
+    bulk_copy(st32 + p.tile_bytes, rec, (unsigned)p.block_bytes, bar);
+    const unsigned box_bytes = (unsigned)(p.RB * p.L * 4);
+    for (int b = 0; b < p.nb; ++b) tensor_copy_2d(st32 + b * box_bytes, map, xq, row0 + c * p.CIc + b * p.RB, bar);
 }
 
 template <int T, int RPW>
-cadnn_status ps_launch_one(const PsParams &p, int blocks, int threads, int smem, bool pdl, cudaStream_t st)
+__global__ void __launch_bounds__(512) sconv_planar_tma_kernel(const PsParams p, const __grid_constant__ CUtensorMap tmap)
 {
+    extern __shared__ __align__(128) unsigned char smem[];
+    const unsigned smem32 = (unsigned)__cvta_generic_to_shared(smem);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    const unsigned r1 = fdiv(blockIdx.x, p.d_groups);
+    const int grp = (int)(blockIdx.x - r1 * p.n_groups);
+    const unsigned img = fdiv(r1, p.d_tiles);
+    const int tile = (int)(r1 - img * p.tiles);
+    const int q0 = p.q_start + tile * (32 * T);
+    const int S = p.stages;
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) mbar_init(smem32 + p.bar_off + s * 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    __syncthreads();
+    grid_dep_wait();   // x (and the residual) are final from here on
+    if (tid == 0) {
+        for (int s = 0; s < S && s < p.n_chunks; ++s) ps_tma_issue(p, &tmap, smem32, s, s, grp, (int)img * p.c_in, q0 - p.A);
+    }
+
+    const int KS = 1 << p.ks_shift;
+    const int rslot = warp >> p.ks_shift, slice = warp & (KS - 1);
+    unsigned okmask = 0;
+#pragma unroll
+    for (int t = 0; t < T; ++t) {
+        const int q = q0 + 32 * t + lane;
+        const int row = (int)fdiv((unsigned)q, p.d_wp);
+        const int col = q - row * p.wp;
+        if (row >= kPlanarHalo && row < kPlanarHalo + p.h && col >= kPlanarHalo && col < kPlanarHalo + p.w) okmask |= 1u << t;
+    }
+    int co_of[RPW];
+#pragma unroll
+    for (int j = 0; j < RPW; ++j) co_of[j] = p.perm[grp * p.G + rslot * RPW + j];
+    float acc[RPW][T];
+#pragma unroll
+    for (int j = 0; j < RPW; ++j)
+#pragma unroll
+        for (int t = 0; t < T; ++t) acc[j][t] = 0.0f;
+    float sc[RPW], bi[RPW];
+#pragma unroll
+    for (int j = 0; j < RPW; ++j) {
+        sc[j] = (p.scale && co_of[j] >= 0) ? p.scale[co_of[j]] : 1.0f;
+        bi[j] = (p.bias && co_of[j] >= 0) ? p.bias[co_of[j]] : 0.0f;
+    }
+
+    int buf = 0;
+    unsigned parity = 0;
+    for (int c = 0; c < p.n_chunks; ++c) {
+        mbar_wait(smem32 + p.bar_off + buf * 8, parity);
+        ps_compute_chunk<T, RPW>(p, smem, (unsigned)(buf * p.stage_bytes), lane, rslot, slice, acc);
+        if (c + S < p.n_chunks) {
+            __syncthreads();   // everyone is done with this stage
+            if (tid == 0) {
+                asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // reads above before the unit's writes
+                ps_tma_issue(p, &tmap, smem32, buf, c + S, grp, (int)img * p.c_in, q0 - p.A);
+            }
+        }
+        if (++buf == S) {
+            buf = 0;
+            parity ^= 1u;
+        }
+    }
+    ps_block_tail<T, RPW>(p, smem, lane, rslot, slice, KS, img, q0, okmask, co_of, sc, bi, acc);
+}
+
+template <int T, int RPW>
+cadnn_status ps_launch_one(const PsParams &p, const CUtensorMap *map, int blocks, int threads, int smem, bool pdl, cudaStream_t st)
+{
+    if (map) {
+        auto kern = sconv_planar_tma_kernel<T, RPW>;
+        static int smem_allowed = 48 * 1024;   // raised once per instantiation, as layers need it
+        if (smem > smem_allowed) {
+            CADNN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            smem_allowed = smem;
+        }
+        return launch_kernel(kern, blocks, threads, (size_t)smem, pdl, st, p, *map);
+    }
     auto kern = sconv_planar_staged_kernel<T, RPW>;
-    static int smem_allowed = 48 * 1024;   // raised once per instantiation, as layers need it
+    static int smem_allowed = 48 * 1024;
     if (smem > smem_allowed) {
         CADNN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         smem_allowed = smem;
@@ -271,15 +438,37 @@ cadnn_status ps_launch_one(const PsParams &p, int blocks, int threads, int smem,
 }
 
 template <int T>
-cadnn_status ps_launch_rpw(const PsParams &p, int rpw, int blocks, int threads, int smem, bool pdl, cudaStream_t st)
+cadnn_status ps_launch_rpw(const PsParams &p, const CUtensorMap *map, int rpw, int blocks, int threads, int smem, bool pdl,
+                           cudaStream_t st)
 {
     switch (rpw) {
-        case 1: return ps_launch_one<T, 1>(p, blocks, threads, smem, pdl, st);
-        case 2: return ps_launch_one<T, 2>(p, blocks, threads, smem, pdl, st);
-        case 4: return ps_launch_one<T, 4>(p, blocks, threads, smem, pdl, st);
-        case 8: if (T <= 4) return ps_launch_one<(T <= 4 ? T : 1), 8>(p, blocks, threads, smem, pdl, st); break;
+        case 1: return ps_launch_one<T, 1>(p, map, blocks, threads, smem, pdl, st);
+        case 2: return ps_launch_one<T, 2>(p, map, blocks, threads, smem, pdl, st);
+        case 4: return ps_launch_one<T, 4>(p, map, blocks, threads, smem, pdl, st);
+        case 8: if (T <= 4) return ps_launch_one<(T <= 4 ? T : 1), 8>(p, map, blocks, threads, smem, pdl, st); break;
     }
     return CADNN_E_UNSUPPORTED;
+}
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no link against the driver library)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)ptr;
+        else
+            cudaGetLastError();
+    }
+    return fn;
 }
 
 }  // namespace
@@ -309,11 +498,30 @@ cadnn_status launch_sconv_planar_staged(const cadnn_weights *w, const void *x, i
     if (blocks <= 0) return CADNN_OK;
     if (blocks > 2147483647LL) return CADNN_E_UNSUPPORTED;
     const int threads = s.NW * 32;
+    CUtensorMap map;
+    const CUtensorMap *mp = nullptr;
+    if (s.tma) {
+        // x as a matrix of n * c_in rows (planes) by pitch columns; a box is RB rows by L columns
+        EncodeTiledFn enc = encode_tiled_fn();
+        if (!enc) return CADNN_E_UNSUPPORTED;
+        const cuuint64_t dims[2] = {(cuuint64_t)p.pitch, (cuuint64_t)n * (cuuint64_t)d.c_in};
+        const cuuint64_t strides[1] = {(cuuint64_t)p.pitch * 4};
+        const cuuint32_t box[2] = {(cuuint32_t)s.L, (cuuint32_t)s.RB};
+        const cuuint32_t estr[2] = {1, 1};
+        if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(x), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return CADNN_E_UNSUPPORTED;
+        mp = &map;
+        p.RB = s.RB; p.nb = s.nb; p.bar_off = s.stages * s.stage_bytes;
+    } else {
+        p.RB = 0; p.nb = 0; p.bar_off = 0;
+    }
     switch (s.T) {
-        case 1: return ps_launch_rpw<1>(p, s.RPW, (int)blocks, threads, s.smem_bytes, ep.pdl, st);
-        case 2: return ps_launch_rpw<2>(p, s.RPW, (int)blocks, threads, s.smem_bytes, ep.pdl, st);
-        case 4: return ps_launch_rpw<4>(p, s.RPW, (int)blocks, threads, s.smem_bytes, ep.pdl, st);
-        case 8: return ps_launch_rpw<8>(p, s.RPW, (int)blocks, threads, s.smem_bytes, ep.pdl, st);
+        case 1: return ps_launch_rpw<1>(p, mp, s.RPW, (int)blocks, threads, s.smem_bytes, ep.pdl, st);
+        case 2: return ps_launch_rpw<2>(p, mp, s.RPW, (int)blocks, threads, s.smem_bytes, ep.pdl, st);
+        case 4: return ps_launch_rpw<4>(p, mp, s.RPW, (int)blocks, threads, s.smem_bytes, ep.pdl, st);
+        case 8: return ps_launch_rpw<8>(p, mp, s.RPW, (int)blocks, threads, s.smem_bytes, ep.pdl, st);
     }
     return CADNN_E_UNSUPPORTED;
 }
