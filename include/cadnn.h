@@ -131,8 +131,8 @@ cadnn_status cadnn_weights_schedule(const cadnn_weights *w, int sched[16]);
  * a filter, filters per block, channel chunk, pipeline stages, channel chunks, tiles per
  * image, shared-memory bytes per block, entries per weight record, and the times measured
  * by CADNN_PACK_AUTOTUNE for the staged and the direct variant in hundredths of a
- * microsecond (negative = not measured), 1 if the tile is staged by TMA copies (0: cp.async);
- * sched[15] = 0.  Host ints.
+ * microsecond (negative = not measured), 1 if the tile is staged by TMA copies (0: cp.async),
+ * blocks per cluster splitting the input channels.  Host ints.
  */
 cadnn_status cadnn_weights_planar_schedule(const cadnn_weights *w, int sched[16]);
 

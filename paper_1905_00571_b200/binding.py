@@ -178,7 +178,7 @@ def cadnn_weights_planar_schedule(w):
     arr = (ctypes.c_int * 16)()
     _check(_lib.cadnn_weights_planar_schedule(w.handle, arr), "cadnn_weights_planar_schedule")
     keys = ("variant", "T", "RPW", "NW", "KS", "G", "CIc", "stages", "chunks", "tiles", "smem", "max_entries",
-            "staged_us_x100", "direct_us_x100", "tma")
+            "staged_us_x100", "direct_us_x100", "tma", "KC")
     return dict(zip(keys, list(arr)))
 
 

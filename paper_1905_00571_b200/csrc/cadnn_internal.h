@@ -56,6 +56,8 @@ struct PsSchedule {
     int stages = 1;
     int tma = 0;      // 1: staged by TMA copies on mbarriers (stages may then cover all chunks), 0: cp.async by all threads
     int RB = 0, nb = 0;          // TMA: channel rows per box (<= 256), boxes per chunk
+    int KC = 1;                  // TMA: blocks per cluster splitting the channel chunks (partial sums meet in DSMEM)
+    int part_off = 0;            // byte offset of the cluster partial sums in shared memory
     int n_chunks = 1, n_groups = 1;
     int A = 0, L = 32;           // staged margin / floats per channel
     int q_start = 0, tiles = 1;  // first computed position, tiles per image
@@ -126,6 +128,7 @@ struct LaunchEpilogue {
     int act = 0;
     int out_dtype = 0;
     bool pdl = false;   // launch as a programmatic dependent of the previous kernel (inside cadnn_forward)
+    bool early_trigger = false;   // trigger dependents at kernel start instead of before the epilogue
     bool planar_out = false;   // dense stem: write the channel-planar layout instead of NHWC
 };
 

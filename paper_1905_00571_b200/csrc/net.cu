@@ -21,6 +21,8 @@ struct cadnn_net {
     std::vector<SlotInfo> slots;
     int out_slot = -1;
     bool use_pdl = true;   // layers after the first launch as programmatic dependents
+    bool pdl_graph = false;      // ... also inside captured graphs
+    bool early_trigger = false;
     bool planar = false;   // intermediate feature maps are channel-planar with a zero halo (planar.cu)
     int64_t workspace = 0;
     // graph cache: [0] caller's device pointers, [1] the net's own staging buffers
@@ -61,6 +63,7 @@ cadnn_status run_op(cadnn_net *net, const cadnn_op &op, const void *x, void *y, 
             le.act = op.act;
             le.out_dtype = CADNN_F32;
             le.pdl = pdl;
+            le.early_trigger = net->early_trigger;
             if (op.w->s.kind == KK_DENSE_SMALLC) {   // the stem reads the NHWC image and writes planes
                 le.planar_out = true;
                 return launch_dense_smallc(op.w, src, si.n, dst, le, st);
@@ -132,7 +135,7 @@ cadnn_status forward_impl(cadnn_net *net, const void *x, void *y, int use_graph,
         }
         cudaError_t e = cudaStreamBeginCapture(cap, cudaStreamCaptureModeThreadLocal);
         if (e != cudaSuccess) { if (own) cudaStreamDestroy(cap); return cadnn_note_cuda(e); }
-        s = run_all(net, x, y, cap);
+        s = run_all(net, x, y, cap, net->pdl_graph);
         e = cudaStreamEndCapture(cap, &gc.graph);
         if (own) cudaStreamDestroy(cap);
         if (s != CADNN_OK) { drop_graph(gc); return s; }
@@ -163,7 +166,9 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
     if (in_dtype != CADNN_F32 && in_dtype != CADNN_S8) return CADNN_E_DTYPE;
     cadnn_net *net = new (std::nothrow) cadnn_net();
     if (!net) return CADNN_E_ALLOC;
-    net->use_pdl = getenv("CADNN_NO_PDL") == nullptr;   // tuning switch: plain stream order between layers
+    net->use_pdl = getenv("CADNN_NO_PDL") == nullptr;
+    net->pdl_graph = getenv("CADNN_PDL_GRAPH") != nullptr;
+    net->early_trigger = getenv("CADNN_PDL_EARLY") != nullptr;   // tuning switch: plain stream order between layers
     cadnn_status st = CADNN_OK;
     int max_slot = 0;
     for (int i = 0; i < n_ops; ++i) {

@@ -707,7 +707,13 @@ bool ps_finish(const cadnn_layer_desc &d, PsSchedule &s)
     s.n_groups = ceil_div(d.c_out, s.G);
     s.CIc = std::max(1, std::min(s.CIc, d.c_in));
     s.n_chunks = ceil_div(d.c_in, s.CIc);
-    s.stages = std::max(1, std::min(std::min(s.stages, s.tma ? 8 : 3), s.n_chunks));
+    if (!s.tma) s.KC = 1;
+    if (s.KC > 1) {   // every block of a cluster takes the same number of chunks
+        s.n_chunks = round_up(s.n_chunks, s.KC);
+        s.CIc = round_up(ceil_div(d.c_in, s.n_chunks), 4);
+        if ((s.n_chunks - 1) * s.CIc >= d.c_in) return false;   // a rank would have nothing to do
+    }
+    s.stages = std::max(1, std::min(std::min(s.stages, s.tma ? 8 : 3), s.n_chunks / s.KC));
     s.A = round_up(d.pad * (wp + 1), 4);
     s.L = 32 * s.T + 2 * s.A;
     if (s.tma && s.L > 256) return false;   // a box is at most 256 elements wide
@@ -730,7 +736,9 @@ void ps_finish_smem(PsSchedule &s)
     s.stage_bytes = s.tile_bytes + s.block_bytes;
     if (s.tma) s.stage_bytes = round_up(s.stage_bytes, 128);
     const int red = (s.NW / s.KS) * (s.KS - 1) * s.RPW * s.T * 128;   // partial sums of the warps that share filters
-    s.smem_bytes = std::max(s.stages * s.stage_bytes + (s.tma ? 8 * s.stages : 0), red);
+    s.part_off = round_up(red, 128);
+    const int part = s.KC > 1 ? s.G * s.T * 128 : 0;                   // partial sums of the blocks of a cluster
+    s.smem_bytes = std::max(s.stages * s.stage_bytes + (s.tma ? 8 * s.stages : 0), s.part_off + part);
 }
 
 // Image for schedule h->ps (through ps_finish): one fixed-size record per (chunk, filter block): a header
@@ -865,37 +873,51 @@ void autotune_ps(cadnn_weights *h, const PsRows &rows, const std::vector<int64_t
 {
     const cadnn_layer_desc &d = h->desc;
     const int batch = std::max(1, d.batch_hint);
-    std::vector<PsSchedule> cands;
-    long long max_warps = 0;
-    // ways of cutting the input channels into chunks: cp.async staging with 1-3 stages, TMA staging
-    // with every chunk in flight at once or a ring of half as many stages
-    static const int kStagingTab[][3] = {{1, 1, 0}, {2, 2, 0}, {4, 2, 0}, {8, 3, 0}, {1, 1, 1}, {2, 2, 1},
-                                         {4, 4, 1}, {8, 8, 1}, {4, 2, 1}, {8, 4, 1}, {16, 4, 1}};
-    std::vector<const int *> kStaging;
-    for (const auto &row : kStagingTab) kStaging.push_back(row);
+    // ways of cutting the input channels into chunks {chunks, stages, tma}: cp.async staging with
+    // 1-3 stages; TMA staging with every chunk in flight at once, or a ring of fewer stages
+    static const int kStaging[][3] = {{4, 4, 1}, {8, 4, 1}, {16, 4, 1}, {4, 2, 0},   // defaults of the first pass, in order of preference
+                                      {1, 1, 1}, {2, 2, 1}, {8, 8, 1}, {4, 2, 1}, {1, 1, 0}, {2, 2, 0}, {8, 3, 0}};
+    const int kDefaults = 4, kAll = 11;
+    const bool no_tma = getenv("CADNN_NO_TMA") != nullptr;
+    const bool no_cluster = getenv("CADNN_NO_CLUSTER") != nullptr;
     const int range = d.in_h * (d.in_w + 2 * kPlanarHalo);   // computed positions of a plane, about
+    auto make = [&](int T, int nw, int ks, int rpw, int kc, const int *o, PsSchedule &s) {
+        s = PsSchedule();
+        s.T = T; s.NW = nw; s.KS = ks; s.RPW = rpw; s.KC = kc;
+        s.tma = o[2];
+        s.CIc = round_up(ceil_div(d.c_in, o[0] * kc), 4);
+        s.stages = o[1];
+        if ((s.tma && no_tma) || (kc > 1 && !s.tma)) return false;
+        if (o[0] * kc > 1 && ceil_div(d.c_in, s.CIc) < 2) return false;
+        if (!ps_finish(d, s)) return false;
+        // nonzeros spread evenly is the optimistic guess for the record size
+        const double rec = s.hdr_bytes + 8.0 * (double)h->nnz / s.n_chunks / s.n_groups;
+        return s.stages * (s.tile_bytes + rec) <= 216.0 * 1024;
+    };
+    // first pass: the launch shape (bands, warps, warps per filter, filters per warp) with a default staging
+    std::vector<PsSchedule> shapes;
+    long long max_warps = 0;
     for (int T : {1, 2, 4, 8})
         for (int nw : {4, 8, 16})
             for (int ks : {1, 2, 4, 8})
                 for (int rpw : {1, 2, 4, 8})
-                    for (const int *o : kStaging) {   // {chunks, stages, tma}
-                        PsSchedule s;
-                        s.T = T; s.NW = nw; s.KS = ks; s.RPW = rpw;
-                        const int div = o[0];
-                        s.tma = o[2];
-                        s.CIc = round_up(ceil_div(d.c_in, div), 4);
-                        s.stages = o[1];
-                        if (s.tma && getenv("CADNN_NO_TMA")) continue;
+                    for (int kc : {1, 2, 4, 8}) {
                         if (ks > nw || rpw * T > 16 || (rpw == 8 && T > 1)) continue;
-                        if (div > 1 && ceil_div(d.c_in, s.CIc) < 2) continue;
-                        if (!ps_finish(d, s)) continue;
                         if (T > 1 && 32 * (T / 2) >= range) continue;   // bands nobody needs
-                        if (s.G > d.c_out && rpw > 1) continue;
-                        // nonzeros spread evenly is the optimistic guess for the record size
-                        const double rec = s.hdr_bytes + 8.0 * (double)h->nnz / s.n_chunks / s.n_groups;
-                        if (s.stages * (s.tile_bytes + rec) > 220.0 * 1024) continue;
-                        cands.push_back(s);
-                        max_warps = std::max(max_warps, (long long)batch * s.tiles * s.n_groups * nw);
+                        if ((nw / ks) * rpw > d.c_out && rpw > 1) continue;
+                        // a cluster split pays when many filters per block share the staged activations
+                        if (kc > 1 && (no_cluster || d.c_in / kc < 64 || nw < 8 || ks > 2 || rpw < 2)) continue;
+                        PsSchedule s;
+                        bool ok = false;
+                        if (kc > 1) {
+                            static const int kc_staging[][3] = {{1, 1, 1}, {2, 2, 1}, {4, 2, 1}};
+                            for (int k = 0; k < 3 && !ok; ++k) ok = make(T, nw, ks, rpw, kc, kc_staging[k], s);
+                        } else {
+                            for (int k = 0; k < kDefaults && !ok; ++k) ok = make(T, nw, ks, rpw, 1, kStaging[k], s);
+                        }
+                        if (!ok) continue;
+                        shapes.push_back(s);
+                        max_warps = std::max(max_warps, (long long)batch * s.tiles * s.n_groups * nw * s.KC);
                     }
     const long long want = std::min<long long>(8L * kSmCount, max_warps) / 2;
     const size_t xb = (size_t)batch * d.c_in * planar_pitch(d.in_h, d.in_w) * 4;
@@ -914,34 +936,52 @@ void autotune_ps(cadnn_weights *h, const PsRows &rows, const std::vector<int64_t
     LaunchEpilogue ep;
     ep.out_dtype = CADNN_F32;
     ep.act = CADNN_ACT_RELU;
-    float best_us = -1.0f;
-    PsSchedule best = h->ps;
-    for (const PsSchedule &c : cands) {
-        const long long warps = (long long)batch * c.tiles * c.n_groups * c.NW;
-        if (warps < want || warps > 64L * kSmCount * 6) continue;
+    auto time_one = [&](const PsSchedule &c, PsSchedule &built) -> float {
         cadnn_weights tmp;
         tmp.desc = d;
         tmp.desc.flags &= ~CADNN_PACK_HOST_ONLY;
         tmp.h_out = h->h_out;
         tmp.w_out = h->w_out;
         tmp.ps = c;
-        if (!build_ps_image(&tmp, rows, row_nnz)) continue;
-        if (upload(&tmp) != CADNN_OK) { if (tmp.d_blob) cudaFree(tmp.d_blob); continue; }
+        if (!build_ps_image(&tmp, rows, row_nnz)) return -1.0f;
+        if (upload(&tmp) != CADNN_OK) { if (tmp.d_blob) cudaFree(tmp.d_blob); return -1.0f; }
         const float us = time_launches([&]() { return launch_sconv_planar_staged(&tmp, x, batch, y, ep, st); }, st, 8);
-        if (us > 0.0f && (best_us < 0.0f || us < best_us)) {
-            best_us = us;
-            best = tmp.ps;
-        }
+        built = tmp.ps;
         cudaFree(tmp.d_blob);
+        return us;
+    };
+    std::vector<std::pair<float, PsSchedule>> timed;
+    for (const PsSchedule &c : shapes) {
+        const long long warps = (long long)batch * c.tiles * c.n_groups * c.NW * c.KC;
+        if (warps < want || warps > 64L * kSmCount * 6) continue;
+        PsSchedule built;
+        const float us = time_one(c, built);
+        if (us > 0.0f) timed.push_back({us, built});
+    }
+    std::stable_sort(timed.begin(), timed.end(), [](const std::pair<float, PsSchedule> &a, const std::pair<float, PsSchedule> &b) { return a.first < b.first; });
+    // second pass: every staging for the best few shapes
+    const size_t keep = std::min<size_t>(timed.size(), 4);
+    for (size_t i = 0; i < keep; ++i) {
+        const PsSchedule base = timed[i].second;
+        for (int k = 0; k < kAll; ++k) {
+            PsSchedule s, built;
+            if (!make(base.T, base.NW, base.KS, base.RPW, base.KC, kStaging[k], s)) continue;
+            if (s.tma == base.tma && s.CIc == base.CIc && s.stages == base.stages) continue;
+            const float us = time_one(s, built);
+            if (us > 0.0f) timed.push_back({us, built});
+        }
     }
     cudaStreamDestroy(st);
     cudaFree(x);
     cudaFree(y);
     cudaGetLastError();
-    if (best_us > 0.0f) {
-        h->ps = best;
-        h->ps_us = best_us;
-    }
+    float best_us = -1.0f;
+    for (const auto &t : timed)
+        if (best_us < 0.0f || t.first < best_us) {
+            best_us = t.first;
+            h->ps = t.second;
+        }
+    if (best_us > 0.0f) h->ps_us = best_us;
 }
 
 void pack_ps(cadnn_weights *h, const Src &src, const std::vector<int64_t> &row_nnz)
@@ -952,7 +992,24 @@ void pack_ps(cadnn_weights *h, const Src &src, const std::vector<int64_t> &row_n
     ps_collect_rows(d, src, rows);
     ps_default(d, h->nnz, h->ps);
     if (!ps_finish(d, h->ps)) return;
-    if ((d.flags & CADNN_PACK_AUTOTUNE) && !(d.flags & CADNN_PACK_HOST_ONLY)) autotune_ps(h, rows, row_nnz);
+    const char *env = getenv("CADNN_PLANAR_SCHEDULE");   // tuning / test switch: "t=2,nw=16,ks=2,rpw=1,chunks=4,stages=2,tma=1,kc=2" (any subset)
+    if (env) {
+        PsSchedule s = h->ps;
+        int v, chunks = s.n_chunks;
+        const char *q;
+        if ((q = strstr(env, "t=")) && sscanf(q + 2, "%d", &v) == 1 && (v == 1 || v == 2 || v == 4 || v == 8)) s.T = v;
+        if ((q = strstr(env, "nw=")) && sscanf(q + 3, "%d", &v) == 1 && (v == 4 || v == 8 || v == 16)) s.NW = v;
+        if ((q = strstr(env, "ks=")) && sscanf(q + 3, "%d", &v) == 1 && (v == 1 || v == 2 || v == 4 || v == 8)) s.KS = v;
+        if ((q = strstr(env, "rpw=")) && sscanf(q + 4, "%d", &v) == 1 && (v == 1 || v == 2 || v == 4 || v == 8)) s.RPW = v;
+        if ((q = strstr(env, "kc=")) && sscanf(q + 3, "%d", &v) == 1 && (v == 1 || v == 2 || v == 4 || v == 8)) s.KC = v;
+        if ((q = strstr(env, "tma=")) && sscanf(q + 4, "%d", &v) == 1 && (v == 0 || v == 1)) s.tma = v;
+        if ((q = strstr(env, "chunks=")) && sscanf(q + 7, "%d", &v) == 1 && v >= 1 && v <= 64) chunks = v;
+        if ((q = strstr(env, "stages=")) && sscanf(q + 7, "%d", &v) == 1 && v >= 1 && v <= 8) s.stages = v;
+        s.CIc = round_up(ceil_div(d.c_in, chunks), 4);
+        if (s.RPW * s.T <= 16 && !(s.RPW == 8 && s.T > 4) && ps_finish(d, s)) h->ps = s;
+    } else if ((d.flags & CADNN_PACK_AUTOTUNE) && !(d.flags & CADNN_PACK_HOST_ONLY)) {
+        autotune_ps(h, rows, row_nnz);
+    }
     ps_finish(d, h->ps);
     for (int attempt = 0; attempt < 8; ++attempt) {
         if (build_ps_image(h, rows, row_nnz)) {
@@ -1168,7 +1225,7 @@ cadnn_status cadnn_weights_planar_schedule(const cadnn_weights *w, int sched[16]
     if (w->has_ps && w->use_ps) {
         const PsSchedule &s = w->ps;
         int t[16] = {2, s.T, s.RPW, s.NW, s.KS, s.G, s.CIc, s.stages, s.n_chunks, s.tiles, s.smem_bytes, s.max_entries,
-                     (int)lrintf(w->ps_us * 100.0f), (int)lrintf(w->pl_us * 100.0f), s.tma, 0};
+                     (int)lrintf(w->ps_us * 100.0f), (int)lrintf(w->pl_us * 100.0f), s.tma, s.KC};
         memcpy(v, t, sizeof(v));
     } else if (w->has_planar) {
         const int slots = std::max(1, w->pl_NW / std::max(1, w->pl_KSW));

@@ -60,6 +60,9 @@ struct PsParams {
     int ks_shift;
     int tile_bytes, stage_bytes, hdr_bytes, block_bytes;
     int act;
+    int kc_shift, chunks_per_rank;   // TMA kernel: log2 of the blocks per cluster that split the channel chunks; chunks each takes
+    int part_off;          // byte offset of the cluster partial sums in shared memory
+    int early_trigger;     // as a programmatic primary: let the next layer's prologue start at once
     int RB, nb, bar_off;   // TMA staging: rows per box, boxes per chunk, byte offset of the stage barriers
     FastDiv d_groups, d_tiles, d_wp, d_l4;
 };
@@ -105,6 +108,24 @@ __device__ __forceinline__ void ps_stage_acts(const PsParams &p, const float *xi
         const float *src = ok ? ximg + (size_t)ci * p.pitch + qa : ximg;
         cp16(st32 + (unsigned)idx * 16u, src, ok);
     }
+}
+
+// thread-block cluster helpers (all threads of all blocks of the cluster call cluster_sync)
+__device__ __forceinline__ void cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ unsigned map_shared_rank(unsigned addr, unsigned rank)
+{
+    unsigned r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float ld_shared_cluster(unsigned addr)
+{
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];\n" : "=f"(v) : "r"(addr) : "memory");
+    return v;
 }
 
 // multiply-adds of one staged chunk for the filters of this warp
@@ -160,7 +181,8 @@ __device__ __forceinline__ void ps_compute_chunk(const PsParams &p, const unsign
 template <int T, int RPW>
 __device__ __forceinline__ void ps_block_tail(const PsParams &p, unsigned char *smem, int lane, int rslot, int slice, int KS,
                                               unsigned img, int q0, unsigned okmask, const int (&co_of)[RPW],
-                                              const float (&sc)[RPW], const float (&bi)[RPW], float (&acc)[RPW][T])
+                                              const float (&sc)[RPW], const float (&bi)[RPW], float (&acc)[RPW][T],
+                                              int KC = 1, int rank = 0)
 {
     // ---- warps that share a filter: partial sums meet in shared memory (the stages are free now) ----
     if (KS > 1) {
@@ -184,14 +206,42 @@ __device__ __forceinline__ void ps_block_tail(const PsParams &p, unsigned char *
             }
         }
     }
-    grid_dep_trigger();
+    if (!p.early_trigger) grid_dep_trigger();
+
+    // ---- blocks of a cluster that split the input channels: every block leaves its partial sums in
+    // its shared memory; filter slot r is then finished by the block whose rank is r mod KC, which
+    // adds the other blocks' partial sums read over distributed shared memory ----
+    if (KC > 1) {
+        float *sPart = reinterpret_cast<float *>(smem + p.part_off);
+        __syncthreads();   // the stages are free: every warp has finished its multiply-adds
+        if (slice == 0) {
+#pragma unroll
+            for (int j = 0; j < RPW; ++j)
+#pragma unroll
+                for (int t = 0; t < T; ++t) sPart[((rslot * RPW + j) * T + t) * 32 + lane] = acc[j][t];
+        }
+        cluster_sync();   // every block's partial sums are in place
+        if (slice == 0) {
+            const unsigned mine = (unsigned)__cvta_generic_to_shared(sPart);
+#pragma unroll
+            for (int j = 0; j < RPW; ++j) {
+                const int slot = rslot * RPW + j;
+                if ((slot & (KC - 1)) != rank) continue;
+                for (int k = 1; k < KC; ++k) {
+                    const unsigned peer = map_shared_rank(mine + (unsigned)((slot * T) * 32 + lane) * 4u, (unsigned)((rank + k) & (KC - 1)));
+#pragma unroll
+                    for (int t = 0; t < T; ++t) acc[j][t] += ld_shared_cluster(peer + t * 128);
+                }
+            }
+        }
+    }
 
     // ---- epilogue: every lane stores its own positions, contiguous in the output plane ----
     if (slice == 0) {
 #pragma unroll
         for (int j = 0; j < RPW; ++j) {
             const int co = co_of[j];
-            if (co < 0) continue;
+            if (co < 0 || (KC > 1 && ((rslot * RPW + j) & (KC - 1)) != rank)) continue;
             const size_t obase = ((size_t)img * p.c_out + co) * p.pitch + q0 + lane;
 #pragma unroll
             for (int t = 0; t < T; ++t) {
@@ -204,6 +254,7 @@ __device__ __forceinline__ void ps_block_tail(const PsParams &p, unsigned char *
             }
         }
     }
+    if (KC > 1) cluster_sync();   // peers may still be reading this block's partial sums
 }
 
 template <int T, int RPW>
@@ -334,17 +385,24 @@ __device__ __forceinline__ void tensor_copy_2d(unsigned dst, const CUtensorMap *
                  ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 
-// one thread: start the copies of chunk c into stage `buf`
+// one thread: start the copies of chunk c into stage `buf`; the weight record first (it never
+// depends on the previous layer), the activation boxes after `before_acts` has run
+template <class F>
 __device__ __forceinline__ void ps_tma_issue(const PsParams &p, const CUtensorMap *map, unsigned smem32, int buf, int c, int grp,
-                                             int row0, int xq)
+                                             int row0, int xq, bool weights, bool acts, F before_acts)
 {
     const unsigned bar = smem32 + p.bar_off + buf * 8;
     const unsigned st32 = smem32 + (unsigned)(buf * p.stage_bytes);
-    mbar_expect_tx(bar, (unsigned)(p.tile_bytes + p.block_bytes));
-    const unsigned char *rec = reinterpret_cast<const unsigned char *>(p.ent) + ((size_t)c * p.n_groups + grp) * p.block_bytes;
-    bulk_copy(st32 + p.tile_bytes, rec, (unsigned)p.block_bytes, bar);
-    const unsigned box_bytes = (unsigned)(p.RB * p.L * 4);
-    for (int b = 0; b < p.nb; ++b) tensor_copy_2d(st32 + b * box_bytes, map, xq, row0 + c * p.CIc + b * p.RB, bar);
+    if (weights) {
+        mbar_expect_tx(bar, (unsigned)(p.tile_bytes + p.block_bytes));
+        const unsigned char *rec = reinterpret_cast<const unsigned char *>(p.ent) + ((size_t)c * p.n_groups + grp) * p.block_bytes;
+        bulk_copy(st32 + p.tile_bytes, rec, (unsigned)p.block_bytes, bar);
+    }
+    before_acts();
+    if (acts) {
+        const unsigned box_bytes = (unsigned)(p.RB * p.L * 4);
+        for (int b = 0; b < p.nb; ++b) tensor_copy_2d(st32 + b * box_bytes, map, xq, row0 + c * p.CIc + b * p.RB, bar);
+    }
 }
 
 template <int T, int RPW>
@@ -354,25 +412,34 @@ __global__ void __launch_bounds__(512) sconv_planar_tma_kernel(const PsParams p,
     const unsigned smem32 = (unsigned)__cvta_generic_to_shared(smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    const unsigned r1 = fdiv(blockIdx.x, p.d_groups);
-    const int grp = (int)(blockIdx.x - r1 * p.n_groups);
+    // consecutive blocks form a cluster: same tile and filters, consecutive ranges of the channel chunks
+    const int KC = 1 << p.kc_shift;
+    const int rank = (int)(blockIdx.x & (unsigned)(KC - 1));
+    const unsigned rest = blockIdx.x >> p.kc_shift;
+    const unsigned r1 = fdiv(rest, p.d_groups);
+    const int grp = (int)(rest - r1 * p.n_groups);
     const unsigned img = fdiv(r1, p.d_tiles);
     const int tile = (int)(r1 - img * p.tiles);
     const int q0 = p.q_start + tile * (32 * T);
     const int S = p.stages;
+    const int my_chunks = p.chunks_per_rank, c_first = rank * my_chunks;
+    const int npre = min(S, my_chunks);
 
+    // Everything up to the grid-dependency wait touches only constants of the layer, so as a
+    // programmatic dependent it overlaps the tail of the previous layer: barriers, the weight
+    // records of the first stages, the filter permutation and the epilogue vectors.
+    if (p.early_trigger) grid_dep_trigger();
     if (tid == 0) {
         for (int s = 0; s < S; ++s) mbar_init(smem32 + p.bar_off + s * 8, 1);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(&tmap) : "memory");
+        for (int s = 0; s < npre; ++s) ps_tma_issue(p, &tmap, smem32, s, c_first + s, grp, 0, 0, true, false, [] {});
     }
-    __syncthreads();
-    grid_dep_wait();   // x (and the residual) are final from here on
-    if (tid == 0) {
-        for (int s = 0; s < S && s < p.n_chunks; ++s) ps_tma_issue(p, &tmap, smem32, s, s, grp, (int)img * p.c_in, q0 - p.A);
-    }
-
     const int KS = 1 << p.ks_shift;
     const int rslot = warp >> p.ks_shift, slice = warp & (KS - 1);
+    int co_of[RPW];
+#pragma unroll
+    for (int j = 0; j < RPW; ++j) co_of[j] = p.perm[grp * p.G + rslot * RPW + j];
     unsigned okmask = 0;
 #pragma unroll
     for (int t = 0; t < T; ++t) {
@@ -381,31 +448,34 @@ __global__ void __launch_bounds__(512) sconv_planar_tma_kernel(const PsParams p,
         const int col = q - row * p.wp;
         if (row >= kPlanarHalo && row < kPlanarHalo + p.h && col >= kPlanarHalo && col < kPlanarHalo + p.w) okmask |= 1u << t;
     }
-    int co_of[RPW];
-#pragma unroll
-    for (int j = 0; j < RPW; ++j) co_of[j] = p.perm[grp * p.G + rslot * RPW + j];
     float acc[RPW][T];
 #pragma unroll
     for (int j = 0; j < RPW; ++j)
 #pragma unroll
         for (int t = 0; t < T; ++t) acc[j][t] = 0.0f;
+
+    grid_dep_wait();   // x (and the residual) are final from here on
+    if (tid == 0) {
+        for (int s = 0; s < npre; ++s) ps_tma_issue(p, &tmap, smem32, s, c_first + s, grp, (int)img * p.c_in, q0 - p.A, false, true, [] {});
+    }
     float sc[RPW], bi[RPW];
 #pragma unroll
     for (int j = 0; j < RPW; ++j) {
         sc[j] = (p.scale && co_of[j] >= 0) ? p.scale[co_of[j]] : 1.0f;
         bi[j] = (p.bias && co_of[j] >= 0) ? p.bias[co_of[j]] : 0.0f;
     }
+    __syncthreads();   // the barriers are initialised for everyone
 
     int buf = 0;
     unsigned parity = 0;
-    for (int c = 0; c < p.n_chunks; ++c) {
+    for (int c = 0; c < my_chunks; ++c) {
         mbar_wait(smem32 + p.bar_off + buf * 8, parity);
         ps_compute_chunk<T, RPW>(p, smem, (unsigned)(buf * p.stage_bytes), lane, rslot, slice, acc);
-        if (c + S < p.n_chunks) {
+        if (c + S < my_chunks) {
             __syncthreads();   // everyone is done with this stage
             if (tid == 0) {
                 asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // reads above before the unit's writes
-                ps_tma_issue(p, &tmap, smem32, buf, c + S, grp, (int)img * p.c_in, q0 - p.A);
+                ps_tma_issue(p, &tmap, smem32, buf, c_first + c + S, grp, (int)img * p.c_in, q0 - p.A, true, true, [] {});
             }
         }
         if (++buf == S) {
@@ -413,7 +483,7 @@ __global__ void __launch_bounds__(512) sconv_planar_tma_kernel(const PsParams p,
             parity ^= 1u;
         }
     }
-    ps_block_tail<T, RPW>(p, smem, lane, rslot, slice, KS, img, q0, okmask, co_of, sc, bi, acc);
+    ps_block_tail<T, RPW>(p, smem, lane, rslot, slice, KS, img, q0, okmask, co_of, sc, bi, acc, KC, rank);
 }
 
 template <int T, int RPW>
@@ -426,7 +496,29 @@ cadnn_status ps_launch_one(const PsParams &p, const CUtensorMap *map, int blocks
             CADNN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
             smem_allowed = smem;
         }
-        return launch_kernel(kern, blocks, threads, (size_t)smem, pdl, st, p, *map);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)blocks, 1, 1);
+        cfg.blockDim = dim3((unsigned)threads, 1, 1);
+        cfg.dynamicSmemBytes = (size_t)smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[2];
+        int na = 0;
+        if (p.kc_shift > 0) {
+            attr[na].id = cudaLaunchAttributeClusterDimension;
+            attr[na].val.clusterDim.x = 1u << p.kc_shift;
+            attr[na].val.clusterDim.y = 1;
+            attr[na].val.clusterDim.z = 1;
+            ++na;
+        }
+        if (pdl) {
+            attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[na].val.programmaticStreamSerializationAllowed = 1;
+            ++na;
+        }
+        cfg.attrs = attr;
+        cfg.numAttrs = (unsigned)na;
+        CADNN_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, p, *map));
+        return CADNN_OK;
     }
     auto kern = sconv_planar_staged_kernel<T, RPW>;
     static int smem_allowed = 48 * 1024;
@@ -490,11 +582,16 @@ cadnn_status launch_sconv_planar_staged(const cadnn_weights *w, const void *x, i
     p.ks_shift = s.KS >= 8 ? 3 : s.KS >= 4 ? 2 : s.KS >= 2 ? 1 : 0;
     p.tile_bytes = s.tile_bytes; p.stage_bytes = s.stage_bytes; p.hdr_bytes = s.hdr_bytes; p.block_bytes = s.block_bytes;
     p.act = ep.act;
+    p.early_trigger = ep.early_trigger ? 1 : 0;
     p.d_groups = make_fastdiv(s.n_groups);
     p.d_tiles = make_fastdiv(s.tiles);
     p.d_wp = make_fastdiv(p.wp);
     p.d_l4 = make_fastdiv(s.L >> 2);
-    const long long blocks = (long long)n * s.tiles * s.n_groups;
+    const int kc = s.tma ? std::max(1, s.KC) : 1;
+    p.kc_shift = kc >= 8 ? 3 : kc >= 4 ? 2 : kc >= 2 ? 1 : 0;
+    p.chunks_per_rank = s.n_chunks / kc;
+    p.part_off = s.part_off;
+    const long long blocks = (long long)n * s.tiles * s.n_groups * kc;
     if (blocks <= 0) return CADNN_OK;
     if (blocks > 2147483647LL) return CADNN_E_UNSUPPORTED;
     const int threads = s.NW * 32;

@@ -248,6 +248,58 @@ def test_planar_sparse_conv(case, staged):
     assert not border.any() and not yc[:, :, (ho + 2) * (wo + 2):].any()
 
 
+PLANAR_OVERRIDES = [
+    # (case, CADNN_PLANAR_SCHEDULE): cp.async and TMA staging, rings and all-in-flight, warps sharing a
+    # filter, clusters splitting the input channels (ragged last chunk included)
+    ((1, 14, 14, 256, 200, 3, 1, 0.125), "t=2,nw=16,ks=2,rpw=1,chunks=4,stages=2,tma=0"),
+    ((1, 14, 14, 256, 200, 3, 1, 0.125), "t=2,nw=16,ks=2,rpw=1,chunks=4,stages=2,tma=1"),
+    ((1, 14, 14, 256, 200, 3, 1, 0.125), "t=4,nw=8,ks=1,rpw=4,chunks=8,stages=8,tma=1"),
+    ((1, 14, 14, 256, 200, 3, 1, 0.125), "t=1,nw=16,ks=1,rpw=4,chunks=4,stages=1,tma=1,kc=4"),
+    ((1, 14, 14, 256, 200, 3, 1, 0.125), "t=2,nw=8,ks=2,rpw=2,chunks=8,stages=2,tma=1,kc=2"),
+    ((2, 7, 7, 2048, 512, 1, 1, 0.125), "t=1,nw=16,ks=1,rpw=8,chunks=8,stages=1,tma=1,kc=8"),
+    ((2, 7, 7, 2048, 512, 1, 1, 0.125), "t=2,nw=16,ks=2,rpw=2,chunks=16,stages=3,tma=1,kc=4"),
+    ((1, 28, 28, 130, 66, 3, 1, 0.3), "t=4,nw=8,ks=2,rpw=2,chunks=2,stages=1,tma=1,kc=2"),
+    ((1, 28, 28, 130, 66, 3, 1, 0.3), "t=8,nw=4,ks=4,rpw=1,chunks=3,stages=3,tma=0"),
+    ((1, 56, 56, 64, 256, 1, 1, 0.125), "t=8,nw=8,ks=1,rpw=2,chunks=1,stages=1,tma=1"),
+    ((3, 7, 7, 512, 96, 3, 1, 0.125), "t=1,nw=8,ks=8,rpw=1,chunks=4,stages=4,tma=1"),
+    ((1, 13, 17, 10, 7, 3, 1, 0.5), "t=1,nw=4,ks=2,rpw=2,chunks=2,stages=2,tma=1"),
+]
+
+
+@pytest.mark.parametrize("case,sched", PLANAR_OVERRIDES)
+def test_planar_staged_schedule_space(case, sched):
+    B = _B()
+    n, h, w, c_in, c_out, k, stride, density = case
+    pad = k // 2
+    g = gen.rng(sum(case[:7]) + 1)
+    x = gen.relu_normal_input(g, (n, h, w, c_in))
+    wt = gen.he_weights(g, c_out, k, k, c_in)
+    mask = gen.magnitude_mask(wt, density)
+    scale, bias = gen.folded_bn(g, c_out)
+    want = ref.conv2d_f32(x, wt, mask, stride, pad, 1, scale, bias, None, "relu")
+    d = B.make_desc(c_in, c_out, k, k, stride, pad, 1, h, w, n, "f32")
+    os.environ["CADNN_PLANAR_SCHEDULE"] = sched
+    try:
+        wh = B.cadnn_pack(d, wt, mask)
+    finally:
+        os.environ.pop("CADNN_PLANAR_SCHEDULE", None)
+    ps = B.cadnn_weights_planar_schedule(wh)
+    asked = dict(kv.split("=") for kv in sched.split(","))
+    assert ps["variant"] == 2 and ps["T"] == int(asked["t"]) and ps["NW"] == int(asked["nw"]) and ps["KS"] == int(asked["ks"])
+    assert ps["tma"] == int(asked["tma"]) and ps["KC"] == int(asked.get("kc", 1)) and ps["RPW"] == int(asked["rpw"])
+    y = torch.zeros((n, c_out, _pitch(h, w)), device=DEV)
+    dev = lambda a: torch.from_numpy(a).to(DEV)
+    B.cadnn_conv2d_planar(wh, _to_planar(x), y, dev(scale), dev(bias), None, "relu")
+    torch.cuda.synchronize()
+    planes = y.cpu().numpy()[:, :, :(h + 2) * (w + 2)].reshape(n, c_out, h + 2, w + 2)
+    # outputs that cancel to ~1e-3 of the operands' magnitude carry a few ulps of the operands: network floor
+    assert_close_f32(planes[:, :, 1:h + 1, 1:w + 1].transpose(0, 2, 3, 1), want, "%s %s" % (case, sched), floor=NET_FLOOR)
+    border = planes.copy()
+    border[:, :, 1:h + 1, 1:w + 1] = 0
+    assert not border.any()
+    assert B.cadnn_device_status()["copy_timeouts"] == 0
+
+
 def test_planar_and_nhwc_networks_agree_with_the_oracle():
     from oracle import forward as oracle_forward
     from paper_1905_00571_b200.network import PackedModel
