@@ -61,6 +61,7 @@ struct PsSchedule {
     int n_chunks = 1, n_groups = 1;
     int A = 0, L = 32;           // staged margin / floats per channel
     int q_start = 0, tiles = 1;  // first computed position, tiles per image
+    int R = 0;                   // row-tile mode (stride 2 layers): output rows per tile; 0 = linear mode
     int max_entries = 0;
     int hdr_bytes = 0, block_bytes = 0, tile_bytes = 0, stage_bytes = 0, smem_bytes = 0;
 };
@@ -106,6 +107,7 @@ struct cadnn_weights {
     bool use_ps = false;             // the network runner prefers it over the direct planar kernel
     PsSchedule ps;
     float ps_us = -1.0f, pl_us = -1.0f;   // measured time of the staged / direct planar kernel (autotune), microseconds
+    float nhwc_us = -1.0f;                // ... and of the NHWC kernel
     std::vector<uint32_t> ps_ent;
     std::vector<int32_t> ps_perm;    // packed row -> output channel, -1 = padding row
     const uint32_t *d_ps_ent = nullptr;

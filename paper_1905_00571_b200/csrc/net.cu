@@ -204,6 +204,20 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
                 if (op.src == 0 || flat[op.src]) planar = false;
             }
         }
+        // Where the packer timed both layouts for every sparse conv, the measured sums decide.
+        if (planar && getenv("CADNN_FORCE_PLANAR") == nullptr) {
+            double t_planar = 0.0, t_nhwc = 0.0;
+            bool all = true;
+            for (int i = 0; i < n_ops; ++i) {
+                const cadnn_weights *w = ops[i].kind == CADNN_OP_CONV ? ops[i].w : nullptr;
+                if (!w || !w->has_planar) continue;
+                const float tp = (w->has_ps && w->use_ps) ? w->ps_us : w->pl_us;
+                if (tp <= 0.0f || w->nhwc_us <= 0.0f) { all = false; break; }
+                t_planar += tp;
+                t_nhwc += w->nhwc_us;
+            }
+            if (all && t_nhwc > 0.0 && t_planar > t_nhwc) planar = false;
+        }
         net->planar = planar;
     }
     for (int i = 0; i < n_ops && st == CADNN_OK; ++i) {

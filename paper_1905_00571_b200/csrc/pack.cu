@@ -516,6 +516,7 @@ cadnn_status autotune_sconv(cadnn_weights *h, const Src &src, const Geometry &g,
     cudaFree(x);
     cudaFree(y);
     h->s = best;
+    h->nhwc_us = best_us;
     Geometry gg = g;
     bool linear = best.kind == KK_SCONV_LINEAR;
     finish_candidate(gg, h->s, linear);
@@ -654,7 +655,8 @@ void autotune_planar(cadnn_weights *h, const std::vector<int64_t> &row_nnz)
                 }
     h->pl_T = bT; h->pl_NW = bNW; h->pl_RPW = bRPW; h->pl_KSW = bKSW;
     h->pl_us = best_us;
-    if (h->has_ps && h->ps_us > 0.0f && best_us > 0.0f) h->use_ps = h->ps_us <= best_us || getenv("CADNN_FORCE_STAGED") != nullptr;
+    // the staged variant runs when it measured faster (an unmeasured one is not trusted against a measured one)
+    if (h->has_ps && best_us > 0.0f) h->use_ps = (h->ps_us > 0.0f && h->ps_us <= best_us) || getenv("CADNN_FORCE_STAGED") != nullptr;
     planar_order(h, row_nnz);
     cudaMemcpyAsync(d_order, h->pl_order.data(), h->pl_order.size() * 4, cudaMemcpyHostToDevice, st);
     cudaStreamSynchronize(st);
@@ -675,7 +677,7 @@ struct PsRows {
 
 bool ps_eligible(const cadnn_layer_desc &d, bool s8)
 {
-    if (s8 || d.groups != 1 || d.stride != 1 || d.kh != d.kw || 2 * d.pad != d.kh - 1 || d.pad > kPlanarHalo) return false;
+    if (s8 || d.groups != 1 || (d.stride != 1 && d.stride != 2) || d.kh != d.kw || 2 * d.pad != d.kh - 1 || d.pad > kPlanarHalo) return false;
     return (long long)planar_pitch(d.in_h, d.in_w) * d.c_in < (1LL << 31);
 }
 
@@ -714,12 +716,29 @@ bool ps_finish(const cadnn_layer_desc &d, PsSchedule &s)
         if ((s.n_chunks - 1) * s.CIc >= d.c_in) return false;   // a rank would have nothing to do
     }
     s.stages = std::max(1, std::min(std::min(s.stages, s.tma ? 8 : 3), s.n_chunks / s.KC));
-    s.A = round_up(d.pad * (wp + 1), 4);
-    s.L = 32 * s.T + 2 * s.A;
-    if (s.tma && s.L > 256) return false;   // a box is at most 256 elements wide
-    s.q_start = (kPlanarHalo * (wp + 1)) & ~3;                         // first interior position, rounded down
-    const int q_end = (d.in_h + kPlanarHalo - 1) * wp + d.in_w + kPlanarHalo;   // one past the last interior position
-    s.tiles = ceil_div(q_end - s.q_start, 32 * s.T);
+    if (d.stride == 1) {
+        s.R = 0;
+        s.A = round_up(d.pad * (wp + 1), 4);
+        s.L = 32 * s.T + 2 * s.A;
+        if (s.tma && s.L > 256) return false;   // a box is at most 256 elements wide
+        s.q_start = (kPlanarHalo * (wp + 1)) & ~3;                         // first interior position, rounded down
+        const int q_end = (d.in_h + kPlanarHalo - 1) * wp + d.in_w + kPlanarHalo;   // one past the last interior position
+        s.tiles = ceil_div(q_end - s.q_start, 32 * s.T);
+    } else {
+        // row tiles: as many output rows as fit the lanes' 32 T positions and a box of 256 input floats
+        if (!s.tma) return false;
+        const int h_out = (d.in_h + 2 * d.pad - d.kh) / d.stride + 1, w_out = (d.in_w + 2 * d.pad - d.kw) / d.stride + 1;
+        const int wp_out = w_out + 2 * kPlanarHalo;
+        int R = std::min(h_out, (32 * s.T) / wp_out);
+        while (R >= 1 && (d.stride * (R - 1) + d.kh) * wp + 3 > 256) --R;
+        if (R < 1) return false;
+        if (s.T > 1 && R * wp_out <= 32 * (s.T / 2)) return false;   // fewer bands would do
+        s.R = R;
+        s.A = d.pad * wp + kPlanarHalo;   // entry offsets count from the first tap of the tile's first position
+        s.L = round_up((d.stride * (R - 1) + d.kh) * wp + 3, 4);
+        s.q_start = 0;
+        s.tiles = ceil_div(h_out, R);
+    }
     s.tile_bytes = s.CIc * s.L * 4;
     if (s.tma) {   // boxes of equal height (a multiple of 4 rows keeps every box 128-byte aligned in shared memory)
         s.nb = ceil_div(s.CIc, 256);
@@ -887,7 +906,7 @@ void autotune_ps(cadnn_weights *h, const PsRows &rows, const std::vector<int64_t
         s.tma = o[2];
         s.CIc = round_up(ceil_div(d.c_in, o[0] * kc), 4);
         s.stages = o[1];
-        if ((s.tma && no_tma) || (kc > 1 && !s.tma)) return false;
+        if ((s.tma && no_tma) || ((kc > 1 || d.stride != 1) && !s.tma)) return false;
         if (o[0] * kc > 1 && ceil_div(d.c_in, s.CIc) < 2) return false;
         if (!ps_finish(d, s)) return false;
         // nonzeros spread evenly is the optimistic guess for the record size
@@ -945,7 +964,7 @@ void autotune_ps(cadnn_weights *h, const PsRows &rows, const std::vector<int64_t
         tmp.ps = c;
         if (!build_ps_image(&tmp, rows, row_nnz)) return -1.0f;
         if (upload(&tmp) != CADNN_OK) { if (tmp.d_blob) cudaFree(tmp.d_blob); return -1.0f; }
-        const float us = time_launches([&]() { return launch_sconv_planar_staged(&tmp, x, batch, y, ep, st); }, st, 8);
+        const float us = time_launches([&]() { return launch_sconv_planar_staged(&tmp, x, batch, y, ep, st); }, st, batch >= 16 ? 3 : 8);
         built = tmp.ps;
         cudaFree(tmp.d_blob);
         return us;
@@ -953,7 +972,7 @@ void autotune_ps(cadnn_weights *h, const PsRows &rows, const std::vector<int64_t
     std::vector<std::pair<float, PsSchedule>> timed;
     for (const PsSchedule &c : shapes) {
         const long long warps = (long long)batch * c.tiles * c.n_groups * c.NW * c.KC;
-        if (warps < want || warps > 64L * kSmCount * 6) continue;
+        if (warps < want) continue;
         PsSchedule built;
         const float us = time_one(c, built);
         if (us > 0.0f) timed.push_back({us, built});
@@ -991,6 +1010,11 @@ void pack_ps(cadnn_weights *h, const Src &src, const std::vector<int64_t> &row_n
     PsRows rows;
     ps_collect_rows(d, src, rows);
     ps_default(d, h->nnz, h->ps);
+    if (d.stride != 1) {   // row tiles are staged by TMA only
+        h->ps.tma = 1;
+        h->ps.T = std::min(h->ps.T, 2);
+        while (h->ps.T < 8 && !ps_finish(d, h->ps)) h->ps.T *= 2;
+    }
     if (!ps_finish(d, h->ps)) return;
     const char *env = getenv("CADNN_PLANAR_SCHEDULE");   // tuning / test switch: "t=2,nw=16,ks=2,rpw=1,chunks=4,stages=2,tma=1,kc=2" (any subset)
     if (env) {

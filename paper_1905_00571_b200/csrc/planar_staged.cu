@@ -53,7 +53,9 @@ struct PsParams {
     const float *bias;
     const float *residual;
     int c_in, c_out;
-    int h, w, wp, pitch;   // interior size, padded row length, floats between planes
+    int h, w, wp, pitch;   // input: interior size, padded row length, floats between planes
+    int h_out, w_out, wp_out, pitch_out;   // output (the same numbers at stride 1)
+    int stride, R, lead_rows;   // row-tile mode (R > 0): output rows per tile; first staged input row = stride * oy0 + lead_rows
     int q_start, tiles;    // first computed position (a multiple of 4), tiles of 32 * T positions per image
     int A, L;              // staged margin on either side and staged floats per channel (multiples of 4)
     int CIc, n_chunks, G, n_groups, stages;
@@ -64,7 +66,7 @@ struct PsParams {
     int part_off;          // byte offset of the cluster partial sums in shared memory
     int early_trigger;     // as a programmatic primary: let the next layer's prologue start at once
     int RB, nb, bar_off;   // TMA staging: rows per box, boxes per chunk, byte offset of the stage barriers
-    FastDiv d_groups, d_tiles, d_wp, d_l4;
+    FastDiv d_groups, d_tiles, d_wp, d_wp_out, d_l4;
 };
 
 __device__ __forceinline__ void cp16(unsigned dst, const void *src, bool pred)
@@ -129,9 +131,10 @@ __device__ __forceinline__ float ld_shared_cluster(unsigned addr)
 }
 
 // multiply-adds of one staged chunk for the filters of this warp
-template <int T, int RPW>
+// (ROWS: the lane's positions are not 32 t apart in the tile, their byte offsets come in lb[])
+template <int T, int RPW, bool ROWS = false>
 __device__ __forceinline__ void ps_compute_chunk(const PsParams &p, const unsigned char *smem, unsigned stage_off, int lane,
-                                                 int rslot, int slice, float (&acc)[RPW][T])
+                                                 int rslot, int slice, float (&acc)[RPW][T], const unsigned *lb = nullptr)
 {
     const int *sP = reinterpret_cast<const int *>(smem + stage_off + p.tile_bytes);
     const unsigned sW = stage_off + p.tile_bytes + p.hdr_bytes;
@@ -163,8 +166,13 @@ __device__ __forceinline__ void ps_compute_chunk(const PsParams &p, const unsign
             for (int i = 0; i < P; ++i)
 #pragma unroll
                 for (int t = 0; t < T; ++t) {
-                    a[i][0][t] = *reinterpret_cast<const float *>(smem + lanep + v[i].y + t * 128);
-                    a[i][1][t] = *reinterpret_cast<const float *>(smem + lanep + v[i].w + t * 128);
+                    if (ROWS) {
+                        a[i][0][t] = *reinterpret_cast<const float *>(smem + stage_off + lb[t] + v[i].y);
+                        a[i][1][t] = *reinterpret_cast<const float *>(smem + stage_off + lb[t] + v[i].w);
+                    } else {
+                        a[i][0][t] = *reinterpret_cast<const float *>(smem + lanep + v[i].y + t * 128);
+                        a[i][1][t] = *reinterpret_cast<const float *>(smem + lanep + v[i].w + t * 128);
+                    }
                 }
 #pragma unroll
             for (int i = 0; i < P; ++i) {
@@ -242,7 +250,7 @@ __device__ __forceinline__ void ps_block_tail(const PsParams &p, unsigned char *
         for (int j = 0; j < RPW; ++j) {
             const int co = co_of[j];
             if (co < 0 || (KC > 1 && ((rslot * RPW + j) & (KC - 1)) != rank)) continue;
-            const size_t obase = ((size_t)img * p.c_out + co) * p.pitch + q0 + lane;
+            const size_t obase = ((size_t)img * p.c_out + co) * p.pitch_out + q0 + lane;
 #pragma unroll
             for (int t = 0; t < T; ++t) {
                 if (okmask & (1u << t)) {
@@ -405,7 +413,7 @@ __device__ __forceinline__ void ps_tma_issue(const PsParams &p, const CUtensorMa
     }
 }
 
-template <int T, int RPW>
+template <int T, int RPW, bool ROWS>
 __global__ void __launch_bounds__(512) sconv_planar_tma_kernel(const PsParams p, const __grid_constant__ CUtensorMap tmap)
 {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -420,7 +428,16 @@ __global__ void __launch_bounds__(512) sconv_planar_tma_kernel(const PsParams p,
     const int grp = (int)(rest - r1 * p.n_groups);
     const unsigned img = fdiv(r1, p.d_tiles);
     const int tile = (int)(r1 - img * p.tiles);
-    const int q0 = p.q_start + tile * (32 * T);
+    // linear mode: 32 T consecutive positions of the (common) plane, staged with a margin of A on
+    // either side.  Row-tile mode (any stride): R output rows; the staged run starts at the input
+    // row of their first tap, rounded down to 16 bytes (`lead` floats of slack in front).
+    const int q0 = ROWS ? (kPlanarHalo + tile * p.R) * p.wp_out : p.q_start + tile * (32 * T);
+    int xq = q0 - p.A, lead = 0;
+    if (ROWS) {
+        const int run = (p.stride * tile * p.R + p.lead_rows) * p.wp;
+        xq = run & ~3;
+        lead = run - xq;
+    }
     const int S = p.stages;
     const int my_chunks = p.chunks_per_rank, c_first = rank * my_chunks;
     const int npre = min(S, my_chunks);
@@ -441,12 +458,21 @@ __global__ void __launch_bounds__(512) sconv_planar_tma_kernel(const PsParams p,
 #pragma unroll
     for (int j = 0; j < RPW; ++j) co_of[j] = p.perm[grp * p.G + rslot * RPW + j];
     unsigned okmask = 0;
+    unsigned lb[T];
 #pragma unroll
     for (int t = 0; t < T; ++t) {
         const int q = q0 + 32 * t + lane;
-        const int row = (int)fdiv((unsigned)q, p.d_wp);
-        const int col = q - row * p.wp;
-        if (row >= kPlanarHalo && row < kPlanarHalo + p.h && col >= kPlanarHalo && col < kPlanarHalo + p.w) okmask |= 1u << t;
+        const int row = (int)fdiv((unsigned)q, p.d_wp_out);
+        const int col = q - row * p.wp_out;
+        bool ok = row >= kPlanarHalo && row < kPlanarHalo + p.h_out && col >= kPlanarHalo && col < kPlanarHalo + p.w_out;
+        lb[t] = 0;
+        if (ROWS) {
+            const int ro = row - kPlanarHalo - tile * p.R;   // output row inside the tile
+            ok = ok && ro < p.R;
+            // lanes that store nothing still load: from the tile's first position
+            lb[t] = ok ? (unsigned)((p.stride * ro * p.wp + p.stride * (col - kPlanarHalo) + lead) * 4) : (unsigned)(lead * 4);
+        }
+        if (ok) okmask |= 1u << t;
     }
     float acc[RPW][T];
 #pragma unroll
@@ -456,7 +482,7 @@ __global__ void __launch_bounds__(512) sconv_planar_tma_kernel(const PsParams p,
 
     grid_dep_wait();   // x (and the residual) are final from here on
     if (tid == 0) {
-        for (int s = 0; s < npre; ++s) ps_tma_issue(p, &tmap, smem32, s, c_first + s, grp, (int)img * p.c_in, q0 - p.A, false, true, [] {});
+        for (int s = 0; s < npre; ++s) ps_tma_issue(p, &tmap, smem32, s, c_first + s, grp, (int)img * p.c_in, xq, false, true, [] {});
     }
     float sc[RPW], bi[RPW];
 #pragma unroll
@@ -470,12 +496,12 @@ __global__ void __launch_bounds__(512) sconv_planar_tma_kernel(const PsParams p,
     unsigned parity = 0;
     for (int c = 0; c < my_chunks; ++c) {
         mbar_wait(smem32 + p.bar_off + buf * 8, parity);
-        ps_compute_chunk<T, RPW>(p, smem, (unsigned)(buf * p.stage_bytes), lane, rslot, slice, acc);
+        ps_compute_chunk<T, RPW, ROWS>(p, smem, (unsigned)(buf * p.stage_bytes), lane, rslot, slice, acc, lb);
         if (c + S < my_chunks) {
             __syncthreads();   // everyone is done with this stage
             if (tid == 0) {
                 asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // reads above before the unit's writes
-                ps_tma_issue(p, &tmap, smem32, buf, c_first + c + S, grp, (int)img * p.c_in, q0 - p.A, true, true, [] {});
+                ps_tma_issue(p, &tmap, smem32, buf, c_first + c + S, grp, (int)img * p.c_in, xq, true, true, [] {});
             }
         }
         if (++buf == S) {
@@ -490,11 +516,12 @@ template <int T, int RPW>
 cadnn_status ps_launch_one(const PsParams &p, const CUtensorMap *map, int blocks, int threads, int smem, bool pdl, cudaStream_t st)
 {
     if (map) {
-        auto kern = sconv_planar_tma_kernel<T, RPW>;
-        static int smem_allowed = 48 * 1024;   // raised once per instantiation, as layers need it
-        if (smem > smem_allowed) {
+        auto kern = p.R > 0 ? sconv_planar_tma_kernel<T, RPW, true> : sconv_planar_tma_kernel<T, RPW, false>;
+        static int smem_allowed[2] = {48 * 1024, 48 * 1024};   // raised once per instantiation, as layers need it
+        int &allowed = smem_allowed[p.R > 0 ? 1 : 0];
+        if (smem > allowed) {
             CADNN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-            smem_allowed = smem;
+            allowed = smem;
         }
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)blocks, 1, 1);
@@ -576,6 +603,9 @@ cadnn_status launch_sconv_planar_staged(const cadnn_weights *w, const void *x, i
     p.scale = ep.scale; p.bias = ep.bias; p.residual = (const float *)ep.residual;
     p.c_in = d.c_in; p.c_out = d.c_out;
     p.h = d.in_h; p.w = d.in_w; p.wp = d.in_w + 2 * kPlanarHalo; p.pitch = planar_pitch(d.in_h, d.in_w);
+    p.h_out = w->h_out; p.w_out = w->w_out; p.wp_out = w->w_out + 2 * kPlanarHalo; p.pitch_out = planar_pitch(w->h_out, w->w_out);
+    p.stride = d.stride; p.R = s.R; p.lead_rows = kPlanarHalo - d.pad;
+    if (s.R > 0 && !s.tma) return CADNN_E_UNSUPPORTED;
     p.q_start = s.q_start; p.tiles = s.tiles;
     p.A = s.A; p.L = s.L;
     p.CIc = s.CIc; p.n_chunks = s.n_chunks; p.G = s.G; p.n_groups = s.n_groups; p.stages = s.stages;
@@ -586,6 +616,7 @@ cadnn_status launch_sconv_planar_staged(const cadnn_weights *w, const void *x, i
     p.d_groups = make_fastdiv(s.n_groups);
     p.d_tiles = make_fastdiv(s.tiles);
     p.d_wp = make_fastdiv(p.wp);
+    p.d_wp_out = make_fastdiv(p.wp_out);
     p.d_l4 = make_fastdiv(s.L >> 2);
     const int kc = s.tma ? std::max(1, s.KC) : 1;
     p.kc_shift = kc >= 8 ? 3 : kc >= 4 ? 2 : kc >= 2 ? 1 : 0;

@@ -212,11 +212,9 @@ PLANAR_CASES = [
 @pytest.mark.parametrize("staged", [True, False])
 @pytest.mark.parametrize("case", PLANAR_CASES)
 def test_planar_sparse_conv(case, staged):
-    """Both planar kernels: the shared-memory-staged one (stride 1) and the direct one (any stride)."""
+    """Both planar kernels: the shared-memory-staged one (linear tiles at stride 1, row tiles at stride 2) and the direct one."""
     B = _B()
     n, h, w, c_in, c_out, k, stride, density = case
-    if staged and stride != 1:
-        pytest.skip("the staged kernel is stride 1 only; the direct kernel covers this case")
     pad = k // 2
     g = gen.rng(sum(case[:7]))
     x = gen.relu_normal_input(g, (n, h, w, c_in))
@@ -263,6 +261,13 @@ PLANAR_OVERRIDES = [
     ((1, 56, 56, 64, 256, 1, 1, 0.125), "t=8,nw=8,ks=1,rpw=2,chunks=1,stages=1,tma=1"),
     ((3, 7, 7, 512, 96, 3, 1, 0.125), "t=1,nw=8,ks=8,rpw=1,chunks=4,stages=4,tma=1"),
     ((1, 13, 17, 10, 7, 3, 1, 0.5), "t=1,nw=4,ks=2,rpw=2,chunks=2,stages=2,tma=1"),
+    # stride 2: row tiles
+    ((2, 28, 28, 128, 128, 3, 2, 0.125), "t=2,nw=8,ks=2,rpw=2,chunks=2,stages=2,tma=1"),
+    ((2, 28, 28, 128, 128, 3, 2, 0.125), "t=1,nw=16,ks=1,rpw=4,chunks=4,stages=1,tma=1,kc=4"),
+    ((1, 56, 56, 256, 512, 1, 2, 0.125), "t=1,nw=16,ks=1,rpw=2,chunks=4,stages=2,tma=1"),
+    ((1, 14, 14, 512, 96, 3, 2, 0.125), "t=2,nw=16,ks=4,rpw=1,chunks=8,stages=2,tma=1,kc=2"),
+    ((1, 13, 17, 10, 7, 3, 2, 0.5), "t=4,nw=4,ks=1,rpw=1,chunks=1,stages=1,tma=1"),
+    ((2, 28, 28, 512, 130, 1, 2, 0.125), "t=2,nw=8,ks=1,rpw=2,chunks=2,stages=2,tma=1"),
 ]
 
 
@@ -277,6 +282,7 @@ def test_planar_staged_schedule_space(case, sched):
     mask = gen.magnitude_mask(wt, density)
     scale, bias = gen.folded_bn(g, c_out)
     want = ref.conv2d_f32(x, wt, mask, stride, pad, 1, scale, bias, None, "relu")
+    ho, wo = ref.out_hw(h, w, k, stride, pad)
     d = B.make_desc(c_in, c_out, k, k, stride, pad, 1, h, w, n, "f32")
     os.environ["CADNN_PLANAR_SCHEDULE"] = sched
     try:
@@ -287,15 +293,15 @@ def test_planar_staged_schedule_space(case, sched):
     asked = dict(kv.split("=") for kv in sched.split(","))
     assert ps["variant"] == 2 and ps["T"] == int(asked["t"]) and ps["NW"] == int(asked["nw"]) and ps["KS"] == int(asked["ks"])
     assert ps["tma"] == int(asked["tma"]) and ps["KC"] == int(asked.get("kc", 1)) and ps["RPW"] == int(asked["rpw"])
-    y = torch.zeros((n, c_out, _pitch(h, w)), device=DEV)
+    y = torch.zeros((n, c_out, _pitch(ho, wo)), device=DEV)
     dev = lambda a: torch.from_numpy(a).to(DEV)
     B.cadnn_conv2d_planar(wh, _to_planar(x), y, dev(scale), dev(bias), None, "relu")
     torch.cuda.synchronize()
-    planes = y.cpu().numpy()[:, :, :(h + 2) * (w + 2)].reshape(n, c_out, h + 2, w + 2)
+    planes = y.cpu().numpy()[:, :, :(ho + 2) * (wo + 2)].reshape(n, c_out, ho + 2, wo + 2)
     # outputs that cancel to ~1e-3 of the operands' magnitude carry a few ulps of the operands: network floor
-    assert_close_f32(planes[:, :, 1:h + 1, 1:w + 1].transpose(0, 2, 3, 1), want, "%s %s" % (case, sched), floor=NET_FLOOR)
+    assert_close_f32(planes[:, :, 1:ho + 1, 1:wo + 1].transpose(0, 2, 3, 1), want, "%s %s" % (case, sched), floor=NET_FLOOR)
     border = planes.copy()
-    border[:, :, 1:h + 1, 1:w + 1] = 0
+    border[:, :, 1:ho + 1, 1:wo + 1] = 0
     assert not border.any()
     assert B.cadnn_device_status()["copy_timeouts"] == 0
 
