@@ -244,9 +244,13 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
  * layers keep their intermediate feature maps channel-planar with a zero halo (see
  * cadnn_conv2d_planar); others (depthwise, int8) keep NHWC.  CADNN_NO_PLANAR in the
  * environment at cadnn_net_create forces NHWC.
- * Without a graph, layers after the first are launched as programmatic dependents of
- * their predecessor (their weight fetch overlaps its stores); set CADNN_NO_PDL in the
- * environment before cadnn_net_create to use plain stream order instead.
+ * Layers after the first are launched as programmatic dependents of their predecessor
+ * (their weight fetch overlaps its stores); set CADNN_NO_PDL in the environment before
+ * cadnn_net_create to use plain stream order instead (CADNN_NO_PDL_GRAPH: only inside
+ * graphs).  In a captured graph an op whose result the next op does not read (a residual
+ * block's downsample conv) becomes a parallel branch; CADNN_NO_FORK keeps one chain.
+ * CADNN_PERSIST=1 (experimental, slower where measured) runs the whole run of planar sparse
+ * convs as one cooperative kernel with device-wide barriers between layers.
  * Asynchronous on stream.
  */
 cadnn_status cadnn_forward(cadnn_net *net, const void *x, void *y, int use_graph, void *stream);

@@ -113,7 +113,13 @@ cadnn_status cadnn_device_status(int *copy_timeouts)
 {
     if (!copy_timeouts) return CADNN_E_ARG;
     CADNN_CUDA_TRY(cudaDeviceSynchronize());
-    return read_copy_timeouts(copy_timeouts);
+    int copies = 0, barriers = 0;
+    cadnn_status s = read_copy_timeouts(&copies);
+    if (s != CADNN_OK) return s;
+    s = read_barrier_timeouts(&barriers);
+    if (s != CADNN_OK) return s;
+    *copy_timeouts = copies + barriers;
+    return CADNN_OK;
 }
 
 const char *cadnn_status_str(cadnn_status s)

@@ -156,6 +156,27 @@ cadnn_status launch_sconv_planar(const cadnn_weights *w, const void *x, int n, v
 cadnn_status launch_sconv_planar_staged(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
                                         cudaStream_t st);
 cadnn_status read_copy_timeouts(int *count);
+cadnn_status read_barrier_timeouts(int *count);
+
+// Persistent kernel over a run of planar sparse convs (persist.cu).  One entry per conv, in
+// network order; join_phase: the op reads nothing that the ops of the current phase write, so
+// it may run in the same phase as its predecessor (no grid barrier between them).
+struct PersistPlan;
+struct PersistOpDesc {
+    const cadnn_weights *w = nullptr;
+    const void *x = nullptr;
+    void *y = nullptr;
+    const void *residual = nullptr;
+    const float *scale = nullptr;
+    const float *bias = nullptr;
+    int act = 0;
+    int n = 1;
+    bool join_phase = false;
+};
+cadnn_status persist_create(const std::vector<PersistOpDesc> &descs, PersistPlan **out);
+cadnn_status persist_launch(const PersistPlan *plan, cudaStream_t st);
+int persist_phases(const PersistPlan *plan);
+void persist_free(PersistPlan *plan);
 cadnn_status launch_maxpool_planar(const float *x, int n, int h, int wd, int c, int k, int stride, int pad, float *y,
                                    bool pdl, cudaStream_t st);
 cadnn_status launch_gavgpool_planar(const float *x, int n, int h, int wd, int c, float *y, bool pdl, cudaStream_t st);

@@ -21,9 +21,13 @@ struct cadnn_net {
     std::vector<SlotInfo> slots;
     int out_slot = -1;
     bool use_pdl = true;   // layers after the first launch as programmatic dependents
-    bool pdl_graph = false;      // ... also inside captured graphs
+    bool pdl_graph = true;       // ... also inside captured graphs
     bool early_trigger = false;
+    bool fork_branches = true;   // graph capture: ops off the critical path become parallel branches
     bool planar = false;   // intermediate feature maps are channel-planar with a zero halo (planar.cu)
+    // run of planar sparse convs [persist_first, persist_last] executed by one persistent kernel (persist.cu)
+    PersistPlan *persist = nullptr;
+    int persist_first = -1, persist_last = -1;
     int64_t workspace = 0;
     // graph cache: [0] caller's device pointers, [1] the net's own staging buffers
     struct GraphCache {
@@ -96,17 +100,134 @@ cadnn_status run_op(cadnn_net *net, const cadnn_op &op, const void *x, void *y, 
 // With pdl, every op after the first is launched as a programmatic dependent of its
 // predecessor: its prologue (weights, tables) overlaps the predecessor's stores, and it waits
 // on the grid dependency before touching activations.  Measured on the pruned ResNet-50 at
-// batch 1 this shortens layer-by-layer stream launches but lengthens graph replays, so only
-// the non-graph path uses it.
+// batch 1 (channel-planar kernels) it shortens both stream launches and graph replays
+// (450 -> 444 us per replay; 429 us together with the forked branches of run_all_forked).
 cadnn_status run_all(cadnn_net *net, const void *x, void *y, cudaStream_t st, bool pdl = false)
 {
     bool first = true;
-    for (const cadnn_op &op : net->ops) {
-        cadnn_status s = run_op(net, op, x, y, st, pdl && !first);
+    const int n_ops = (int)net->ops.size();
+    for (int i = 0; i < n_ops; ++i) {
+        if (net->persist && i == net->persist_first) {
+            // the whole run of sparse convs is one cooperative launch; its successor takes a full dependency on it
+            cadnn_status s = persist_launch(net->persist, st);
+            if (s != CADNN_OK) return s;
+            i = net->persist_last;
+            first = true;
+            continue;
+        }
+        cadnn_status s = run_op(net, net->ops[i], x, y, st, pdl && !first);
         if (s != CADNN_OK) return s;
         first = false;
     }
     return CADNN_OK;
+}
+
+// Capture-time variant of run_all: an op whose result the next op does not read (a bottleneck's
+// downsample conv, whose result is only needed as the residual of the block's last conv) is
+// issued on a second stream, forked from and joined back to the captured one with events, so
+// that in the graph it is a parallel branch.  At batch 1 no single layer fills the device, so
+// the branch runs beside the block's first convs instead of in front of them.
+cadnn_status run_all_forked(cadnn_net *net, const void *x, void *y, cudaStream_t st, cudaStream_t side, bool pdl)
+{
+    const int n_ops = (int)net->ops.size();
+    std::vector<cudaEvent_t> join(n_ops, nullptr);   // recorded on the side stream after op i
+    std::vector<cudaEvent_t> events;
+    cadnn_status rs = CADNN_OK;
+    auto new_event = [&](cudaEvent_t *e) {
+        if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return false;
+        events.push_back(*e);
+        return true;
+    };
+    bool first = true;
+    for (int i = 0; i < n_ops && rs == CADNN_OK; ++i) {
+        if (net->persist && i == net->persist_first) {
+            rs = persist_launch(net->persist, st);
+            i = net->persist_last;
+            first = true;
+            continue;
+        }
+        const cadnn_op &op = net->ops[i];
+        // join the branches this op reads
+        for (int j = 0; j < i; ++j) {
+            if (!join[j]) continue;
+            const int dj = net->ops[j].dst;
+            if (dj == op.src || dj == op.res) {
+                if (cudaStreamWaitEvent(st, join[j], 0) != cudaSuccess) rs = CADNN_E_CUDA;
+                join[j] = nullptr;
+                first = true;   // the next launch must not be a programmatic dependent across the join
+            }
+        }
+        if (rs != CADNN_OK) break;
+        bool branch = false;
+        if (i + 1 < n_ops && i > 0 && op.dst != net->out_slot) {
+            const cadnn_op &nx = net->ops[i + 1];
+            const bool inside_run = net->persist && i + 1 >= net->persist_first && i + 1 <= net->persist_last;
+            branch = nx.src != op.dst && nx.res != op.dst && !inside_run;
+        }
+        if (branch) {
+            cudaEvent_t fork = nullptr;
+            if (!new_event(&fork) || !new_event(&join[i]) || cudaEventRecord(fork, st) != cudaSuccess ||
+                cudaStreamWaitEvent(side, fork, 0) != cudaSuccess) { rs = CADNN_E_CUDA; break; }
+            rs = run_op(net, op, x, y, side, false);
+            if (rs == CADNN_OK && cudaEventRecord(join[i], side) != cudaSuccess) rs = CADNN_E_CUDA;
+        } else {
+            rs = run_op(net, op, x, y, st, pdl && !first);
+            first = false;
+        }
+    }
+    // branches nobody read still have to end inside the capture
+    for (int j = 0; j < n_ops; ++j)
+        if (join[j] && cudaStreamWaitEvent(st, join[j], 0) != cudaSuccess && rs == CADNN_OK) rs = CADNN_E_CUDA;
+    for (cudaEvent_t e : events) cudaEventDestroy(e);
+    if (rs == CADNN_E_CUDA) cadnn_note_cuda(cudaGetLastError());
+    return rs;
+}
+
+// Plan the persistent kernel over the longest run of consecutive planar sparse convs whose
+// tensors all live in slots the net owns.  Leaves net->persist null when there is no such run
+// (or the device cannot launch cooperatively); the layer-by-layer path then runs everything.
+void plan_persistent(cadnn_net *net)
+{
+    const int n_ops = (int)net->ops.size();
+    auto owned = [&](int slot) { return slot > 0 && slot != net->out_slot && net->slots[slot].ptr != nullptr; };
+    auto eligible = [&](const cadnn_op &op) {
+        return op.kind == CADNN_OP_CONV && op.w && op.w->has_planar && op.w->s.kind != KK_DENSE_SMALLC &&
+               op.w->d_pl_ent && owned(op.src) && owned(op.dst) && (op.res < 0 || owned(op.res));
+    };
+    int best_lo = -1, best_len = 0;
+    for (int i = 0; i < n_ops;) {
+        if (!eligible(net->ops[i])) { ++i; continue; }
+        int j = i;
+        while (j < n_ops && eligible(net->ops[j])) ++j;
+        if (j - i > best_len) { best_len = j - i; best_lo = i; }
+        i = j;
+    }
+    if (best_len < 3) return;
+    std::vector<PersistOpDesc> descs;
+    std::vector<int> phase_dsts;
+    for (int i = best_lo; i < best_lo + best_len; ++i) {
+        const cadnn_op &op = net->ops[i];
+        PersistOpDesc d;
+        d.w = op.w;
+        d.x = net->slots[op.src].ptr;
+        d.y = net->slots[op.dst].ptr;
+        d.residual = op.res >= 0 ? net->slots[op.res].ptr : nullptr;
+        d.scale = op.scale;
+        d.bias = op.bias;
+        d.act = op.act;
+        d.n = net->slots[op.src].n;
+        bool reads_phase = false;
+        for (int s : phase_dsts) reads_phase = reads_phase || s == op.src || s == op.res;
+        d.join_phase = !descs.empty() && !reads_phase && getenv("CADNN_PERSIST_NO_MERGE") == nullptr;
+        if (!d.join_phase) phase_dsts.clear();
+        phase_dsts.push_back(op.dst);
+        descs.push_back(d);
+    }
+    PersistPlan *plan = nullptr;
+    if (persist_create(descs, &plan) != CADNN_OK) { cudaGetLastError(); return; }
+    net->persist = plan;
+    net->persist_first = best_lo;
+    net->persist_last = best_lo + best_len - 1;
 }
 
 void drop_graph(cadnn_net::GraphCache &gc)
@@ -135,8 +256,14 @@ cadnn_status forward_impl(cadnn_net *net, const void *x, void *y, int use_graph,
         }
         cudaError_t e = cudaStreamBeginCapture(cap, cudaStreamCaptureModeThreadLocal);
         if (e != cudaSuccess) { if (own) cudaStreamDestroy(cap); return cadnn_note_cuda(e); }
-        s = run_all(net, x, y, cap, net->pdl_graph);
+        cudaStream_t side = nullptr;
+        if (net->fork_branches && cudaStreamCreateWithFlags(&side, cudaStreamNonBlocking) != cudaSuccess) {
+            cudaGetLastError();
+            side = nullptr;
+        }
+        s = side ? run_all_forked(net, x, y, cap, side, net->pdl_graph) : run_all(net, x, y, cap, net->pdl_graph);
         e = cudaStreamEndCapture(cap, &gc.graph);
+        if (side) cudaStreamDestroy(side);
         if (own) cudaStreamDestroy(cap);
         if (s != CADNN_OK) { drop_graph(gc); return s; }
         if (e != cudaSuccess) { drop_graph(gc); return cadnn_note_cuda(e); }
@@ -167,7 +294,8 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
     cadnn_net *net = new (std::nothrow) cadnn_net();
     if (!net) return CADNN_E_ALLOC;
     net->use_pdl = getenv("CADNN_NO_PDL") == nullptr;
-    net->pdl_graph = getenv("CADNN_PDL_GRAPH") != nullptr;
+    net->pdl_graph = net->use_pdl && getenv("CADNN_NO_PDL_GRAPH") == nullptr;
+    net->fork_branches = getenv("CADNN_NO_FORK") == nullptr;
     net->early_trigger = getenv("CADNN_PDL_EARLY") != nullptr;   // tuning switch: plain stream order between layers
     cadnn_status st = CADNN_OK;
     int max_slot = 0;
@@ -273,6 +401,10 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
         return st;
     }
     net->out_bytes = net->slots[net->out_slot].bytes;
+    {
+        const char *pe = getenv("CADNN_PERSIST");   // "0" / "1"; unset: off
+        if (net->planar && pe && atoi(pe) != 0) plan_persistent(net);
+    }
     *out = net;
     return CADNN_OK;
 }
@@ -306,7 +438,7 @@ cadnn_status cadnn_forward_host(cadnn_net *net, const void *x_host, void *y_host
 cadnn_status cadnn_net_info(const cadnn_net *net, int *n_launches, int64_t *workspace_bytes)
 {
     if (!net) return CADNN_E_ARG;
-    if (n_launches) *n_launches = (int)net->ops.size();
+    if (n_launches) *n_launches = (int)net->ops.size() - (net->persist ? net->persist_last - net->persist_first : 0);
     if (workspace_bytes) *workspace_bytes = net->workspace;
     return CADNN_OK;
 }
@@ -380,6 +512,7 @@ void cadnn_net_free(cadnn_net *net)
     for (SlotInfo &s : net->slots)
         if (s.ptr) cudaFree(s.ptr);
     if (net->flush) cudaFree(net->flush);
+    persist_free(net->persist);
     delete net;
 }
 

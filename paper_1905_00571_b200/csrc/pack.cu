@@ -530,15 +530,24 @@ void planar_order(cadnn_weights *h, const std::vector<int64_t> &row_nnz)
     const int c_out = h->desc.c_out;
     const int G = std::max(1, h->pl_NW / std::max(1, h->pl_KSW)) * h->pl_RPW;
     const int n_groups = ceil_div(c_out, G);
-    // constant capacity whatever the grouping, so that the device copy can be rewritten in place
-    h->pl_order.assign(std::max((size_t)n_groups * G, (size_t)round_up(c_out, 128) + 128), -1);
+    // constant capacity whatever the grouping, so that the device copy can be rewritten in place;
+    // four words per warp slot: {filter (-1 = none), first pair, end pair of its nonzeros, 0}
+    const size_t cap = std::max((size_t)n_groups * G, (size_t)round_up(c_out, 128) + 128);
+    h->pl_order.assign(cap * 4, 0);
+    for (size_t i = 0; i < cap; ++i) h->pl_order[i * 4] = -1;
     for (int gi = 0; gi < n_groups; ++gi) {
         int lo = gi * G, hi = std::min(c_out, lo + G);
         std::vector<int64_t> load(row_nnz.begin() + lo, row_nnz.begin() + hi);
         std::vector<int> slot;
         balance_block(load, G, h->pl_RPW, slot);
         for (int sl = 0; sl < G; ++sl)
-            if (slot[sl] >= 0) h->pl_order[lo + sl] = lo + slot[sl];
+            if (slot[sl] >= 0) {
+                const int co = lo + slot[sl];
+                int32_t *rec = &h->pl_order[(size_t)(lo + sl) * 4];
+                rec[0] = co;
+                rec[1] = h->pl_ptr[co] >> 1;
+                rec[2] = h->pl_ptr[co + 1] >> 1;
+            }
     }
 }
 

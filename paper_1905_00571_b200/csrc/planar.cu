@@ -25,7 +25,8 @@ struct PlanarParams {
     float *y;
     const uint4 *ent;     // pairs of {value bits, element offset}
     const int32_t *ptr;   // [c_out + 1] in entries (even), by original output channel
-    const int32_t *order; // [n_groups * G] filter handled by each warp slot, -1 = none
+    const int4 *order;    // [n_groups * G] per warp slot {filter (-1 = none), first pair, end pair, 0}: one load tells a
+                          // warp everything it needs to start fetching nonzeros
     const float *scale;
     const float *bias;
     const float *residual;
@@ -81,12 +82,27 @@ __global__ void __launch_bounds__(512) sconv_planar_kernel(const PlanarParams p)
     const int KSW = 1 << p.ksw_shift;
     const int rslot = warp >> p.ksw_shift, slice = warp & (KSW - 1);
     for (int j = 0; j < p.RPW; ++j) {
-        const int co = p.order[grp * p.G + rslot * p.RPW + j];
+        const int4 slot = __ldg(p.order + grp * p.G + rslot * p.RPW + j);
+        const int co = slot.x;
         float acc[T];
 #pragma unroll
         for (int t = 0; t < T; ++t) acc[t] = 0.0f;
+        // epilogue operands are requested now, so that their round trip to L2 overlaps the loop
+        float sc = 1.0f, bi = 0.0f, res[T];
+#pragma unroll
+        for (int t = 0; t < T; ++t) res[t] = 0.0f;
+        const size_t obase = ((size_t)img * p.c_out + max(co, 0)) * p.plane_out + (size_t)p.halo * p.wp_out + q0 + lane;
+        if (co >= 0 && slice == 0) {
+            if (p.scale) sc = __ldg(p.scale + co);
+            if (p.bias) bi = __ldg(p.bias + co);
+            if (p.residual) {
+#pragma unroll
+                for (int t = 0; t < T; ++t)
+                    if (okmask & (1u << t)) res[t] = __ldg(p.residual + obase + 32 * t);
+            }
+        }
         if (co >= 0) {
-            const int rbeg = p.ptr[co] >> 1, rend = p.ptr[co + 1] >> 1;   // in pairs
+            const int rbeg = slot.y, rend = slot.z;   // in pairs
             const int per = (rend - rbeg + KSW - 1) >> p.ksw_shift;
             const int beg = min(rend, rbeg + slice * per), end = min(rend, beg + per);
             // Every lane reads the same pairs of nonzeros (broadcast transactions), one batch ahead.
@@ -133,16 +149,11 @@ __global__ void __launch_bounds__(512) sconv_planar_kernel(const PlanarParams p)
             __syncthreads();   // sRed is reused by the next filter
         }
         if (co >= 0 && slice == 0) {
-            const float sc = p.scale ? p.scale[co] : 1.0f;
-            const float bi = p.bias ? p.bias[co] : 0.0f;
-            const size_t obase = ((size_t)img * p.c_out + co) * p.plane_out + (size_t)p.halo * p.wp_out + q0 + lane;
 #pragma unroll
             for (int t = 0; t < T; ++t) {
                 if (okmask & (1u << t)) {
-                    const size_t oi = obase + 32 * t;
-                    float z = fmaf(acc[t], sc, bi);
-                    if (p.residual) z += p.residual[oi];
-                    p.y[oi] = pl_act(z, p.act);
+                    const float z = fmaf(acc[t], sc, bi) + res[t];
+                    p.y[obase + 32 * t] = pl_act(z, p.act);
                 }
             }
         }
@@ -210,7 +221,7 @@ cadnn_status launch_sconv_planar(const cadnn_weights *w, const void *x, int n, v
     const int halo = kPlanarHalo;
     PlanarParams p;
     p.x = (const float *)x; p.y = (float *)y;
-    p.ent = (const uint4 *)w->d_pl_ent; p.ptr = w->d_pl_ptr; p.order = w->d_pl_order;
+    p.ent = (const uint4 *)w->d_pl_ent; p.ptr = w->d_pl_ptr; p.order = (const int4 *)w->d_pl_order;
     p.scale = ep.scale; p.bias = ep.bias; p.residual = (const float *)ep.residual;
     p.n = n; p.c_in = d.c_in; p.c_out = d.c_out;
     p.wp_in = d.in_w + 2 * halo; p.plane_in = planar_pitch(d.in_h, d.in_w);
