@@ -305,7 +305,7 @@ def run_ours(args):
                 "e2e": {"value": images / (e2e_ms * 1e-3), "unit": "images/s", "ms_per_step": e2e_ms,
                         "h2d_bytes_per_step": int(x_host.numel() * x_host.element_size()),
                         "d2h_bytes_per_step": int(y_host.numel() * y_host.element_size())},
-                "gpu_launches": K * n_ops, "clocks": clocks,
+                "gpu_launches": K * pm.launches_per_forward(), "clocks": clocks,
                 "paper_context": "26 ms (title) / 21 ms (text) ResNet-50 on a Snapdragon 835 / Adreno 540 phone"}
         print(json.dumps(line))
     dist.finalize()

@@ -128,7 +128,8 @@ cadnn_status cadnn_weights_schedule(const cadnn_weights *w, int sched[16]);
  * Schedule of the layer's channel-planar variant (the one cadnn_forward and
  * cadnn_conv2d_planar run): sched[0..13] = variant (0 none, 1 direct loads, 2 tile staged in
  * shared memory), position bands per lane, filters per warp, warps per block, warps sharing
- * a filter, filters per block, channel chunk, pipeline stages, channel chunks, tiles per
+ * a filter, filters per block, channel chunk, pipeline stages (direct variant: batch depth,
+ * 16 x depth activation loads in flight per lane), channel chunks, tiles per
  * image, shared-memory bytes per block, entries per weight record, and the times measured
  * by CADNN_PACK_AUTOTUNE for the staged and the direct variant in hundredths of a
  * microsecond (negative = not measured), 1 if the tile is staged by TMA copies (0: cp.async),
@@ -301,6 +302,14 @@ cadnn_status cadnn_forward_static(const cadnn_op *ops, int n_ops, int n, int h, 
 
 /* Number of kernel launches one forward issues; bytes of slot memory the net owns. */
 cadnn_status cadnn_net_info(const cadnn_net *net, int *n_launches, int64_t *workspace_bytes);
+
+/*
+ * How cadnn_forward runs this net: *planar = 1 if the intermediate feature maps are
+ * channel-planar (the planar kernels and schedules apply), 0 for NHWC; *persistent_ops =
+ * number of consecutive sparse convs executed by the one persistent kernel (0 = none).
+ * Either pointer may be NULL.  Host ints.
+ */
+cadnn_status cadnn_net_layout(const cadnn_net *net, int *planar, int *persistent_ops);
 
 /*
  * Measurement aid: time every op on its own.  Each op is captured into a CUDA graph of

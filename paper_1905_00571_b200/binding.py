@@ -66,6 +66,7 @@ _SIGS = {
     "cadnn_forward_host": (_i, [_vp, _vp, _vp, _i, _vp]),
     "cadnn_forward_static": (_i, [ctypes.POINTER(Op), _i, _i, _i, _i, _i, _i, _vp, _vp, _vp]),
     "cadnn_net_info": (_i, [_vp, ctypes.POINTER(_i), _i64p]),
+    "cadnn_net_layout": (_i, [_vp, ctypes.POINTER(_i), ctypes.POINTER(_i)]),
     "cadnn_net_layer_times": (_i, [_vp, _vp, _vp, _i, _i, ctypes.POINTER(ctypes.c_float), _vp]),
     "cadnn_net_slot": (_i, [_vp, _i, ctypes.POINTER(_vp), _i64p]),
     "cadnn_net_free": (None, [_vp]),
@@ -313,6 +314,12 @@ def cadnn_net_info(net):
     nl, ws = ctypes.c_int(), ctypes.c_int64()
     _check(_lib.cadnn_net_info(net.handle, ctypes.byref(nl), ctypes.byref(ws)), "cadnn_net_info")
     return {"launches": nl.value, "workspace_bytes": ws.value}
+
+
+def cadnn_net_layout(net):
+    pl, po = ctypes.c_int(), ctypes.c_int()
+    _check(_lib.cadnn_net_layout(net.handle, ctypes.byref(pl), ctypes.byref(po)), "cadnn_net_layout")
+    return {"planar": bool(pl.value), "persistent_ops": po.value}
 
 
 def cadnn_net_layer_times(net, x, y, n_ops, flush_l2=False, reps=1, stream=None):

@@ -98,6 +98,7 @@ struct cadnn_weights {
     std::vector<int32_t> pl_order;   // warp slot -> output channel (filters dealt to warps by load)
     std::vector<int64_t> row_nnz;    // stored nonzeros per output channel
     int pl_T = 2, pl_NW = 8, pl_RPW = 1, pl_KSW = 1;   // bands per lane, warps per block, filters per warp slot, warps per filter
+    int pl_D = 1;                                      // batch depth of the direct planar kernel (1, 2 or 4)
     const uint32_t *d_pl_ent = nullptr;
     const int32_t *d_pl_ptr = nullptr;
     const int32_t *d_pl_order = nullptr;

@@ -6,6 +6,7 @@
 // output and is bound by reading the input and writing the output once, so the
 // kernel maps lanes to channels (contiguous in NHWC) and keeps the filter taps in
 // the tap-major layout the packer wrote.
+#include <cstdlib>
 #include "cadnn_internal.h"
 
 namespace {
@@ -189,6 +190,163 @@ __global__ void __launch_bounds__(256) stem_kernel(const StemParams p)
     }
 }
 
+// asynchronous global -> shared copies (4 bytes with zero fill when !ok, 16 bytes)
+__device__ __forceinline__ void stem_cp4(unsigned dst, const float *src, bool ok)
+{
+    const int sz = ok ? 4 : 0;
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;\n" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void stem_cp16(unsigned dst, const float *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
+}
+
+// The same register tile specialised at compile time for the stems that occur (7x7x3 and 3x3x3 at
+// stride 2): a block is 4 warps (16 channels each) on ONE pair of output rows, so a 112 x 112 map
+// gives 224 blocks (the generic kernel's 112 leave a quarter of the SMs idle); the staged input
+// is split by channel and by column parity, so that lanes on consecutive output columns read
+// consecutive words whatever the tap (at stride 2 the interleaved layout is a 2-way bank
+// conflict); weights and input rows are copied without any division; the taps of one kernel
+// row are fully unrolled with constant offsets.
+template <int KH, int KW, int CIN>
+__global__ void __launch_bounds__(128) stem2_kernel(const StemParams p)
+{
+    constexpr int STRIDE = 2;
+    constexpr int IN_ROWS = STRIDE + KH;            // two output rows
+    constexpr int IN_COLS = 31 * STRIDE + KW;
+    constexpr int HALF = (IN_COLS + 1) / 2 + 1;     // words per (row, channel, parity); odd or even does not matter: lanes differ in the last index only
+    constexpr int ROW_WORDS = CIN * 2 * HALF;
+    constexpr int TAPS = KH * KW * CIN;
+    extern __shared__ __align__(16) float sm[];
+    float *sW = sm;                                  // [TAPS][64]
+    float *sIn = sm + TAPS * kStemCoBlock;           // [IN_ROWS][CIN][2][HALF]
+    const int tid = threadIdx.x, lane = tid & 31, wc = tid >> 5;
+    int b = blockIdx.x;
+    const int cb = b % p.co_blocks; b /= p.co_blocks;
+    const int tx = b % p.tiles_x; b /= p.tiles_x;
+    const int ty = b % p.tiles_y;
+    const int img = b / p.tiles_y;
+    const int ox0 = tx * 32, oy0 = ty * 2, co0 = cb * kStemCoBlock;
+
+    // Staging is all asynchronous copies: every request is in flight before the first one is
+    // waited for (a loop of load-then-store would pay one L2 round trip per iteration).
+    // Weights of this block's 64 channels first (static data: before the grid-dependency wait).
+    const unsigned sW32 = (unsigned)__cvta_generic_to_shared(sW), sIn32 = (unsigned)__cvta_generic_to_shared(sIn);
+    if ((p.c_out & 3) == 0 && co0 + kStemCoBlock <= p.c_out) {
+        for (int i = tid; i < TAPS * (kStemCoBlock / 4); i += 128) {
+            const int t = i >> 4, c4 = i & 15;
+            stem_cp16(sW32 + i * 16, p.wt + (size_t)t * p.c_out + co0 + c4 * 4);
+        }
+    } else {
+        for (int i = tid; i < TAPS * kStemCoBlock; i += 128) {
+            const int t = i >> 6, c = i & 63;
+            const bool ok = co0 + c < p.c_out;
+            stem_cp4(sW32 + i * 4, ok ? p.wt + (size_t)t * p.c_out + co0 + c : p.wt, ok);
+        }
+    }
+    grid_dep_wait();
+    grid_dep_trigger();
+    const int iy0 = oy0 * STRIDE - p.pad, ix0 = ox0 * STRIDE - p.pad;
+    // input rows: IN_COLS * CIN consecutive floats of the NHWC image each; warp r mod 4 takes row r
+    for (int r = wc; r < IN_ROWS; r += 4) {
+        const int iy = iy0 + r;
+        const bool row_ok = iy >= 0 && iy < p.h;
+        const float *src = p.x + (((size_t)img * p.h + (row_ok ? iy : 0)) * p.w) * CIN;
+        const unsigned dst = sIn32 + r * ROW_WORDS * 4;
+        int col = 0, ci = lane;      // element e = col * CIN + ci, starting at e = lane
+        while (ci >= CIN) { ci -= CIN; ++col; }
+#pragma unroll
+        for (int e0 = 0; e0 < IN_COLS * CIN; e0 += 32) {
+            if (e0 + lane < IN_COLS * CIN) {
+                const int ix = ix0 + col;
+                const bool ok = row_ok && ix >= 0 && ix < p.w;
+                stem_cp4(dst + ((ci * 2 + (col & 1)) * HALF + (col >> 1)) * 4, ok ? src + (size_t)ix * CIN + ci : p.x, ok);
+            }
+            ci += 32 % CIN;
+            col += 32 / CIN;
+            if (ci >= CIN) { ci -= CIN; ++col; }
+        }
+    }
+    asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
+    __syncthreads();
+
+    float acc0[kStemCo], acc1[kStemCo];
+#pragma unroll
+    for (int c = 0; c < kStemCo; ++c) acc0[c] = acc1[c] = 0.0f;
+    const float *w_base = sW + wc * kStemCo;
+    const float *in0 = sIn + lane;
+#pragma unroll 1
+    for (int ky = 0; ky < KH; ++ky) {
+        const float *r0 = in0 + ky * ROW_WORDS;
+        const float *r1 = r0 + STRIDE * ROW_WORDS;
+        const float *wk = w_base + ky * (KW * CIN) * kStemCoBlock;
+#pragma unroll
+        for (int kx = 0; kx < KW; ++kx)
+#pragma unroll
+            for (int ci = 0; ci < CIN; ++ci) {
+                const int off = (ci * 2 + (kx & 1)) * HALF + (kx >> 1);
+                const float a0 = r0[off], a1 = r1[off];
+                const float4 *wq = reinterpret_cast<const float4 *>(wk + (kx * CIN + ci) * kStemCoBlock);
+#pragma unroll
+                for (int q = 0; q < kStemCo / 4; ++q) {
+                    const float4 wv = wq[q];
+                    acc0[4 * q + 0] = fmaf(a0, wv.x, acc0[4 * q + 0]);
+                    acc0[4 * q + 1] = fmaf(a0, wv.y, acc0[4 * q + 1]);
+                    acc0[4 * q + 2] = fmaf(a0, wv.z, acc0[4 * q + 2]);
+                    acc0[4 * q + 3] = fmaf(a0, wv.w, acc0[4 * q + 3]);
+                    acc1[4 * q + 0] = fmaf(a1, wv.x, acc1[4 * q + 0]);
+                    acc1[4 * q + 1] = fmaf(a1, wv.y, acc1[4 * q + 1]);
+                    acc1[4 * q + 2] = fmaf(a1, wv.z, acc1[4 * q + 2]);
+                    acc1[4 * q + 3] = fmaf(a1, wv.w, acc1[4 * q + 3]);
+                }
+            }
+    }
+
+    const int ox = ox0 + lane;
+    const int cbase = co0 + wc * kStemCo;
+    if (ox < p.w_out) {
+#pragma unroll
+        for (int rr = 0; rr < 2; ++rr) {
+            const int oy = oy0 + rr;
+            if (oy >= p.h_out) continue;
+            const float *acc = rr ? acc1 : acc0;
+            const size_t o = (((size_t)img * p.h_out + oy) * p.w_out + ox) * p.c_out + cbase;
+            const int wp = p.w_out + 2 * p.halo;
+            const size_t plane = (size_t)planar_pitch(p.h_out, p.w_out);
+            const size_t opl = (size_t)img * p.c_out * plane + (size_t)(oy + p.halo) * wp + ox + p.halo;
+#pragma unroll
+            for (int c = 0; c < kStemCo; ++c) {
+                const int co = cbase + c;
+                if (co >= p.c_out) break;
+                float z = fmaf(acc[c], p.scale ? __ldg(p.scale + co) : 1.0f, p.bias ? __ldg(p.bias + co) : 0.0f);
+                if (p.planar_out) {
+                    p.y[opl + (size_t)co * plane] = dw_act(z, p.act);   // lanes are consecutive columns: contiguous
+                } else {
+                    if (p.residual) z += p.residual[o + c];
+                    p.y[o + c] = dw_act(z, p.act);
+                }
+            }
+        }
+    }
+}
+
+template <int KH, int KW, int CIN>
+cadnn_status launch_stem2(StemParams &p, int n, bool pdl, cudaStream_t st)
+{
+    constexpr int IN_ROWS = 2 + KH, IN_COLS = 31 * 2 + KW, HALF = (IN_COLS + 1) / 2 + 1;
+    p.tiles_y = (p.h_out + 1) / 2;
+    long long blocks = (long long)n * p.tiles_y * p.tiles_x * p.co_blocks;
+    if (blocks <= 0) return CADNN_OK;
+    if (blocks > 2147483647LL) return CADNN_E_UNSUPPORTED;
+    const size_t smem = ((size_t)KH * KW * CIN * kStemCoBlock + (size_t)IN_ROWS * CIN * 2 * HALF) * 4;
+    static bool raised = false;
+    if (!raised && smem > 48 * 1024) {
+        CADNN_CUDA_TRY(cudaFuncSetAttribute(stem2_kernel<KH, KW, CIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        raised = true;
+    }
+    return launch_kernel(stem2_kernel<KH, KW, CIN>, (int)blocks, 128, smem, pdl, st, p);
+}
+
 }  // namespace
 
 cadnn_status launch_dw(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
@@ -232,6 +390,10 @@ cadnn_status launch_dense_smallc(const cadnn_weights *w, const void *x, int n, v
     p.in_cols = 31 * d.stride + d.kw;
     p.taps = d.kh * d.kw * d.c_in;
     p.co_blocks = (d.c_out + kStemCoBlock - 1) / kStemCoBlock;
+    if (d.stride == 2 && d.c_in == 3 && getenv("CADNN_GENERIC_STEM") == nullptr) {
+        if (d.kh == 7 && d.kw == 7) return launch_stem2<7, 7, 3>(p, n, ep.pdl, st);
+        if (d.kh == 3 && d.kw == 3) return launch_stem2<3, 3, 3>(p, n, ep.pdl, st);
+    }
     long long blocks = (long long)n * p.tiles_y * p.tiles_x * p.co_blocks;
     if (blocks <= 0) return CADNN_OK;
     if (blocks > 2147483647LL) return CADNN_E_UNSUPPORTED;

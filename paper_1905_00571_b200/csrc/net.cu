@@ -443,6 +443,14 @@ cadnn_status cadnn_net_info(const cadnn_net *net, int *n_launches, int64_t *work
     return CADNN_OK;
 }
 
+cadnn_status cadnn_net_layout(const cadnn_net *net, int *planar, int *persistent_ops)
+{
+    if (!net) return CADNN_E_ARG;
+    if (planar) *planar = net->planar ? 1 : 0;
+    if (persistent_ops) *persistent_ops = net->persist ? net->persist_last - net->persist_first + 1 : 0;
+    return CADNN_OK;
+}
+
 cadnn_status cadnn_net_layer_times(cadnn_net *net, const void *x, void *y, int flush_l2, int reps, float *ms,
                                    void *stream)
 {

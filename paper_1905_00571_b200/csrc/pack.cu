@@ -621,16 +621,18 @@ void autotune_planar(cadnn_weights *h, const std::vector<int64_t> &row_nnz)
     int32_t *d_order = const_cast<int32_t *>(h->d_pl_order);
     const size_t order_cap = h->pl_order.size();   // device room reserved for the order array
     float best_us = -1.0f;
-    int bT = h->pl_T, bNW = h->pl_NW, bRPW = h->pl_RPW, bKSW = h->pl_KSW;
+    int bT = h->pl_T, bNW = h->pl_NW, bRPW = h->pl_RPW, bKSW = h->pl_KSW, bD = h->pl_D;
     LaunchEpilogue ep;
     ep.out_dtype = CADNN_F32;
     ep.act = CADNN_ACT_RELU;
     for (int T : {1, 2, 4, 8})
         for (int nw : {4, 8, 16})
             for (int ksw : {1, 2, 4, 8})
-                for (int rpw : {1, 2, 4}) {
+                for (int rpw : {1, 2, 4})
+                  for (int dep : {1, 2, 4}) {
                     if (ksw > nw || nw > (T <= 4 ? 16 : 8)) continue;
-                    h->pl_T = T; h->pl_NW = nw; h->pl_KSW = ksw; h->pl_RPW = rpw;
+                    if (dep > 1 && (T == 1 || dep > T)) continue;   // the kernel has no deeper variant there
+                    h->pl_T = T; h->pl_NW = nw; h->pl_KSW = ksw; h->pl_RPW = rpw; h->pl_D = dep;
                     planar_order(h, row_nnz);
                     if (h->pl_order.size() > order_cap) continue;
                     if (cudaMemcpyAsync(d_order, h->pl_order.data(), h->pl_order.size() * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
@@ -653,7 +655,7 @@ void autotune_planar(cadnn_weights *h, const std::vector<int64_t> &row_nnz)
                             float ms = 0.0f;
                             cudaEventElapsedTime(&ms, e0, e1);
                             float us = ms * 1e3f / 8.0f;
-                            if (best_us < 0.0f || us < best_us) { best_us = us; bT = T; bNW = nw; bRPW = rpw; bKSW = ksw; }
+                            if (best_us < 0.0f || us < best_us) { best_us = us; bT = T; bNW = nw; bRPW = rpw; bKSW = ksw; bD = dep; }
                         }
                         cudaEventDestroy(e0);
                         cudaEventDestroy(e1);
@@ -662,7 +664,7 @@ void autotune_planar(cadnn_weights *h, const std::vector<int64_t> &row_nnz)
                     if (g) cudaGraphDestroy(g);
                     cudaGetLastError();
                 }
-    h->pl_T = bT; h->pl_NW = bNW; h->pl_RPW = bRPW; h->pl_KSW = bKSW;
+    h->pl_T = bT; h->pl_NW = bNW; h->pl_RPW = bRPW; h->pl_KSW = bKSW; h->pl_D = bD;
     h->pl_us = best_us;
     // the staged variant runs when it measured faster (an unmeasured one is not trusted against a measured one)
     if (h->has_ps && best_us > 0.0f) h->use_ps = (h->ps_us > 0.0f && h->ps_us <= best_us) || getenv("CADNN_FORCE_STAGED") != nullptr;
@@ -1262,7 +1264,7 @@ cadnn_status cadnn_weights_planar_schedule(const cadnn_weights *w, int sched[16]
         memcpy(v, t, sizeof(v));
     } else if (w->has_planar) {
         const int slots = std::max(1, w->pl_NW / std::max(1, w->pl_KSW));
-        int t[16] = {1, w->pl_T, w->pl_RPW, w->pl_NW, w->pl_KSW, slots * w->pl_RPW, w->desc.c_in, 0, 1, 0, 0, 0,
+        int t[16] = {1, w->pl_T, w->pl_RPW, w->pl_NW, w->pl_KSW, slots * w->pl_RPW, w->desc.c_in, w->pl_D, 1, 0, 0, 0,
                      (int)lrintf(w->ps_us * 100.0f), (int)lrintf(w->pl_us * 100.0f), 0, 0};
         memcpy(v, t, sizeof(v));
     }

@@ -45,7 +45,10 @@ __device__ __forceinline__ float pl_act(float z, int act)
     return z;
 }
 
-template <int T>
+// D: depth of a batch of nonzeros (16 * D activation loads in flight per lane).  At batch 1 no
+// layer fills the device, registers are free, and what a warp pays is one L1 / L2 round trip per
+// batch: deeper batches mean fewer of them.
+template <int T, int D>
 __global__ void __launch_bounds__(512) sconv_planar_kernel(const PlanarParams p)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -109,7 +112,7 @@ __global__ void __launch_bounds__(512) sconv_planar_kernel(const PlanarParams p)
             // A batch issues all its activation loads before the first multiply-add: the loads are
             // independent L1/L2 round trips and only their number in flight hides that latency.
             // Slots past the end of the slice hold {0, offset 0}: they add nothing.
-            constexpr int P = T == 1 ? 8 : T == 2 ? 4 : T == 4 ? 2 : 1;   // pairs per batch
+            constexpr int P = (8 * D / T) > 8 ? 8 : (8 * D / T);   // pairs per batch
             const uint4 zero4 = make_uint4(0, 0, 0, 0);
             uint4 nx[P];
 #pragma unroll
@@ -243,11 +246,16 @@ cadnn_status launch_sconv_planar(const cadnn_weights *w, const void *x, int n, v
     if (blocks <= 0) return CADNN_OK;
     if (blocks > 2147483647LL) return CADNN_E_UNSUPPORTED;
     const int threads = w->pl_NW * 32;
-    switch (T) {
-        case 1: return launch_kernel(sconv_planar_kernel<1>, (int)blocks, threads, 0, ep.pdl, st, p);
-        case 2: return launch_kernel(sconv_planar_kernel<2>, (int)blocks, threads, 0, ep.pdl, st, p);
-        case 4: return launch_kernel(sconv_planar_kernel<4>, (int)blocks, threads, 0, ep.pdl, st, p);
-        case 8: return launch_kernel(sconv_planar_kernel<8>, (int)blocks, threads, 0, ep.pdl, st, p);
+    switch (T * 10 + (w->pl_D >= 4 ? 4 : w->pl_D >= 2 ? 2 : 1)) {
+        case 11: case 12: case 14: return launch_kernel(sconv_planar_kernel<1, 1>, (int)blocks, threads, 0, ep.pdl, st, p);
+        case 21: return launch_kernel(sconv_planar_kernel<2, 1>, (int)blocks, threads, 0, ep.pdl, st, p);
+        case 22: case 24: return launch_kernel(sconv_planar_kernel<2, 2>, (int)blocks, threads, 0, ep.pdl, st, p);
+        case 41: return launch_kernel(sconv_planar_kernel<4, 1>, (int)blocks, threads, 0, ep.pdl, st, p);
+        case 42: return launch_kernel(sconv_planar_kernel<4, 2>, (int)blocks, threads, 0, ep.pdl, st, p);
+        case 44: return launch_kernel(sconv_planar_kernel<4, 4>, (int)blocks, threads, 0, ep.pdl, st, p);
+        case 81: return launch_kernel(sconv_planar_kernel<8, 1>, (int)blocks, threads, 0, ep.pdl, st, p);
+        case 82: return launch_kernel(sconv_planar_kernel<8, 2>, (int)blocks, threads, 0, ep.pdl, st, p);
+        case 84: return launch_kernel(sconv_planar_kernel<8, 4>, (int)blocks, threads, 0, ep.pdl, st, p);
     }
     return CADNN_E_UNSUPPORTED;
 }

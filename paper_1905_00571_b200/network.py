@@ -71,5 +71,9 @@ class PackedModel:
     def forward_host(self, x_host, y_host, use_graph=True, stream=None):
         return B.cadnn_forward_host(self.net, x_host, y_host, use_graph, stream)
 
+    def launches_per_forward(self):
+        """Kernel launches one forward issues (cadnn_net_info)."""
+        return B.cadnn_net_info(self.net)["launches"]
+
     def layer_times(self, x, y, flush_l2=False, reps=1):
         return B.cadnn_net_layer_times(self.net, x, y, len(self.model.ops), flush_l2, reps)
