@@ -269,6 +269,11 @@ def run_ours(args):
         roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
     roof.update(kernel=top, launches_per_step=ft["launches"], avg_launch_us=ft["ms"] * 1e3 / ft["launches"])
+    if top.startswith("sconv"):   # CUDA kernels behind the family in this net's layout
+        from paper_1905_00571_b200 import binding as B
+        planar = B.cadnn_net_layout(pm.net)["planar"]
+        roof["cuda_kernels"] = (["sconv_planar_kernel", "sconv_planar_tma_kernel", "sconv_planar_staged_kernel"]
+                                if planar else ["sconv_kernel"])
     t_roof_nom = sum(r["t_roof_us"] for r in rows_nom)
     t_roof_meas = sum(r["t_roof_us"] for r in rows_meas)
     k3 = [(r, ms) for r, ms in zip(rows_nom, per) if r["family"] == "sconv_kxk" and r["nnz"] and r["name"] not in ("conv1", "stem")]

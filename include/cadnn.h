@@ -61,7 +61,11 @@ typedef enum {
 #define CADNN_PACK_HOST_ONLY 1 /* build the packed image on the host only (no device needed, no compute) */
 #define CADNN_PACK_AUTOTUNE 2  /* conv layers: time the candidate schedules on the current device (batch_hint
                                   images of zeros, scratch buffers allocated and freed inside the call) and
-                                  keep the fastest, instead of trusting the packer's time model */
+                                  keep the fastest, instead of trusting the packer's time model.  With
+                                  CADNN_TUNE_CACHE=<file> in the environment the choices are appended to that
+                                  text file and a later pack of the same layer (geometry, batch hint, nonzeros
+                                  per filter) reads them back instead of timing: tune once per machine, and a
+                                  profiled run executes the schedules of the plain run */
 
 /*
  * One layer.  The packer is the offline stage of Section 4 ("Memory layout

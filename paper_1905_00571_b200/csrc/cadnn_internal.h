@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <memory>
 #include <vector>
 #include "cadnn.h"
 
@@ -66,8 +67,18 @@ struct PsSchedule {
     int hdr_bytes = 0, block_bytes = 0, tile_bytes = 0, stage_bytes = 0, smem_bytes = 0;
 };
 
+// measured schedule choices of one layer, as kept in the schedule cache (pack.cu)
+struct TuneRecord {
+    Schedule s;
+    PsSchedule ps;
+    int pl_T, pl_NW, pl_RPW, pl_KSW, pl_D, use_ps;
+    float pl_us, ps_us, nhwc_us;
+};
+
 struct cadnn_weights {
     cadnn_layer_desc desc;
+    uint64_t tune_key = 0;                 // key of this layer in the schedule cache (0 = not a tuned pack)
+    std::shared_ptr<TuneRecord> tuned;     // choices taken from the cache instead of timing
     int fmt = 0;
     int h_out = 1, w_out = 1;
     int64_t nnz = 0;

@@ -190,7 +190,7 @@ template <int T, int RPW>
 __device__ __forceinline__ void ps_block_tail(const PsParams &p, unsigned char *smem, int lane, int rslot, int slice, int KS,
                                               unsigned img, int q0, unsigned okmask, const int (&co_of)[RPW],
                                               const float (&sc)[RPW], const float (&bi)[RPW], float (&acc)[RPW][T],
-                                              int KC = 1, int rank = 0)
+                                              int KC = 1, int rank = 0, const float (*res)[T] = nullptr)
 {
     // ---- warps that share a filter: partial sums meet in shared memory (the stages are free now) ----
     if (KS > 1) {
@@ -256,7 +256,8 @@ __device__ __forceinline__ void ps_block_tail(const PsParams &p, unsigned char *
                 if (okmask & (1u << t)) {
                     const size_t oi = obase + 32 * t;
                     float z = fmaf(acc[j][t], sc[j], bi[j]);
-                    if (p.residual) z += p.residual[oi];
+                    if (res) z += res[j][t];               // fetched before the multiply-add loop
+                    else if (p.residual) z += p.residual[oi];
                     p.y[oi] = ps_act(z, p.act);
                 }
             }
@@ -490,6 +491,16 @@ __global__ void __launch_bounds__(512) sconv_planar_tma_kernel(const PsParams p,
         sc[j] = (p.scale && co_of[j] >= 0) ? p.scale[co_of[j]] : 1.0f;
         bi[j] = (p.bias && co_of[j] >= 0) ? p.bias[co_of[j]] : 0.0f;
     }
+    // the residual is requested now, so that its round trip to L2 overlaps the multiply-add loop
+    float res[RPW][T];
+#pragma unroll
+    for (int j = 0; j < RPW; ++j)
+#pragma unroll
+        for (int t = 0; t < T; ++t) {
+            res[j][t] = 0.0f;
+            if (p.residual && slice == 0 && co_of[j] >= 0 && (okmask & (1u << t)))
+                res[j][t] = __ldg(p.residual + ((size_t)img * p.c_out + co_of[j]) * p.pitch_out + q0 + lane + 32 * t);
+        }
     __syncthreads();   // the barriers are initialised for everyone
 
     int buf = 0;
@@ -509,7 +520,8 @@ __global__ void __launch_bounds__(512) sconv_planar_tma_kernel(const PsParams p,
             parity ^= 1u;
         }
     }
-    ps_block_tail<T, RPW>(p, smem, lane, rslot, slice, KS, img, q0, okmask, co_of, sc, bi, acc, KC, rank);
+    ps_block_tail<T, RPW>(p, smem, lane, rslot, slice, KS, img, q0, okmask, co_of, sc, bi, acc, KC, rank,
+                          p.residual ? res : nullptr);
 }
 
 template <int T, int RPW>

@@ -125,8 +125,38 @@ def test_timed_schedule_selection_keeps_results():
     assert_close_f32(got, want, str(info))
 
 
+def test_schedule_cache_reproduces_the_timed_choice(tmp_path, monkeypatch):
+    """CADNN_TUNE_CACHE: the second pack of a layer reads the measured schedules back (no timing) and computes the same."""
+    B = _B()
+    cache = tmp_path / "tune.cache"
+    monkeypatch.setenv("CADNN_TUNE_CACHE", str(cache))
+    g = gen.rng(46)
+    x = gen.relu_normal_input(g, (1, 14, 14, 128))
+    wt = gen.he_weights(g, 96, 3, 3, 128)
+    mask = gen.magnitude_mask(wt, 0.125)
+    want = ref.conv2d_f32(x, wt, mask, 1, 1, act="relu")
+    d = B.make_desc(128, 96, 3, 3, 1, 1, 1, 14, 14, 1, "f32", autotune=True)
+    w1 = B.cadnn_pack(d, wt, mask)
+    assert cache.exists() and len(cache.read_text().splitlines()) == 1
+    w2 = B.cadnn_pack(d, wt, mask)
+    assert len(cache.read_text().splitlines()) == 1          # nothing was timed again
+    assert B.cadnn_weights_schedule(w1) == B.cadnn_weights_schedule(w2)
+    assert B.cadnn_weights_planar_schedule(w1) == B.cadnn_weights_planar_schedule(w2)
+    xd = torch.from_numpy(x).to(DEV)
+    for w in (w1, w2):
+        y = torch.empty((1, 14, 14, 96), device=DEV)
+        B.cadnn_conv2d(w, xd, y, act="relu")
+        torch.cuda.synchronize()
+        assert_close_f32(y.cpu().numpy(), want, "cached schedule")
+    # another layer (different nonzeros per filter) is a different key
+    mask2 = gen.magnitude_mask(wt, 0.25)
+    B.cadnn_pack(d, wt, mask2)
+    assert len(cache.read_text().splitlines()) == 2
+
+
 STEM_CASES = [(1, 64, 64, 3, 64, 7, 2, 3), (2, 33, 47, 3, 32, 3, 2, 1), (1, 20, 20, 4, 24, 3, 1, 1),
-              (1, 18, 70, 1, 70, 5, 1, 2), (1, 224, 224, 3, 64, 7, 2, 3)]
+              (1, 18, 70, 1, 70, 5, 1, 2), (1, 224, 224, 3, 64, 7, 2, 3), (2, 30, 141, 3, 70, 7, 2, 3),
+              (1, 9, 9, 3, 8, 3, 2, 1)]
 
 
 @pytest.mark.parametrize("case", STEM_CASES)
