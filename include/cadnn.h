@@ -252,7 +252,8 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
  * Layers after the first are launched as programmatic dependents of their predecessor
  * (their weight fetch overlaps its stores); set CADNN_NO_PDL in the environment before
  * cadnn_net_create to use plain stream order instead (CADNN_NO_PDL_GRAPH: only inside
- * graphs).  In a captured graph an op whose result the next op does not read (a residual
+ * graphs; NHWC networks use them inside graphs only with CADNN_PDL_GRAPH set, they measured
+ * slower there).  In a captured graph an op whose result the next op does not read (a residual
  * block's downsample conv) becomes a parallel branch; CADNN_NO_FORK keeps one chain.
  * CADNN_PERSIST=1 (experimental, slower where measured) runs the whole run of planar sparse
  * convs as one cooperative kernel with device-wide barriers between layers.

@@ -401,6 +401,9 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
         return st;
     }
     net->out_bytes = net->slots[net->out_slot].bytes;
+    // inside graphs, programmatic launches pay off for the planar kernels only (the NHWC sparse conv
+    // measured slower with them: 556 -> 608 us on ResNet-50, 367 -> 410 us on the int8 VGG-16)
+    if (!net->planar && getenv("CADNN_PDL_GRAPH") == nullptr) net->pdl_graph = false;
     {
         const char *pe = getenv("CADNN_PERSIST");   // "0" / "1"; unset: off
         if (net->planar && pe && atoi(pe) != 0) plan_persistent(net);
