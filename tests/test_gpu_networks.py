@@ -72,3 +72,35 @@ def test_vgg16_int8_full_batch1_bit_exact():
     x, got = _run(m, 1)
     want, _ = oracle_forward.forward(m, x)
     assert_exact(got, want, "vgg logits")
+
+
+def test_graph_with_parallel_branches_matches_layer_by_layer():
+    """A hand-made op list with a branch read later as a residual and a branch nobody reads: the captured
+    graph (forked branches, joined where read or at the end) gives the oracle's result, as does the
+    plain launch order."""
+    from paper_1905_00571_b200 import binding as B
+    from oracle import ref
+    from workloads import gen
+    g = gen.rng(77)
+    c = 16
+    x = gen.relu_normal_input(g, (2, 12, 12, c))
+    ws, masks, handles = [], [], []
+    for _ in range(5):
+        w = gen.he_weights(g, c, 3, 3, c)
+        m = gen.random_mask(g, w.shape, 0.3)
+        d = B.make_desc(c, c, 3, 3, 1, 1, 1, 12, 12, 2, "f32")
+        ws.append(w); masks.append(m); handles.append(B.cadnn_pack(d, w, m))
+    # slots: 0 input; A: 0->1; B: 1->2 (read only by D, as residual); C: 1->3; D: 3->4 (+2); E: 1->5 (never read); F: 4->6
+    plan = [(0, 0, 1, -1), (1, 1, 2, -1), (2, 1, 3, -1), (3, 3, 4, 2), (4, 1, 5, -1), (0, 4, 6, -1)]
+    ops = [B.Op(B.OP_CONV, handles[wi].handle, src, dst, res, None, None, B.ACT["relu"], B.DTYPE["f32"], 0, 0, 0)
+           for wi, src, dst, res in plan]
+    vals = {0: x}
+    for wi, src, dst, res in plan:
+        vals[dst] = ref.conv2d_f32(vals[src], ws[wi], masks[wi], 1, 1, residual=vals[res] if res >= 0 else None, act="relu")
+    net = B.cadnn_net_create(ops, 2, 12, 12, c, "f32", keep=handles)
+    xd = torch.from_numpy(x).to(DEV)
+    for use_graph in (True, True, False):
+        y = torch.zeros((2, 12, 12, c), device=DEV)
+        B.cadnn_forward(net, xd, y, use_graph, None)
+        torch.cuda.synchronize()
+        assert_close_f32(y.cpu().numpy(), vals[6], "forked graph" if use_graph else "stream order")
