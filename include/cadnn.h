@@ -245,9 +245,10 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
  * cadnn_forward - run the network: x device input, y device output of the last op.
  * use_graph != 0 replays a CUDA graph captured on the first call with this (x, y)
  * pair (re-captured when either pointer changes); 0 launches the layers one by one.
- * Float networks made of a dense stem, sparse convs, max pools, a global average pool and fc
- * layers keep their intermediate feature maps channel-planar with a zero halo (see
- * cadnn_conv2d_planar); others (depthwise, int8) keep NHWC.  CADNN_NO_PLANAR in the
+ * Float networks made of a dense stem, sparse convs, dense depthwise convs of up to 9 taps,
+ * max pools, a global average pool and fc layers keep their intermediate feature maps
+ * channel-planar with a zero halo (see cadnn_conv2d_planar); others (int8) keep NHWC
+ * (CADNN_NO_PLANAR_DW: networks with depthwise layers too).  CADNN_NO_PLANAR in the
  * environment at cadnn_net_create forces NHWC.
  * Layers after the first are launched as programmatic dependents of their predecessor
  * (their weight fetch overlaps its stores); set CADNN_NO_PDL in the environment before

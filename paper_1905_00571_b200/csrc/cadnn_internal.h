@@ -167,6 +167,9 @@ cadnn_status launch_sconv_planar(const cadnn_weights *w, const void *x, int n, v
                                  cudaStream_t st);
 cadnn_status launch_sconv_planar_staged(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
                                         cudaStream_t st);
+bool dw_planar_ok(const cadnn_weights *w);   // a depthwise layer the planar layout can run (float, <= 9 taps, pad within the halo)
+cadnn_status launch_dw_planar(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
+                              cudaStream_t st);
 cadnn_status read_copy_timeouts(int *count);
 cadnn_status read_barrier_timeouts(int *count);
 

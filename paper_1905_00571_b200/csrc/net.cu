@@ -72,6 +72,7 @@ cadnn_status run_op(cadnn_net *net, const cadnn_op &op, const void *x, void *y, 
                 le.planar_out = true;
                 return launch_dense_smallc(op.w, src, si.n, dst, le, st);
             }
+            if (op.w->s.kind == KK_DW) return launch_dw_planar(op.w, src, si.n, dst, le, st);
             if (op.w->has_ps && op.w->use_ps) return launch_sconv_planar_staged(op.w, src, si.n, dst, le, st);
             return launch_sconv_planar(op.w, src, si.n, dst, le, st);
         }
@@ -312,7 +313,7 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
         net->in_bytes = (int64_t)n * h * wd * c * dtype_size(in_dtype);
         // Channel-planar intermediates are used when every op has a planar kernel: a dense stem on
         // the NHWC input, then sparse float convs, max pools, a global average pool, and fc layers
-        // fed by it.  (Depthwise and int8 layers keep NHWC.)
+        // fed by it, and dense depthwise layers of up to 9 taps.  (int8 layers keep NHWC.)
         bool planar = in_dtype == CADNN_F32 && getenv("CADNN_NO_PLANAR") == nullptr && n_ops >= 2 &&
                       ops[n_ops - 1].kind == CADNN_OP_FC;
         std::vector<char> flat(max_slot + 1, 0);   // slot holds a dense [n][c] vector
@@ -321,7 +322,8 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
             if (op.kind == CADNN_OP_CONV) {
                 if (!op.w) { planar = false; break; }
                 const bool stem = op.w->s.kind == KK_DENSE_SMALLC && op.src == 0 && op.res < 0;
-                if (!stem && (!op.w->has_planar || op.src == 0 || flat[op.src])) planar = false;
+                const bool dw = dw_planar_ok(op.w) && op.res < 0 && op.src != 0 && !flat[op.src] && getenv("CADNN_NO_PLANAR_DW") == nullptr;
+                if (!stem && !dw && (!op.w->has_planar || op.src == 0 || flat[op.src])) planar = false;
             } else if (op.kind == CADNN_OP_FC) {
                 if (!flat[op.src]) planar = false;
                 flat[op.dst] = 1;

@@ -215,6 +215,71 @@ __global__ void __launch_bounds__(256) gavgpool_planar_kernel(const float *x, fl
     if (lane == 0) y[pl] = s * inv;
 }
 
+// Dense depthwise convolution over planar tensors: a warp takes 32 * T consecutive positions of ONE
+// channel plane; a tap is one contiguous 128-byte load per band, the zero halo is the padding,
+// the kh * kw taps of the channel are broadcast loads from the tap-major weights.
+struct DwPlanarParams {
+    const float *x;
+    float *y;
+    const float *wt;   // [kh * kw][c]
+    const float *scale;
+    const float *bias;
+    int nc, c, wp_in, plane_in, wp_out, plane_out, h_out, w_out, kh, kw, stride, off0, halo, qtot, tiles, act;
+    FastDiv d_wp_out, d_tiles, d_c;
+};
+
+template <int T>
+__global__ void __launch_bounds__(256) dw_planar_kernel(const DwPlanarParams p)
+{
+    const int lane = threadIdx.x & 31;
+    const unsigned task = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const unsigned pl = fdiv(task, p.d_tiles);
+    const int tile = (int)(task - pl * p.tiles);
+    const bool live = pl < (unsigned)p.nc;
+    const int ch = live ? (int)(pl - fdiv(pl, p.d_c) * p.c) : 0;
+    const int q0 = tile * (32 * T);
+    int inb[T];
+    unsigned okmask = 0;
+#pragma unroll
+    for (int t = 0; t < T; ++t) {
+        const int q = q0 + 32 * t + lane;
+        const int qc = min(q, p.qtot - 1);
+        const int oy = (int)fdiv((unsigned)qc, p.d_wp_out);
+        const int oxp = qc - oy * p.wp_out;
+        const bool ok = live && q < p.qtot && oxp >= p.halo && oxp < p.halo + p.w_out;
+        if (ok) okmask |= 1u << t;
+        const int oxs = ok ? oxp : p.halo;
+        inb[t] = (oy * p.stride + p.off0) * p.wp_in + (oxs - p.halo) * p.stride + p.off0;
+    }
+    // static data first: the taps and the epilogue pair of this channel
+    float wv[9];
+    const int taps = p.kh * p.kw;   // <= 9 (the host checks)
+#pragma unroll
+    for (int k = 0; k < 9; ++k) wv[k] = k < taps ? __ldg(p.wt + (size_t)k * p.c + ch) : 0.0f;
+    const float sc = p.scale ? __ldg(p.scale + ch) : 1.0f;
+    const float bi = p.bias ? __ldg(p.bias + ch) : 0.0f;
+    grid_dep_wait();
+    grid_dep_trigger();
+    if (!live) return;
+    const float *xp = p.x + (size_t)pl * p.plane_in;
+    float acc[T];
+#pragma unroll
+    for (int t = 0; t < T; ++t) acc[t] = 0.0f;
+#pragma unroll
+    for (int k = 0; k < 9; ++k) {
+        if (k < taps) {
+            const int ky = k / p.kw, kx = k - ky * p.kw;
+            const int off = ky * p.wp_in + kx;
+#pragma unroll
+            for (int t = 0; t < T; ++t) acc[t] = fmaf(wv[k], __ldg(xp + inb[t] + off), acc[t]);
+        }
+    }
+    float *yp = p.y + (size_t)pl * p.plane_out + (size_t)p.halo * p.wp_out + q0 + lane;
+#pragma unroll
+    for (int t = 0; t < T; ++t)
+        if (okmask & (1u << t)) yp[32 * t] = pl_act(fmaf(acc[t], sc, bi), p.act);
+}
+
 }  // namespace
 
 cadnn_status launch_sconv_planar(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
@@ -280,4 +345,43 @@ cadnn_status launch_gavgpool_planar(const float *x, int n, int h, int wd, int c,
     if (n * c <= 0) return CADNN_OK;
     return launch_kernel(gavgpool_planar_kernel, (n * c + 7) / 8, 256, 0, pdl, st, x, y, n * c, h, wd, wd + 2 * halo,
                          planar_pitch(h, wd), halo, 1.0f / (float)(h * wd));
+}
+
+bool dw_planar_ok(const cadnn_weights *w)
+{
+    const cadnn_layer_desc &d = w->desc;
+    return w->s.kind == KK_DW && d.dtype == CADNN_F32 && d.kh * d.kw <= 9 && d.pad <= kPlanarHalo &&
+           d.kh - 1 - d.pad <= kPlanarHalo && d.kw - 1 - d.pad <= kPlanarHalo && w->d_dense != nullptr;
+}
+
+cadnn_status launch_dw_planar(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
+                              cudaStream_t st)
+{
+    const cadnn_layer_desc &d = w->desc;
+    if (!dw_planar_ok(w) || ep.residual) return CADNN_E_UNSUPPORTED;
+    const int halo = kPlanarHalo;
+    DwPlanarParams p;
+    p.x = (const float *)x; p.y = (float *)y; p.wt = w->d_dense;
+    p.scale = ep.scale; p.bias = ep.bias;
+    p.nc = n * d.c_out; p.c = d.c_out;
+    p.wp_in = d.in_w + 2 * halo; p.plane_in = planar_pitch(d.in_h, d.in_w);
+    p.h_out = w->h_out; p.w_out = w->w_out;
+    p.wp_out = w->w_out + 2 * halo; p.plane_out = planar_pitch(w->h_out, w->w_out);
+    p.kh = d.kh; p.kw = d.kw; p.stride = d.stride; p.off0 = halo - d.pad; p.halo = halo;
+    p.qtot = w->h_out * p.wp_out;
+    p.act = ep.act;
+    const int T = p.qtot >= 1024 ? 4 : p.qtot >= 256 ? 2 : 1;
+    p.tiles = (p.qtot + 32 * T - 1) / (32 * T);
+    p.d_wp_out = make_fastdiv(p.wp_out);
+    p.d_tiles = make_fastdiv(p.tiles);
+    p.d_c = make_fastdiv(p.c);
+    const long long tasks = (long long)p.nc * p.tiles;
+    if (tasks <= 0) return CADNN_OK;
+    const long long blocks = (tasks + 7) / 8;
+    if (blocks > 2147483647LL || tasks >= (1LL << 31)) return CADNN_E_UNSUPPORTED;
+    switch (T) {
+        case 1: return launch_kernel(dw_planar_kernel<1>, (int)blocks, 256, 0, ep.pdl, st, p);
+        case 2: return launch_kernel(dw_planar_kernel<2>, (int)blocks, 256, 0, ep.pdl, st, p);
+        default: return launch_kernel(dw_planar_kernel<4>, (int)blocks, 256, 0, ep.pdl, st, p);
+    }
 }

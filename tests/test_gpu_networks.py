@@ -104,3 +104,30 @@ def test_graph_with_parallel_branches_matches_layer_by_layer():
         B.cadnn_forward(net, xd, y, use_graph, None)
         torch.cuda.synchronize()
         assert_close_f32(y.cpu().numpy(), vals[6], "forked graph" if use_graph else "stream order")
+
+
+@pytest.mark.parametrize("image,batch", [(80, 3), (72, 1)])
+def test_mobilenet_v2_runs_channel_planar(image, batch, monkeypatch):
+    """Depthwise layers have a planar kernel: the whole MobileNet-V2 keeps planar feature maps (odd map
+    sizes at stride 2 included) and matches the oracle; the NHWC route gives the same logits."""
+    from paper_1905_00571_b200 import binding as B
+    from paper_1905_00571_b200.network import PackedModel
+    m = models.mobilenet_v2(width=0.5, image=image, classes=100)
+    x = models.make_input(m, batch)
+    want, _ = oracle_forward.forward(m, x)
+    xd = torch.from_numpy(x).to(DEV)
+    outs = []
+    for planar in (True, False):
+        if planar:
+            monkeypatch.delenv("CADNN_NO_PLANAR_DW", raising=False)
+        else:
+            monkeypatch.setenv("CADNN_NO_PLANAR_DW", "1")
+        pm = PackedModel(m, batch, DEV)
+        assert B.cadnn_net_layout(pm.net)["planar"] == planar
+        y = pm.new_output()
+        pm.forward(xd, y)
+        pm.forward(xd, y, use_graph=False)
+        torch.cuda.synchronize()
+        _check_logits(y.cpu().numpy(), want)
+        outs.append(y.cpu().numpy())
+    assert_close_f32(outs[0], outs[1], "planar vs NHWC", floor=NET_FLOOR)
