@@ -29,8 +29,10 @@
  *
  * Pins (see tests/test_oracle_pins.py): hand-worked literals, shift and
  * identity filters, 1x1 == matrix product, FC == mat-vec, linearity, mask
- * additivity, channel-permutation equivariance, a float64 library convolution,
- * and an exact rational check of the requantization scalar.
+ * additivity, channel-permutation equivariance, a float64 library convolution
+ * (square and rectangular kernels, grouped int8 included), library pooling
+ * routines with and without padding, and an exact rational check of the
+ * requantization scalars (with and without the int8 residual).
  * Parity unpinned: ImageNet accuracy of the paper's Table 2 (needs its data
  * and trained weights).
  */
@@ -101,17 +103,17 @@ static float epilogue_f32(double acc, const float *scale, const float *bias,
  * mask same shape as wt or NULL (= all kept), y [n][h_out][w_out][c_out].
  * Returns 0, or -1 on an invalid shape.
  */
-int ref_conv2d_f32(const float *x, int n, int h, int w, int c_in,
-                   const float *wt, const uint8_t *mask,
-                   int c_out, int kh, int kw, int stride, int pad, int groups,
-                   const float *scale, const float *bias, const float *residual,
-                   int act, float *y)
+int ref_conv2d_f32_hw(const float *x, int n, int h, int w, int c_in,
+                      const float *wt, const uint8_t *mask,
+                      int c_out, int kh, int kw, int stride, int pad_h, int pad_w, int groups,
+                      const float *scale, const float *bias, const float *residual,
+                      int act, float *y)
 {
-    if (groups < 1 || c_in % groups || c_out % groups || stride < 1 || pad < 0) return -1;
+    if (groups < 1 || c_in % groups || c_out % groups || stride < 1 || pad_h < 0 || pad_w < 0) return -1;
     const int cg = c_in / groups;      /* input channels seen by one filter */
     const int og = c_out / groups;     /* filters per group */
-    const int ho = out_extent(h, kh, stride, pad);
-    const int wo = out_extent(w, kw, stride, pad);
+    const int ho = out_extent(h, kh, stride, pad_h);
+    const int wo = out_extent(w, kw, stride, pad_w);
     const long rows = (long)n * ho;
 #pragma omp parallel for schedule(dynamic, 1)
     for (long row = 0; row < rows; ++row) {
@@ -121,9 +123,9 @@ int ref_conv2d_f32(const float *x, int n, int h, int w, int c_in,
                 const int g = co / og;
                 double acc = 0.0;
                 for (int ky = 0; ky < kh; ++ky) {
-                    const int iy = oy * stride + ky - pad;
+                    const int iy = oy * stride + ky - pad_h;
                     for (int kx = 0; kx < kw; ++kx) {
-                        const int ix = ox * stride + kx - pad;
+                        const int ix = ox * stride + kx - pad_w;
                         const int inside = (iy >= 0 && iy < h && ix >= 0 && ix < w);
                         for (int ci = 0; ci < cg; ++ci) {
                             const size_t wi = (((size_t)co * kh + ky) * kw + kx) * cg + ci;
@@ -141,6 +143,17 @@ int ref_conv2d_f32(const float *x, int n, int h, int w, int c_in,
         }
     }
     return 0;
+}
+
+/* The same layer with one padding for both axes (square-kernel networks). */
+int ref_conv2d_f32(const float *x, int n, int h, int w, int c_in,
+                   const float *wt, const uint8_t *mask,
+                   int c_out, int kh, int kw, int stride, int pad, int groups,
+                   const float *scale, const float *bias, const float *residual,
+                   int act, float *y)
+{
+    return ref_conv2d_f32_hw(x, n, h, w, c_in, wt, mask, c_out, kh, kw, stride, pad, pad, groups,
+                             scale, bias, residual, act, y);
 }
 
 /*
@@ -206,12 +219,41 @@ int8_t ref_requant_s8(int32_t acc, float m, float b, int act)
     return (int8_t)lrintf(t);
 }
 
+/*
+ * Requantization with an int8 residual (the shortcut of a quantized residual
+ * block): two fused multiply-adds in this order,
+ *   t = fmaf((float)acc, M, B);  t = fmaf((float)r, residual_scale, t);
+ * then ReLU, clamp, round half to even as above.  residual_scale = s_r / s_y is
+ * precomputed by the caller.
+ */
+float ref_requant_res_f32(int32_t acc, float m, float b, int8_t r, float residual_scale, int act)
+{
+    float t = fmaf((float)acc, m, b);
+    t = fmaf((float)r, residual_scale, t);
+    if (act == REF_ACT_RELU) t = t > 0.0f ? t : 0.0f;
+    return t;
+}
+
+int8_t ref_requant_res_s8(int32_t acc, float m, float b, int8_t r, float residual_scale, int act)
+{
+    float t = ref_requant_res_f32(acc, m, b, r, residual_scale, act);
+    if (t > 127.0f) t = 127.0f;
+    if (t < -127.0f) t = -127.0f;
+    return (int8_t)lrintf(t);
+}
+
 static void store_q(void *y, size_t oi, int32_t acc, const float *m, const float *b,
-                    int co, int act, int out_kind)
+                    const int8_t *residual, float residual_scale, int co, int act, int out_kind)
 {
     const float mm = m ? m[co] : 1.0f;
     const float bb = b ? b[co] : 0.0f;
     if (out_kind == REF_OUT_S32) ((int32_t *)y)[oi] = acc;
+    else if (residual) {
+        if (out_kind == REF_OUT_F32)
+            ((float *)y)[oi] = ref_requant_res_f32(acc, mm, bb, residual[oi], residual_scale, act);
+        else
+            ((int8_t *)y)[oi] = ref_requant_res_s8(acc, mm, bb, residual[oi], residual_scale, act);
+    }
     else if (out_kind == REF_OUT_F32) ((float *)y)[oi] = ref_requant_f32(acc, mm, bb, act);
     else ((int8_t *)y)[oi] = ref_requant_s8(acc, mm, bb, act);
 }
@@ -221,10 +263,11 @@ static void store_q(void *y, size_t oi, int32_t acc, const float *m, const float
  * accumulation over the dense masked weights, then store_q.  ReLU6 is not
  * defined for this path (returns -1).
  */
-int ref_conv2d_s8(const int8_t *x, int n, int h, int w, int c_in,
-                  const int8_t *wq, const uint8_t *mask,
-                  int c_out, int kh, int kw, int stride, int pad, int groups,
-                  const float *m, const float *b, int act, int out_kind, void *y)
+int ref_conv2d_s8_res(const int8_t *x, int n, int h, int w, int c_in,
+                      const int8_t *wq, const uint8_t *mask,
+                      int c_out, int kh, int kw, int stride, int pad, int groups,
+                      const float *m, const float *b, const int8_t *residual, float residual_scale,
+                      int act, int out_kind, void *y)
 {
     if (groups < 1 || c_in % groups || c_out % groups || stride < 1 || pad < 0) return -1;
     if (act == REF_ACT_RELU6) return -1;
@@ -256,11 +299,20 @@ int ref_conv2d_s8(const int8_t *x, int n, int h, int w, int c_in,
                     }
                 }
                 const size_t oi = (((size_t)bi * ho + oy) * wo + ox) * c_out + co;
-                store_q(y, oi, acc, m, b, co, act, out_kind);
+                store_q(y, oi, acc, m, b, residual, residual_scale, co, act, out_kind);
             }
         }
     }
     return 0;
+}
+
+int ref_conv2d_s8(const int8_t *x, int n, int h, int w, int c_in,
+                  const int8_t *wq, const uint8_t *mask,
+                  int c_out, int kh, int kw, int stride, int pad, int groups,
+                  const float *m, const float *b, int act, int out_kind, void *y)
+{
+    return ref_conv2d_s8_res(x, n, h, w, c_in, wq, mask, c_out, kh, kw, stride, pad, groups,
+                             m, b, NULL, 0.0f, act, out_kind, y);
 }
 
 int ref_fc_s8(const int8_t *x, int n, int k, const int8_t *wq, const uint8_t *mask,
@@ -276,7 +328,7 @@ int ref_fc_s8(const int8_t *x, int n, int k, const int8_t *wq, const uint8_t *ma
                 const int32_t wv = (mask == NULL || mask[wi]) ? (int32_t)wq[wi] : 0;
                 acc += wv * (int32_t)x[(size_t)bi * k + j];
             }
-            store_q(y, (size_t)bi * c_out + co, acc, m, b, co, act, out_kind);
+            store_q(y, (size_t)bi * c_out + co, acc, m, b, NULL, 0.0f, co, act, out_kind);
         }
     }
     return 0;
@@ -324,6 +376,32 @@ int ref_maxpool_s8(const int8_t *x, int n, int h, int w, int c, int k, int strid
                             if (v > best) best = v;
                         }
                     y[(((size_t)b * ho + oy) * wo + ox) * c + ch] = (int8_t)best;
+                }
+    return 0;
+}
+
+/*
+ * Average pooling with a k x k window.  Taps that fall in the padding count as
+ * zeros and the divisor is always k * k (the convention of the Inception-V3
+ * definition the synthetic workload follows).  Double sum, one division, rounded
+ * once to float.
+ */
+int ref_avgpool_f32(const float *x, int n, int h, int w, int c, int k, int stride, int pad, float *y)
+{
+    if (pad >= k || k < 1 || stride < 1) return -1;
+    const int ho = out_extent(h, k, stride, pad), wo = out_extent(w, k, stride, pad);
+    for (int b = 0; b < n; ++b)
+        for (int oy = 0; oy < ho; ++oy)
+            for (int ox = 0; ox < wo; ++ox)
+                for (int ch = 0; ch < c; ++ch) {
+                    double s = 0.0;
+                    for (int ky = 0; ky < k; ++ky)
+                        for (int kx = 0; kx < k; ++kx) {
+                            const int iy = oy * stride + ky - pad, ix = ox * stride + kx - pad;
+                            if (iy < 0 || iy >= h || ix < 0 || ix >= w) continue;
+                            s += (double)x[(((size_t)b * h + iy) * w + ix) * c + ch];
+                        }
+                    y[(((size_t)b * ho + oy) * wo + ox) * c + ch] = (float)(s / (double)(k * k));
                 }
     return 0;
 }

@@ -44,6 +44,12 @@ def lib():
         _lib.ref_requant_f32.argtypes = [ctypes.c_int32, ctypes.c_float, ctypes.c_float, ctypes.c_int]
         _lib.ref_requant_s8.restype = ctypes.c_int8
         _lib.ref_requant_s8.argtypes = [ctypes.c_int32, ctypes.c_float, ctypes.c_float, ctypes.c_int]
+        _lib.ref_requant_res_f32.restype = ctypes.c_float
+        _lib.ref_requant_res_f32.argtypes = [ctypes.c_int32, ctypes.c_float, ctypes.c_float, ctypes.c_int8,
+                                             ctypes.c_float, ctypes.c_int]
+        _lib.ref_requant_res_s8.restype = ctypes.c_int8
+        _lib.ref_requant_res_s8.argtypes = [ctypes.c_int32, ctypes.c_float, ctypes.c_float, ctypes.c_int8,
+                                            ctypes.c_float, ctypes.c_int]
     return _lib
 
 
@@ -67,21 +73,30 @@ def out_hw(h, w, k, stride, pad):
     return (h + 2 * pad - k) // stride + 1, (w + 2 * pad - k) // stride + 1
 
 
+def _pads(pad):
+    """pad may be one int (both axes) or a (pad_h, pad_w) pair."""
+    if isinstance(pad, (tuple, list)):
+        return int(pad[0]), int(pad[1])
+    return int(pad), int(pad)
+
+
 def conv2d_f32(x, wt, mask=None, stride=1, pad=0, groups=1, scale=None, bias=None,
                residual=None, act="none"):
-    """x [n,h,w,c_in] float32, wt [c_out,kh,kw,c_in/groups] float32 -> y [n,ho,wo,c_out]."""
+    """x [n,h,w,c_in] float32, wt [c_out,kh,kw,c_in/groups] float32 -> y [n,ho,wo,c_out].
+    pad: int, or (pad_h, pad_w) for rectangular kernels."""
     x = _c(x, np.float32); wt = _c(wt, np.float32); mask = _c(mask, np.uint8)
     scale = _c(scale, np.float32); bias = _c(bias, np.float32); residual = _c(residual, np.float32)
     n, h, w, c_in = x.shape
     c_out, kh, kw, cg = wt.shape
     assert cg * groups == c_in, "weight shape does not match c_in/groups"
-    ho, wo = (h + 2 * pad - kh) // stride + 1, (w + 2 * pad - kw) // stride + 1
+    ph, pw = _pads(pad)
+    ho, wo = (h + 2 * ph - kh) // stride + 1, (w + 2 * pw - kw) // stride + 1
     y = np.empty((n, ho, wo, c_out), np.float32)
     if residual is not None:
         assert residual.shape == y.shape
-    rc = lib().ref_conv2d_f32(_p(x), n, h, w, c_in, _p(wt), _p(mask), c_out, kh, kw,
-                              stride, pad, groups, _p(scale), _p(bias), _p(residual),
-                              ACT[act], _p(y))
+    rc = lib().ref_conv2d_f32_hw(_p(x), n, h, w, c_in, _p(wt), _p(mask), c_out, kh, kw,
+                                 stride, ph, pw, groups, _p(scale), _p(bias), _p(residual),
+                                 ACT[act], _p(y))
     if rc != 0:
         raise ValueError("ref_conv2d_f32 rejected the shape")
     return y
@@ -116,16 +131,31 @@ def requant_f32(acc, m, b, act="none"):
     return np.float32(lib().ref_requant_f32(int(acc), float(np.float32(m)), float(np.float32(b)), ACT[act]))
 
 
-def conv2d_s8(x, wq, mask=None, stride=1, pad=0, groups=1, m=None, b=None, act="none", out="s8"):
+def requant_res_s8(acc, m, b, r, rs, act="none"):
+    return int(lib().ref_requant_res_s8(int(acc), float(np.float32(m)), float(np.float32(b)), int(r),
+                                        float(np.float32(rs)), ACT[act]))
+
+
+def requant_res_f32(acc, m, b, r, rs, act="none"):
+    return np.float32(lib().ref_requant_res_f32(int(acc), float(np.float32(m)), float(np.float32(b)), int(r),
+                                                float(np.float32(rs)), ACT[act]))
+
+
+def conv2d_s8(x, wq, mask=None, stride=1, pad=0, groups=1, m=None, b=None, act="none", out="s8",
+              residual=None, residual_scale=0.0):
+    """Int8 layer; residual (int8, y's shape) joins the requantization as a second fmaf."""
     x = _c(x, np.int8); wq = _c(wq, np.int8); mask = _c(mask, np.uint8)
-    m = _c(m, np.float32); b = _c(b, np.float32)
+    m = _c(m, np.float32); b = _c(b, np.float32); residual = _c(residual, np.int8)
     n, h, w, c_in = x.shape
     c_out, kh, kw, cg = wq.shape
     assert cg * groups == c_in
     ho, wo = (h + 2 * pad - kh) // stride + 1, (w + 2 * pad - kw) // stride + 1
     y = np.empty((n, ho, wo, c_out), _OUT_NP[out])
-    rc = lib().ref_conv2d_s8(_p(x), n, h, w, c_in, _p(wq), _p(mask), c_out, kh, kw, stride, pad,
-                             groups, _p(m), _p(b), ACT[act], OUT[out], _p(y))
+    if residual is not None:
+        assert residual.shape == y.shape
+    rc = lib().ref_conv2d_s8_res(_p(x), n, h, w, c_in, _p(wq), _p(mask), c_out, kh, kw, stride, pad,
+                                 groups, _p(m), _p(b), _p(residual), ctypes.c_float(float(residual_scale)),
+                                 ACT[act], OUT[out], _p(y))
     if rc != 0:
         raise ValueError("ref_conv2d_s8 rejected the arguments")
     return y
@@ -155,6 +185,18 @@ def maxpool(x, k, stride, pad=0):
         rc = lib().ref_maxpool_f32(_p(x), n, h, w, c, k, stride, pad, _p(y))
     if rc != 0:
         raise ValueError("ref_maxpool rejected the arguments")
+    return y
+
+
+def avgpool(x, k, stride, pad=0):
+    """k x k average pool; padded taps count as zeros, divisor k*k."""
+    x = _c(x, np.float32)
+    n, h, w, c = x.shape
+    ho, wo = out_hw(h, w, k, stride, pad)
+    y = np.empty((n, ho, wo, c), np.float32)
+    rc = lib().ref_avgpool_f32(_p(x), n, h, w, c, k, stride, pad, _p(y))
+    if rc != 0:
+        raise ValueError("ref_avgpool rejected the arguments")
     return y
 
 

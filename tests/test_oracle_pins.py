@@ -304,3 +304,212 @@ def test_empty_row_gives_epilogue_of_zero():
     bias = np.array([0.1, 0.7], np.float32)
     y = ref.conv2d_f32(x, wt, mask, 1, 1, bias=bias, act="relu")
     np.testing.assert_array_equal(y[..., 1], np.full((1, 4, 4), 0.7, np.float32))
+
+
+# ---- the network walker (oracle/forward.py) ----
+
+def _op(kind, src, dst, **kw):
+    from workloads.models import Op
+    return Op(kind, kw.pop("name", kind), src, dst, **kw)
+
+
+def _model(ops, dtype, in_shape):
+    from workloads.models import Model
+    return Model("pin", dtype, in_shape, ops=ops, n_slots=max(o.dst for o in ops) + 1)
+
+
+def test_walker_handworked_network():
+    from oracle import forward as F
+    G = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "walker_handworked.json")))
+    one = lambda v: np.array(v, np.float32)
+    ops = [
+        _op("conv", 0, 1, c_in=1, c_out=1, k=2, act="relu", w=_w22(), scale=one([2.0]), bias=one([-20.0])),
+        _op("conv", 1, 2, res=1, c_in=1, c_out=1, k=1, act="relu", w=one([0.5]).reshape(1, 1, 1, 1), bias=one([1.0])),
+        _op("conv", 2, 3, res=1, c_in=1, c_out=1, k=1, act="none", w=one([-1.0]).reshape(1, 1, 1, 1)),
+        _op("gavgpool", 3, 4, c_in=1, c_out=1),
+        _op("fc", 4, 5, c_in=1, c_out=2, w=one([[2.0], [-1.0]]).reshape(2, 1, 1, 1), bias=one([0.25, 0.5])),
+    ]
+    y, slots = F.forward(_model(ops, "f32", (3, 3, 1)), _x33())
+    np.testing.assert_array_equal(slots[1][0, :, :, 0], one(G["slot1"]))
+    np.testing.assert_array_equal(slots[2][0, :, :, 0], one(G["slot2"]))
+    np.testing.assert_array_equal(slots[3][0, :, :, 0], one(G["slot3"]))
+    np.testing.assert_array_equal(slots[4].reshape(-1), one(G["slot4"]))
+    np.testing.assert_array_equal(y.reshape(-1), one(G["logits"]))
+    assert y is slots[5]
+
+
+def test_walker_equals_the_composition_of_pinned_layer_calls_f32():
+    """conv A -> conv B (+ the network input as residual) -> max pool -> fc, plus a side conv C that
+    reads A's output and lands in a channel window beside a pooled copy: every slot equals the layer
+    routines called one by one with explicitly named tensors."""
+    from oracle import forward as F
+    g = np.random.default_rng(77)
+    rn = lambda *s: g.standard_normal(s).astype(np.float32)
+    x = rn(2, 6, 6, 4)
+    wa, wb, wc, wf = rn(4, 3, 3, 4), rn(4, 3, 3, 4), rn(3, 1, 3, 4), rn(5, 1, 1, 3 * 3 * 4)
+    ma, mb = (g.random(wa.shape) < 0.5).astype(np.uint8), (g.random(wb.shape) < 0.5).astype(np.uint8)
+    mf = (g.random(wf.shape) < 0.5).astype(np.uint8)
+    sa, ba, sb, bb, sf, bf = rn(4), rn(4), rn(4), rn(4), rn(5), rn(5)
+    ops = [
+        _op("conv", 0, 1, c_in=4, c_out=4, k=3, pad=1, act="relu", w=wa, mask=ma, scale=sa, bias=ba),
+        _op("conv", 1, 2, res=0, c_in=4, c_out=4, k=3, pad=1, act="relu6", w=wb, mask=mb, scale=sb, bias=bb),
+        _op("maxpool", 2, 3, k=2, stride=2, pad=0, c_in=4, c_out=4),
+        # a concatenation: slot 4 = [conv C of slot 1 (3 channels, 1x3 kernel, pad (0,1)) | avg pool of slot 2 (4 channels)]
+        _op("conv", 1, 4, c_in=4, c_out=3, k=3, pad=0, pad_w=1, act="none", w=wc, dst_off=0, dst_total=7),
+        _op("avgpool", 2, 4, k=3, stride=1, pad=1, c_in=4, c_out=4, dst_off=3, dst_total=7),
+        _op("fc", 3, 5, c_in=36, c_out=5, w=wf, mask=mf, scale=sf, bias=bf),
+    ]
+    y, slots = F.forward(_model(ops, "f32", (6, 6, 4)), x)
+    a = ref.conv2d_f32(x, wa, ma, 1, 1, 1, sa, ba, None, "relu")
+    b = ref.conv2d_f32(a, wb, mb, 1, 1, 1, sb, bb, x, "relu6")
+    p = ref.maxpool(b, 2, 2, 0)
+    c = ref.conv2d_f32(a, wc, None, 1, (0, 1))
+    q = ref.avgpool(b, 3, 1, 1)
+    f = ref.fc_f32(p.reshape(2, -1), wf.reshape(5, -1), mf.reshape(5, -1), sf, bf)
+    np.testing.assert_array_equal(slots[1], a)
+    np.testing.assert_array_equal(slots[2], b)
+    np.testing.assert_array_equal(slots[3], p)
+    np.testing.assert_array_equal(slots[4], np.concatenate([c, q], axis=-1))
+    np.testing.assert_array_equal(y, f)
+    # the residual matters and comes from slot 0, not from the layer's own input
+    assert not np.array_equal(b, ref.conv2d_f32(a, wb, mb, 1, 1, 1, sb, bb, a, "relu6"))
+    assert not np.array_equal(b, ref.conv2d_f32(a, wb, mb, 1, 1, 1, sb, bb, None, "relu6"))
+
+
+def test_walker_equals_the_composition_of_pinned_layer_calls_int8():
+    from oracle import forward as F
+    g = np.random.default_rng(78)
+    ri = lambda *s: g.integers(-127, 128, size=s).astype(np.int8)
+    x = ri(2, 6, 6, 4)
+    wa, wb, wf = ri(4, 3, 3, 4), ri(4, 3, 3, 4), ri(5, 1, 1, 36)
+    ma = (g.random(wa.shape) < 0.5).astype(np.uint8)
+    m_a = np.full(4, 2e-3, np.float32); b_a = g.standard_normal(4).astype(np.float32)
+    m_b = np.full(4, 3e-3, np.float32); b_b = g.standard_normal(4).astype(np.float32)
+    m_f = np.full(5, 1e-3, np.float32); b_f = g.standard_normal(5).astype(np.float32)
+    ops = [
+        _op("conv", 0, 1, c_in=4, c_out=4, k=3, pad=1, act="relu", w=wa, mask=ma, scale=m_a, bias=b_a, out="s8"),
+        _op("conv", 1, 2, res=0, res_scale=0.75, c_in=4, c_out=4, k=3, pad=1, act="relu", w=wb, scale=m_b, bias=b_b, out="s8"),
+        _op("maxpool", 2, 3, k=2, stride=2, pad=0, c_in=4, c_out=4, out="s8"),
+        _op("fc", 3, 4, c_in=36, c_out=5, w=wf, scale=m_f, bias=b_f, out="f32"),
+    ]
+    y, slots = F.forward(_model(ops, "s8", (6, 6, 4)), x)
+    a = ref.conv2d_s8(x, wa, ma, 1, 1, 1, m_a, b_a, "relu", "s8")
+    b = ref.conv2d_s8(a, wb, None, 1, 1, 1, m_b, b_b, "relu", "s8", x, 0.75)
+    p = ref.maxpool(b, 2, 2, 0)
+    f = ref.fc_s8(p.reshape(2, -1), wf.reshape(5, -1), None, m_f, b_f, "none", "f32")
+    for got, want in ((slots[1], a), (slots[2], b), (slots[3], p), (y, f)):
+        assert got.dtype == want.dtype
+        np.testing.assert_array_equal(got, want)
+    assert not np.array_equal(b, ref.conv2d_s8(a, wb, None, 1, 1, 1, m_b, b_b, "relu", "s8"))
+
+
+# ---- corners ----
+
+@pytest.mark.parametrize("k,s,p", [(3, 2, 1), (3, 1, 1), (2, 2, 1), (5, 3, 2)])
+def test_padded_max_pools_against_int64_window_max(k, s, p):
+    xq = R.integers(-128, 128, size=(2, 9, 7, 3)).astype(np.int8)
+    n, h, w, c = xq.shape
+    ho, wo = (h + 2 * p - k) // s + 1, (w + 2 * p - k) // s + 1
+    lo = np.iinfo(np.int64).min
+    xp = np.full((n, h + 2 * p, w + 2 * p, c), lo, np.int64)
+    xp[:, p:p + h, p:p + w] = xq
+    want = np.empty((n, ho, wo, c), np.int64)
+    for oy in range(ho):
+        for ox in range(wo):
+            want[:, oy, ox] = xp[:, oy * s:oy * s + k, ox * s:ox * s + k].max(axis=(1, 2))
+    got = ref.maxpool(xq, k, s, p)
+    assert got.dtype == np.int8
+    np.testing.assert_array_equal(got.astype(np.int64), want)
+    # all-negative input: a padded tap must never win as a zero
+    neg = (-np.abs(xq.astype(np.int16)) - 1).clip(-128, -1).astype(np.int8)
+    assert ref.maxpool(neg, k, s, p).max() < 0
+
+
+@pytest.mark.parametrize("groups", [2, 4])
+def test_grouped_int8_convolution_against_brute_force(groups):
+    xq = R.integers(-127, 128, size=(2, 5, 6, 8)).astype(np.int8)
+    wq = R.integers(-127, 128, size=(8, 3, 3, 8 // groups)).astype(np.int8)
+    mask = (R.random(wq.shape) < 0.6).astype(np.uint8)
+    got = ref.conv2d_s8(xq, wq, mask, 2, 1, groups, out="s32")
+    want = _brute_conv(xq.astype(np.float64), wq.astype(np.float64), mask, 2, 1, groups)
+    np.testing.assert_array_equal(got.astype(np.int64), want.astype(np.int64))
+
+
+@pytest.mark.parametrize("kh,kw,ph,pw,stride", [(1, 7, 0, 3, 1), (7, 1, 3, 0, 1), (1, 3, 0, 1, 1), (3, 1, 1, 0, 2), (5, 5, 2, 2, 1), (3, 3, 0, 0, 2)])
+def test_rectangular_kernels_against_float64_library_convolution(kh, kw, ph, pw, stride):
+    x = R.standard_normal((2, 10, 9, 6)).astype(np.float32)
+    wt = R.standard_normal((5, kh, kw, 6)).astype(np.float32)
+    mask = (R.random(wt.shape) < 0.4).astype(np.uint8)
+    y = ref.conv2d_f32(x, wt, mask, stride, (ph, pw))
+    xt = torch.from_numpy(x.astype(np.float64)).permute(0, 3, 1, 2)
+    wtt = torch.from_numpy((wt * mask).astype(np.float64)).permute(0, 3, 1, 2)
+    want = torch.nn.functional.conv2d(xt, wtt, None, stride, (ph, pw)).permute(0, 2, 3, 1).numpy()
+    assert y.shape == want.shape
+    np.testing.assert_allclose(y, want.astype(np.float32), rtol=0, atol=2e-6)
+    # a single tap at (ky, kx) is a shift: pins which axis pad_h and pad_w belong to
+    one = np.zeros((1, kh, kw, 1), np.float32)
+    one[0, kh - 1, 0, 0] = 1.0
+    xs = R.standard_normal((1, 10, 9, 1)).astype(np.float32)
+    ys = ref.conv2d_f32(xs, one, None, 1, (ph, pw))
+    for oy in range(ys.shape[1]):
+        for ox in range(ys.shape[2]):
+            iy, ix = oy + kh - 1 - ph, ox - pw
+            want1 = xs[0, iy, ix, 0] if (0 <= iy < 10 and 0 <= ix < 9) else 0.0
+            assert ys[0, oy, ox, 0] == want1
+
+
+@pytest.mark.parametrize("k,s,p", [(3, 1, 1), (3, 2, 0), (5, 3, 2), (2, 2, 0)])
+def test_average_pool_against_library_routine(k, s, p):
+    x = R.standard_normal((2, 9, 8, 3)).astype(np.float32)
+    xt = torch.from_numpy(x.astype(np.float64)).permute(0, 3, 1, 2)
+    want = torch.nn.functional.avg_pool2d(xt, k, s, p, count_include_pad=True).permute(0, 2, 3, 1).numpy()
+    np.testing.assert_allclose(ref.avgpool(x, k, s, p), want.astype(np.float32), rtol=0, atol=1e-7)
+    # constant map: a corner window of a padded 3x3 pool sees 4 of 9 taps
+    if (k, s, p) == (3, 1, 1):
+        c = ref.avgpool(np.ones((1, 4, 4, 1), np.float32), 3, 1, 1)
+        assert c[0, 0, 0, 0] == np.float32(4.0 / 9.0) and c[0, 1, 1, 0] == 1.0 and c[0, 0, 1, 0] == np.float32(6.0 / 9.0)
+
+
+def _requant_res_exact(acc, m, b, r, rs, act):
+    accf = _to_f32_exact(Fraction(acc))
+    t = _to_f32_exact(accf * Fraction(float(np.float32(m))) + Fraction(float(np.float32(b))))
+    t = _to_f32_exact(Fraction(int(r)) * Fraction(float(np.float32(rs))) + t)
+    if act == "relu" and t < 0:
+        t = Fraction(0)
+    tf = t
+    t = min(max(t, Fraction(-127)), Fraction(127))
+    return _round_half_even(t), tf
+
+
+def test_requant_with_int8_residual_against_exact_rational_arithmetic():
+    accs = [0, 1, -1, 3, 5, 127, 255, 2 ** 24 + 1, -(2 ** 24) - 3, 33554433, 400000001]
+    accs += [int(v) for v in R.integers(-40000, 40000, size=150)]
+    for acc in accs:
+        for m in (0.5, 1e-3, 0.0123456, 1.0 / 3.0):
+            for b in (0.0, 0.5, -3.3):
+                for r in (-127, -1, 0, 1, 3, 127):
+                    for rs in (0.5, 0.75, 1.0 / 3.0, 1.37):
+                        for act in ("none", "relu"):
+                            q, tf = _requant_res_exact(acc, m, b, r, rs, act)
+                            assert ref.requant_res_s8(acc, m, b, r, rs, act) == q, (acc, m, b, r, rs, act)
+                            assert Fraction(float(ref.requant_res_f32(acc, m, b, r, rs, act))) == tf
+    # literals: halves round to even AFTER the residual joined (0.5*1 + 0 + 0.5*2 = 1.5 -> 2; 2.5 -> 2)
+    assert ref.requant_res_s8(1, 0.5, 0.0, 2, 0.5, "none") == 2
+    assert ref.requant_res_s8(3, 0.5, 0.0, 2, 0.5, "none") == 2
+    assert ref.requant_res_s8(-9, 0.5, 0.0, 2, 0.5, "relu") == 0
+    assert ref.requant_res_s8(100, 1.0, 0.0, 127, 1.0, "none") == 127
+
+
+def test_int8_conv_with_residual_is_the_scalar_rule_per_element():
+    xq = R.integers(-127, 128, size=(1, 5, 5, 4)).astype(np.int8)
+    wq = R.integers(-127, 128, size=(6, 3, 3, 4)).astype(np.int8)
+    rq = R.integers(-127, 128, size=(1, 5, 5, 6)).astype(np.int8)
+    m = (R.random(6) * 1e-3 + 1e-4).astype(np.float32)
+    b = R.standard_normal(6).astype(np.float32)
+    acc = ref.conv2d_s8(xq, wq, None, 1, 1, out="s32")
+    yq = ref.conv2d_s8(xq, wq, None, 1, 1, m=m, b=b, act="relu", out="s8", residual=rq, residual_scale=0.6)
+    yf = ref.conv2d_s8(xq, wq, None, 1, 1, m=m, b=b, act="none", out="f32", residual=rq, residual_scale=0.6)
+    for idx in np.ndindex(acc.shape):
+        co = idx[-1]
+        assert yq[idx] == ref.requant_res_s8(int(acc[idx]), m[co], b[co], int(rq[idx]), 0.6, "relu")
+        assert yf[idx] == ref.requant_res_f32(int(acc[idx]), m[co], b[co], int(rq[idx]), 0.6, "none")

@@ -20,7 +20,7 @@ from . import gen
 
 @dataclass
 class Op:
-    kind: str                      # 'conv' | 'fc' | 'maxpool' | 'gavgpool'
+    kind: str                      # 'conv' | 'fc' | 'maxpool' | 'avgpool' | 'gavgpool'
     name: str
     src: int
     dst: int
@@ -40,6 +40,10 @@ class Op:
     density: float = 1.0
     in_hw: Tuple[int, int] = (0, 0)
     out_hw: Tuple[int, int] = (0, 0)
+    pad_w: int = -1                # padding along the width when it differs from `pad` (rectangular kernels)
+    res_scale: float = 0.0         # int8 residual: s_r / s_y
+    dst_off: int = 0               # first channel of dst this op writes (channel concatenation)
+    dst_total: int = 0             # channels of the dst slot; 0 = the op's own c_out
 
     @property
     def nnz(self):
