@@ -154,6 +154,7 @@ cadnn_status cadnn_weights_warp_loads(const cadnn_weights *w, int64_t *loads, in
 cadnn_status cadnn_weights_unpack(const cadnn_weights *w, float *dense_f32, uint8_t *mask);
 
 void cadnn_weights_free(cadnn_weights *w);
+void cadnn_free_weights(cadnn_weights *w); /* the same call under the name the problem statement uses */
 
 /*
  * Fused epilogue (Section 4, "Model computation fusion": Conv/DWConv + BatchNorm +
@@ -266,7 +267,10 @@ cadnn_status cadnn_forward(cadnn_net *net, const void *x, void *y, int use_graph
  * cadnn_forward_host - the same network run from HOST buffers: copies x_host
  * ([n][h][w][c], pinned memory recommended) to a device staging buffer the net owns
  * (allocated on the first call), runs the network, copies the output to y_host and
- * synchronizes stream before returning.
+ * synchronizes stream before returning.  Every wait inside a kernel is bounded; the words in
+ * which kernels count waits that ran out are read in stream order behind the output, and
+ * CADNN_E_DEVICE_STATUS is returned (y_host is then not to be trusted) when one of them moved
+ * since this net last looked.
  */
 cadnn_status cadnn_forward_host(cadnn_net *net, const void *x_host, void *y_host, int use_graph, void *stream);
 
@@ -326,6 +330,10 @@ cadnn_status cadnn_net_layout(const cadnn_net *net, int *planar, int *persistent
  */
 cadnn_status cadnn_net_layer_times(cadnn_net *net, const void *x, void *y, int flush_l2, int reps, float *ms,
                                    void *stream);
+/* The same for the single op `op`: ms (host) receives one value.  Both return
+ * CADNN_E_DEVICE_STATUS like cadnn_forward_host when a kernel's bounded wait ran out. */
+cadnn_status cadnn_net_layer_time(cadnn_net *net, int op, const void *x, void *y, int flush_l2, int reps, float *ms,
+                                  void *stream);
 
 /*
  * cadnn_device_status - health flags the kernels leave on the current device (the paper has no
@@ -335,6 +343,25 @@ cadnn_status cadnn_net_layer_times(cadnn_net *net, const void *x, void *y, int f
  * the device.  Errors: E_ARG, E_CUDA.
  */
 cadnn_status cadnn_device_status(int *copy_timeouts);
+
+/*
+ * cadnn_debug_set_device_status - overwrite the two device words in which kernels count waits
+ * that ran out (copy barriers; the persistent kernel's grid barrier).  For tests of the error
+ * path only: it lets a test see CADNN_E_DEVICE_STATUS without making any kernel wait.  The
+ * paper has no counterpart.  Synchronous.
+ */
+cadnn_status cadnn_debug_set_device_status(int copy_timeouts, int barrier_timeouts);
+
+/*
+ * cadnn_measure_alu_peak - measurement aid: the multiply-add rate the plain ALUs of the current
+ * device sustain, in operations per second (a multiply-add counts 2), from a kernel that does
+ * nothing but independent chains of fused multiply-adds.  dtype CADNN_F32: the FP32 lanes (FFMA);
+ * CADNN_S8: the 32-bit integer multiply-add the int8 kernels issue.  This is the compute-side
+ * denominator of the sparse roofline (the paper has no counterpart; its Section 5 reports
+ * latencies only).  Allocates and frees a small scratch buffer; runs a few milliseconds;
+ * synchronizes stream.
+ */
+cadnn_status cadnn_measure_alu_peak(int dtype, double *ops_per_second, void *stream);
 
 /* Device pointer and byte size of slot `slot` (for per-layer inspection). */
 cadnn_status cadnn_net_slot(const cadnn_net *net, int slot, void **ptr, int64_t *bytes);

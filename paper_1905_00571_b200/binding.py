@@ -56,6 +56,7 @@ _SIGS = {
     "cadnn_weights_warp_loads": (_i, [_vp, _i64p, _i, ctypes.POINTER(_i)]),
     "cadnn_weights_unpack": (_i, [_vp, _vp, _vp]),
     "cadnn_weights_free": (None, [_vp]),
+    "cadnn_free_weights": (None, [_vp]),
     "cadnn_conv2d": (_i, [_vp, _vp, _i, _i, _i, _vp, ctypes.POINTER(Epilogue), _vp]),
     "cadnn_conv2d_planar": (_i, [_vp, _vp, _i, _vp, ctypes.POINTER(Epilogue), _vp]),
     "cadnn_fc": (_i, [_vp, _vp, _i, _vp, ctypes.POINTER(Epilogue), _vp]),
@@ -68,6 +69,9 @@ _SIGS = {
     "cadnn_net_info": (_i, [_vp, ctypes.POINTER(_i), _i64p]),
     "cadnn_net_layout": (_i, [_vp, ctypes.POINTER(_i), ctypes.POINTER(_i)]),
     "cadnn_net_layer_times": (_i, [_vp, _vp, _vp, _i, _i, ctypes.POINTER(ctypes.c_float), _vp]),
+    "cadnn_net_layer_time": (_i, [_vp, _i, _vp, _vp, _i, _i, ctypes.POINTER(ctypes.c_float), _vp]),
+    "cadnn_debug_set_device_status": (_i, [_i, _i]),
+    "cadnn_measure_alu_peak": (_i, [_i, ctypes.POINTER(ctypes.c_double), _vp]),
     "cadnn_net_slot": (_i, [_vp, _i, ctypes.POINTER(_vp), _i64p]),
     "cadnn_net_free": (None, [_vp]),
     "cadnn_device_status": (_i, [ctypes.POINTER(_i)]),
@@ -328,6 +332,29 @@ def cadnn_net_layer_times(net, x, y, n_ops, flush_l2=False, reps=1, stream=None)
                                       _stream(stream)),
            "cadnn_net_layer_times")
     return [float(v) for v in ms]
+
+
+def cadnn_net_layer_time(net, op, x, y, flush_l2=False, reps=1, stream=None):
+    ms = ctypes.c_float()
+    _check(_lib.cadnn_net_layer_time(net.handle, int(op), _dev_ptr(x), _dev_ptr(y), 1 if flush_l2 else 0, int(reps),
+                                     ctypes.byref(ms), _stream(stream)), "cadnn_net_layer_time")
+    return float(ms.value)
+
+
+def cadnn_debug_set_device_status(copy_timeouts, barrier_timeouts):
+    _check(_lib.cadnn_debug_set_device_status(int(copy_timeouts), int(barrier_timeouts)), "cadnn_debug_set_device_status")
+
+
+def cadnn_free_weights(w):
+    """Alias of Weights.free (the C ABI exports both names)."""
+    w.free()
+
+
+def cadnn_measure_alu_peak(dtype="f32", stream=None):
+    """Measured multiply-add rate of the plain ALUs, operations per second (a multiply-add counts 2)."""
+    v = ctypes.c_double()
+    _check(_lib.cadnn_measure_alu_peak(DTYPE[dtype], ctypes.byref(v), _stream(stream)), "cadnn_measure_alu_peak")
+    return float(v.value)
 
 
 def cadnn_net_slot(net, slot):

@@ -2,6 +2,7 @@
 // kernel the packer scheduled.  No arithmetic lives here.
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include "cadnn_internal.h"
 
 namespace {
@@ -13,6 +14,20 @@ cadnn_status cadnn_note_cuda(cudaError_t e)
     snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
     cudaGetLastError();  // clear a non-sticky error so that later calls are not blamed for it
     return CADNN_E_CUDA;
+}
+
+cadnn_status raise_smem_limit(const void *kern, int smem, SmemLimit *lim)
+{
+    static std::mutex mu;
+    int dev = 0;
+    CADNN_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CADNN_E_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(mu);
+    const int have = lim->allowed[dev] > 0 ? lim->allowed[dev] : 48 * 1024;
+    if (smem <= have) return CADNN_OK;
+    CADNN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    lim->allowed[dev] = smem;
+    return CADNN_OK;
 }
 
 namespace {
@@ -43,6 +58,20 @@ cadnn_status check_epilogue(const cadnn_weights *w, const cadnn_epilogue *ep, La
 }
 
 }  // namespace
+
+cadnn_status check_layer_call(const cadnn_weights *w, bool has_residual, int act, int out_dtype)
+{
+    if (!w || !w->on_device) return CADNN_E_ARG;
+    int dev = -1;
+    CADNN_CUDA_TRY(cudaGetDevice(&dev));
+    if (w->device != dev) return CADNN_E_ARG;   // packed on another GPU
+    cadnn_epilogue ep;
+    alignas(16) static const char some_residual[16] = {0};   // only its presence matters here
+    ep.scale = nullptr; ep.bias = nullptr; ep.residual = has_residual ? some_residual : nullptr;
+    ep.act = act; ep.out_dtype = out_dtype;
+    LaunchEpilogue le;
+    return check_epilogue(w, &ep, le);
+}
 
 cadnn_status conv2d_impl(const cadnn_weights *w, const void *x, int n, int h, int wd, void *y, const cadnn_epilogue *ep,
                          bool pdl, cudaStream_t s)
@@ -121,6 +150,15 @@ cadnn_status cadnn_device_status(int *copy_timeouts)
     *copy_timeouts = copies + barriers;
     return CADNN_OK;
 }
+
+cadnn_status cadnn_debug_set_device_status(int copy_timeouts, int barrier_timeouts)
+{
+    cadnn_status s = write_copy_timeouts(copy_timeouts);
+    if (s != CADNN_OK) return s;
+    return write_barrier_timeouts(barrier_timeouts);
+}
+
+void cadnn_free_weights(cadnn_weights *w) { cadnn_weights_free(w); }
 
 const char *cadnn_status_str(cadnn_status s)
 {

@@ -154,6 +154,18 @@ cadnn_status cadnn_note_cuda(cudaError_t e);
         if (e__ != cudaSuccess) return cadnn_note_cuda(e__);  \
     } while (0)
 
+// Dynamic shared memory above 48 KB has to be allowed per kernel AND per device.  One
+// SmemLimit per kernel instantiation remembers, for each device, what has been allowed;
+// raise_smem_limit raises it when a launch needs more (serialized by one mutex).
+const int kMaxDevices = 64;
+struct SmemLimit {
+    int allowed[kMaxDevices];   // zero = the default 48 KB
+};
+cadnn_status raise_smem_limit(const void *kern, int smem, SmemLimit *lim);
+
+// epilogue / device checks of one layer call (no launch): what conv2d_impl would refuse
+cadnn_status check_layer_call(const cadnn_weights *w, bool has_residual, int act, int out_dtype);
+
 // kernel launchers (each validates nothing; callers did)
 cadnn_status launch_sconv(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
                           cudaStream_t st);
@@ -172,6 +184,11 @@ cadnn_status launch_dw_planar(const cadnn_weights *w, const void *x, int n, void
                               cudaStream_t st);
 cadnn_status read_copy_timeouts(int *count);
 cadnn_status read_barrier_timeouts(int *count);
+// the same counters copied to (pinned) host memory in stream order, and overwritten (tests)
+cadnn_status read_copy_timeouts_async(int *host_dst, cudaStream_t st);
+cadnn_status read_barrier_timeouts_async(int *host_dst, cudaStream_t st);
+cadnn_status write_copy_timeouts(int value);
+cadnn_status write_barrier_timeouts(int value);
 
 // Persistent kernel over a run of planar sparse convs (persist.cu).  One entry per conv, in
 // network order; join_phase: the op reads nothing that the ops of the current phase write, so
@@ -235,6 +252,23 @@ __device__ __forceinline__ unsigned fdiv(unsigned n, const FastDiv &f)
 // until grid_dep_wait() returns.  Without the attribute both calls do nothing.
 __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
 __device__ __forceinline__ void grid_dep_trigger() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+
+// Activations and residuals may have been written by the kernel this one depends on
+// programmatically, i.e. while this kernel was already running: they are read with ordinary
+// loads.  The read-only path (ld.global.nc / __ldg) promises data that is constant for the whole
+// lifetime of the kernel and is kept for weights, scales and biases.
+__device__ __forceinline__ float ld_act(const float *p)
+{
+    float v;
+    asm volatile("ld.global.f32 %0, [%1];\n" : "=f"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ signed char ld_act(const signed char *p)
+{
+    int v;
+    asm volatile("ld.global.s8 %0, [%1];\n" : "=r"(v) : "l"(p));
+    return (signed char)v;
+}
 
 template <typename... KArgs, typename... Args>
 cadnn_status launch_kernel(void (*kern)(KArgs...), int blocks, int threads, size_t smem, bool pdl, cudaStream_t st,

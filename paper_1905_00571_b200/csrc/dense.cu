@@ -398,11 +398,11 @@ cadnn_status launch_dense_smallc(const cadnn_weights *w, const void *x, int n, v
     if (blocks <= 0) return CADNN_OK;
     if (blocks > 2147483647LL) return CADNN_E_UNSUPPORTED;
     size_t smem = ((size_t)p.taps * kStemCoBlock + (size_t)p.in_rows * p.in_cols * d.c_in) * 4;
-    static size_t smem_allowed = 48 * 1024;
-    if (smem > smem_allowed) {
+    static SmemLimit lim;
+    if (smem > 48 * 1024) {
         if (smem > 200 * 1024) return CADNN_E_UNSUPPORTED;
-        CADNN_CUDA_TRY(cudaFuncSetAttribute(stem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        smem_allowed = smem;
+        cadnn_status rs = raise_smem_limit((const void *)stem_kernel, (int)smem, &lim);
+        if (rs != CADNN_OK) return rs;
     }
     return launch_kernel(stem_kernel, (int)blocks, 256, smem, ep.pdl, st, p);
 }

@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(256) fc_spmv_kernel(const FcParams p)
             const int k = p.idx[e];
 #pragma unroll
             for (int b = 0; b < NB; ++b)
-                if (b0 + b < p.n) acc[b] += wv * (AT)__ldg(x + (size_t)(b0 + b) * p.k + k);
+                if (b0 + b < p.n) acc[b] += wv * (AT)ld_act(x + (size_t)(b0 + b) * p.k + k);
         }
 #pragma unroll
         for (int b = 0; b < NB; ++b)

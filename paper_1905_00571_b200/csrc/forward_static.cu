@@ -23,7 +23,6 @@ static __device__ __align__(256) unsigned char g_arena[CADNN_STATIC_WORKSPACE_BY
 
 // In host code `g_arena` is only a handle for the runtime's symbol calls; its device
 // address has to be asked for, once per device, with that device current.
-const int kMaxDevices = 64;
 std::mutex g_mu;
 unsigned char *g_arena_dev[kMaxDevices] = {nullptr};
 
@@ -146,6 +145,11 @@ cadnn_status cadnn_forward_static(const cadnn_op *ops, int n_ops, int n, int h, 
                 if (!sr.defined || sr.h != so.h || sr.w != so.w || sr.c != so.c || sr.dtype != so.dtype)
                     return CADNN_E_SHAPE;
             }
+            // everything the layer call itself would refuse is refused here, before the first launch:
+            // the epilogue combination, weights packed on another GPU, an input beyond the staging limit
+            cadnn_status cs = check_layer_call(op.w, op.res >= 0, op.act, op.out_dtype);
+            if (cs != CADNN_OK) return cs;
+            if ((long long)si.n * si.h * si.w * si.c * dtype_size(si.dtype) >= (1LL << 34)) return CADNN_E_UNSUPPORTED;
         } else if (op.kind == CADNN_OP_MAXPOOL) {
             if (op.pool_k < 1 || op.pool_stride < 1 || op.pool_pad < 0 || op.pool_pad >= op.pool_k ||
                 si.h + 2 * op.pool_pad < op.pool_k || si.w + 2 * op.pool_pad < op.pool_k)

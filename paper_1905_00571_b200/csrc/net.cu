@@ -42,6 +42,10 @@ struct cadnn_net {
     // L2 flush buffer for layer timing
     void *flush = nullptr;
     size_t flush_bytes = 0;
+    // device status words (bounded waits that ran out): pinned host copy written in stream order
+    // at the net's synchronization points, and the values seen when the net was created
+    int *status_host = nullptr;
+    int status_seen[2] = {0, 0};
 };
 
 namespace {
@@ -277,6 +281,25 @@ cadnn_status forward_impl(cadnn_net *net, const void *x, void *y, int use_graph,
     return CADNN_OK;
 }
 
+// The kernels' waits are bounded; one that ran out leaves a count in a device word.  The net
+// reads the words in stream order right before it synchronizes, so a forward whose kernels gave
+// up is reported instead of returning wrong numbers silently.
+cadnn_status queue_status_read(cadnn_net *net, cudaStream_t st)
+{
+    cadnn_status s = read_copy_timeouts_async(&net->status_host[0], st);
+    if (s == CADNN_OK && net->persist) s = read_barrier_timeouts_async(&net->status_host[1], st);
+    return s;
+}
+
+// after the stream has been synchronized: did a counter move since the net last looked?
+bool status_moved(cadnn_net *net)
+{
+    const bool moved = net->status_host[0] != net->status_seen[0] || net->status_host[1] != net->status_seen[1];
+    net->status_seen[0] = net->status_host[0];
+    net->status_seen[1] = net->status_host[1];
+    return moved;
+}
+
 __global__ void flush_kernel(float *buf, size_t n)
 {
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
@@ -324,6 +347,8 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
                 const bool stem = op.w->s.kind == KK_DENSE_SMALLC && op.src == 0 && op.res < 0;
                 const bool dw = dw_planar_ok(op.w) && op.res < 0 && op.src != 0 && !flat[op.src] && getenv("CADNN_NO_PLANAR_DW") == nullptr;
                 if (!stem && !dw && (!op.w->has_planar || op.src == 0 || flat[op.src])) planar = false;
+                // a residual must be a padded planar tensor too: not the NHWC input, not an [n][c] vector
+                if (op.res == 0 || (op.res > 0 && flat[op.res])) planar = false;
             } else if (op.kind == CADNN_OP_FC) {
                 if (!flat[op.src]) planar = false;
                 flat[op.dst] = 1;
@@ -371,6 +396,9 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
                     break;
                 }
             }
+            // what the layer call would refuse (epilogue combination, weights of another GPU) is refused now
+            st = check_layer_call(op.w, op.res >= 0, op.act, op.out_dtype);
+            if (st != CADNN_OK) break;
         } else if (op.kind == CADNN_OP_MAXPOOL) {
             if (op.pool_k < 1 || op.pool_stride < 1 || op.pool_pad < 0 || op.pool_pad >= op.pool_k ||
                 si.h + 2 * op.pool_pad < op.pool_k || si.w + 2 * op.pool_pad < op.pool_k) { st = CADNN_E_SHAPE; break; }
@@ -403,6 +431,17 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
         return st;
     }
     net->out_bytes = net->slots[net->out_slot].bytes;
+    if (cudaHostAlloc((void **)&net->status_host, 2 * sizeof(int), cudaHostAllocDefault) != cudaSuccess) {
+        cudaGetLastError();
+        cadnn_net_free(net);
+        return CADNN_E_ALLOC;
+    }
+    if (read_copy_timeouts(&net->status_seen[0]) != CADNN_OK || read_barrier_timeouts(&net->status_seen[1]) != CADNN_OK) {
+        cadnn_net_free(net);
+        return CADNN_E_CUDA;
+    }
+    net->status_host[0] = net->status_seen[0];
+    net->status_host[1] = net->status_seen[1];
     // inside graphs, programmatic launches pay off for the planar kernels only (the NHWC sparse conv
     // measured slower with them: 556 -> 608 us on ResNet-50, 367 -> 410 us on the int8 VGG-16)
     if (!net->planar && getenv("CADNN_PDL_GRAPH") == nullptr) net->pdl_graph = false;
@@ -436,8 +475,10 @@ cadnn_status cadnn_forward_host(cadnn_net *net, const void *x_host, void *y_host
     cadnn_status s = forward_impl(net, net->stage_x, net->stage_y, use_graph, st, 1);
     if (s != CADNN_OK) return s;
     CADNN_CUDA_TRY(cudaMemcpyAsync(y_host, net->stage_y, (size_t)net->out_bytes, cudaMemcpyDeviceToHost, st));
+    s = queue_status_read(net, st);
+    if (s != CADNN_OK) return s;
     CADNN_CUDA_TRY(cudaStreamSynchronize(st));
-    return CADNN_OK;
+    return status_moved(net) ? CADNN_E_DEVICE_STATUS : CADNN_OK;
 }
 
 cadnn_status cadnn_net_info(const cadnn_net *net, int *n_launches, int64_t *workspace_bytes)
@@ -456,12 +497,10 @@ cadnn_status cadnn_net_layout(const cadnn_net *net, int *planar, int *persistent
     return CADNN_OK;
 }
 
-cadnn_status cadnn_net_layer_times(cadnn_net *net, const void *x, void *y, int flush_l2, int reps, float *ms,
-                                   void *stream)
+static cadnn_status layer_times_range(cadnn_net *net, const void *x, void *y, int flush_l2, int reps, float *ms,
+                                      size_t op_lo, size_t op_hi, cudaStream_t st)
 {
-    if (!net || !x || !y || !ms || reps < 1) return CADNN_E_ARG;
-    cudaStream_t st = (cudaStream_t)stream;
-    const size_t nops = net->ops.size();
+    const size_t nops = op_hi;
     if (flush_l2 && !net->flush) {
         net->flush_bytes = 256u << 20;
         CADNN_CUDA_TRY(cudaMalloc(&net->flush, net->flush_bytes));
@@ -475,7 +514,7 @@ cadnn_status cadnn_net_layer_times(cadnn_net *net, const void *x, void *y, int f
     cudaEvent_t e0, e1;
     cudaEventCreate(&e0);
     cudaEventCreate(&e1);
-    for (size_t i = 0; i < nops && s == CADNN_OK; ++i) {
+    for (size_t i = op_lo; i < nops && s == CADNN_OK; ++i) {
         // a graph of `reps` back-to-back launches of this op: the host launch cost stays out of the timing
         cudaGraph_t g = nullptr;
         cudaGraphExec_t ge = nullptr;
@@ -494,8 +533,8 @@ cadnn_status cadnn_net_layer_times(cadnn_net *net, const void *x, void *y, int f
             e = cudaStreamSynchronize(st);
             if (e != cudaSuccess) s = cadnn_note_cuda(e);
             else {
-                cudaEventElapsedTime(&ms[i], e0, e1);
-                ms[i] /= (float)reps;
+                cudaEventElapsedTime(&ms[i - op_lo], e0, e1);
+                ms[i - op_lo] /= (float)reps;
             }
         }
         if (ge) cudaGraphExecDestroy(ge);
@@ -504,7 +543,26 @@ cadnn_status cadnn_net_layer_times(cadnn_net *net, const void *x, void *y, int f
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);
     cudaStreamDestroy(cap);
+    if (s == CADNN_OK) {
+        s = queue_status_read(net, st);
+        if (s == CADNN_OK && cudaStreamSynchronize(st) != cudaSuccess) s = cadnn_note_cuda(cudaGetLastError());
+        if (s == CADNN_OK && status_moved(net)) s = CADNN_E_DEVICE_STATUS;
+    }
     return s;
+}
+
+cadnn_status cadnn_net_layer_times(cadnn_net *net, const void *x, void *y, int flush_l2, int reps, float *ms,
+                                   void *stream)
+{
+    if (!net || !x || !y || !ms || reps < 1) return CADNN_E_ARG;
+    return layer_times_range(net, x, y, flush_l2, reps, ms, 0, net->ops.size(), (cudaStream_t)stream);
+}
+
+cadnn_status cadnn_net_layer_time(cadnn_net *net, int op, const void *x, void *y, int flush_l2, int reps, float *ms,
+                                  void *stream)
+{
+    if (!net || !x || !y || !ms || reps < 1 || op < 0 || op >= (int)net->ops.size()) return CADNN_E_ARG;
+    return layer_times_range(net, x, y, flush_l2, reps, ms, (size_t)op, (size_t)op + 1, (cudaStream_t)stream);
 }
 
 cadnn_status cadnn_net_slot(const cadnn_net *net, int slot, void **ptr, int64_t *bytes)
@@ -525,6 +583,7 @@ void cadnn_net_free(cadnn_net *net)
     for (SlotInfo &s : net->slots)
         if (s.ptr) cudaFree(s.ptr);
     if (net->flush) cudaFree(net->flush);
+    if (net->status_host) cudaFreeHost(net->status_host);
     persist_free(net->persist);
     delete net;
 }

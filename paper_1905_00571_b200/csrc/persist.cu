@@ -41,6 +41,18 @@ cadnn_status read_barrier_timeouts(int *count)
     return CADNN_OK;
 }
 
+cadnn_status read_barrier_timeouts_async(int *host_dst, cudaStream_t st)
+{
+    CADNN_CUDA_TRY(cudaMemcpyFromSymbolAsync(host_dst, g_barrier_timeout, sizeof(int), 0, cudaMemcpyDeviceToHost, st));
+    return CADNN_OK;
+}
+
+cadnn_status write_barrier_timeouts(int value)
+{
+    CADNN_CUDA_TRY(cudaMemcpyToSymbol(g_barrier_timeout, &value, sizeof(int)));
+    return CADNN_OK;
+}
+
 namespace {
 
 const int kPersistWarps = 16;            // warps per block
@@ -74,14 +86,6 @@ __device__ __forceinline__ float pp_act(float z, int act)
     if (act == CADNN_ACT_RELU) return z > 0.0f ? z : 0.0f;
     if (act == CADNN_ACT_RELU6) return fminf(z > 0.0f ? z : 0.0f, 6.0f);
     return z;
-}
-
-// coherent global load (default caching; an acquire at device scope orders it)
-__device__ __forceinline__ float ld_act(const float *p)
-{
-    float v;
-    asm volatile("ld.global.f32 %0, [%1];\n" : "=f"(v) : "l"(p));
-    return v;
 }
 
 __device__ __forceinline__ unsigned ld_acquire(const unsigned *p)

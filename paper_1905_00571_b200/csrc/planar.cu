@@ -101,7 +101,7 @@ __global__ void __launch_bounds__(512) sconv_planar_kernel(const PlanarParams p)
             if (p.residual) {
 #pragma unroll
                 for (int t = 0; t < T; ++t)
-                    if (okmask & (1u << t)) res[t] = __ldg(p.residual + obase + 32 * t);
+                    if (okmask & (1u << t)) res[t] = ld_act(p.residual + obase + 32 * t);
             }
         }
         if (co >= 0) {
@@ -128,8 +128,8 @@ __global__ void __launch_bounds__(512) sconv_planar_kernel(const PlanarParams p)
                 for (int i = 0; i < P; ++i)
 #pragma unroll
                     for (int t = 0; t < T; ++t) {
-                        a[i][0][t] = __ldg(ximg + v[i].y + inb[t]);
-                        a[i][1][t] = __ldg(ximg + v[i].w + inb[t]);
+                        a[i][0][t] = ld_act(ximg + v[i].y + inb[t]);
+                        a[i][1][t] = ld_act(ximg + v[i].w + inb[t]);
                     }
 #pragma unroll
                 for (int i = 0; i < P; ++i) {
@@ -271,7 +271,7 @@ __global__ void __launch_bounds__(256) dw_planar_kernel(const DwPlanarParams p)
             const int ky = k / p.kw, kx = k - ky * p.kw;
             const int off = ky * p.wp_in + kx;
 #pragma unroll
-            for (int t = 0; t < T; ++t) acc[t] = fmaf(wv[k], __ldg(xp + inb[t] + off), acc[t]);
+            for (int t = 0; t < T; ++t) acc[t] = fmaf(wv[k], ld_act(xp + inb[t] + off), acc[t]);
         }
     }
     float *yp = p.y + (size_t)pl * p.plane_out + (size_t)p.halo * p.wp_out + q0 + lane;

@@ -42,6 +42,18 @@ cadnn_status read_copy_timeouts(int *count)
     return CADNN_OK;
 }
 
+cadnn_status read_copy_timeouts_async(int *host_dst, cudaStream_t st)
+{
+    CADNN_CUDA_TRY(cudaMemcpyFromSymbolAsync(host_dst, g_copy_timeout, sizeof(int), 0, cudaMemcpyDeviceToHost, st));
+    return CADNN_OK;
+}
+
+cadnn_status write_copy_timeouts(int value)
+{
+    CADNN_CUDA_TRY(cudaMemcpyToSymbol(g_copy_timeout, &value, sizeof(int)));
+    return CADNN_OK;
+}
+
 namespace {
 
 struct PsParams {
@@ -499,7 +511,7 @@ __global__ void __launch_bounds__(512) sconv_planar_tma_kernel(const PsParams p,
         for (int t = 0; t < T; ++t) {
             res[j][t] = 0.0f;
             if (p.residual && slice == 0 && co_of[j] >= 0 && (okmask & (1u << t)))
-                res[j][t] = __ldg(p.residual + ((size_t)img * p.c_out + co_of[j]) * p.pitch_out + q0 + lane + 32 * t);
+                res[j][t] = ld_act(p.residual + ((size_t)img * p.c_out + co_of[j]) * p.pitch_out + q0 + lane + 32 * t);
         }
     __syncthreads();   // the barriers are initialised for everyone
 
@@ -529,11 +541,10 @@ cadnn_status ps_launch_one(const PsParams &p, const CUtensorMap *map, int blocks
 {
     if (map) {
         auto kern = p.R > 0 ? sconv_planar_tma_kernel<T, RPW, true> : sconv_planar_tma_kernel<T, RPW, false>;
-        static int smem_allowed[2] = {48 * 1024, 48 * 1024};   // raised once per instantiation, as layers need it
-        int &allowed = smem_allowed[p.R > 0 ? 1 : 0];
-        if (smem > allowed) {
-            CADNN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-            allowed = smem;
+        static SmemLimit lim[2];   // per instantiation (row-tile / linear), per device
+        if (smem > 48 * 1024) {
+            cadnn_status rs = raise_smem_limit((const void *)kern, smem, &lim[p.R > 0 ? 1 : 0]);
+            if (rs != CADNN_OK) return rs;
         }
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)blocks, 1, 1);
@@ -560,10 +571,10 @@ cadnn_status ps_launch_one(const PsParams &p, const CUtensorMap *map, int blocks
         return CADNN_OK;
     }
     auto kern = sconv_planar_staged_kernel<T, RPW>;
-    static int smem_allowed = 48 * 1024;
-    if (smem > smem_allowed) {
-        CADNN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        smem_allowed = smem;
+    static SmemLimit lim;
+    if (smem > 48 * 1024) {
+        cadnn_status rs = raise_smem_limit((const void *)kern, smem, &lim);
+        if (rs != CADNN_OK) return rs;
     }
     return launch_kernel(kern, blocks, threads, (size_t)smem, pdl, st, p);
 }

@@ -501,10 +501,10 @@ template <typename XT, int T, int RPW>
 cadnn_status launch_one(const SconvParams &p, int blocks, int threads, int smem, bool pdl, cudaStream_t st)
 {
     auto kern = sconv_kernel<XT, T, RPW>;
-    static int smem_allowed = 48 * 1024;  // raised once per instantiation, as layers need it
-    if (smem > smem_allowed) {
-        CADNN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        smem_allowed = smem;
+    static SmemLimit lim;   // per instantiation, per device
+    if (smem > 48 * 1024) {
+        cadnn_status rs = raise_smem_limit((const void *)kern, smem, &lim);
+        if (rs != CADNN_OK) return rs;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)blocks, 1, 1);
