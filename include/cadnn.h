@@ -257,8 +257,11 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
  * graphs; NHWC networks use them inside graphs only with CADNN_PDL_GRAPH set, they measured
  * slower there).  In a captured graph an op whose result the next op does not read (a residual
  * block's downsample conv) becomes a parallel branch; CADNN_NO_FORK keeps one chain.
- * CADNN_PERSIST=1 (experimental, slower where measured) runs the whole run of planar sparse
- * convs as one cooperative kernel with device-wide barriers between layers.
+ * Planar networks run at a batch of up to 2 images execute their longest run of consecutive sparse
+ * convs as ONE persistent cooperative kernel (one thread block per SM, device-wide barriers between
+ * layers, every wait bounded): at such batches a layer's work is far below the cost of a kernel
+ * boundary.  CADNN_PERSIST=0 / 1 in the environment at cadnn_net_create forces it off / on for any
+ * batch.  The folded scale / bias vectors of those layers are read once, when the net is created.
  * Asynchronous on stream.
  */
 cadnn_status cadnn_forward(cadnn_net *net, const void *x, void *y, int use_graph, void *stream);
@@ -320,6 +323,23 @@ cadnn_status cadnn_net_info(const cadnn_net *net, int *n_launches, int64_t *work
  * Either pointer may be NULL.  Host ints.
  */
 cadnn_status cadnn_net_layout(const cadnn_net *net, int *planar, int *persistent_ops);
+
+/*
+ * Measurement aids for the persistent kernel (E_UNSUPPORTED when the net has none).
+ * cadnn_net_persistent_plan: what the host planner chose for op `op` (Section 4, "Optimization
+ * parameters selection"): plan[0..11] = bands of 32 positions per tile, bands per unit, filters per
+ * group, tiles, groups, staged floats per channel, channels per chunk, chunks per pass, passes,
+ * strided addressing, modelled clocks per item, phase.  Host ints.
+ * cadnn_net_persistent_profile: with CADNN_PERSIST_PROFILE set in the environment at
+ * cadnn_net_create, every launch records SM clock samples; after the last launch this returns,
+ * per phase (up to cap; *n_phases receives how many there are), the clocks from the phase's start to
+ * the next one's (mean over blocks), the longest / mean clocks a block spent on its own items, and
+ * the mean clocks until a block had issued its tile copies / until they had landed.  Any output
+ * pointer but n_phases may be NULL.  Synchronizes the device.
+ */
+cadnn_status cadnn_net_persistent_plan(const cadnn_net *net, int op, int plan[12]);
+cadnn_status cadnn_net_persistent_profile(const cadnn_net *net, int cap, float *wall_clk, float *busy_max_clk,
+                                          float *busy_mean_clk, float *issued_clk, float *landed_clk, int *n_phases);
 
 /*
  * Measurement aid: time every op on its own.  Each op is captured into a CUDA graph of

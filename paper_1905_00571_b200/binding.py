@@ -72,6 +72,8 @@ _SIGS = {
     "cadnn_net_layer_time": (_i, [_vp, _i, _vp, _vp, _i, _i, ctypes.POINTER(ctypes.c_float), _vp]),
     "cadnn_debug_set_device_status": (_i, [_i, _i]),
     "cadnn_measure_alu_peak": (_i, [_i, ctypes.POINTER(ctypes.c_double), _vp]),
+    "cadnn_net_persistent_plan": (_i, [_vp, _i, ctypes.POINTER(_i)]),
+    "cadnn_net_persistent_profile": (_i, [_vp, _i] + [ctypes.POINTER(ctypes.c_float)] * 5 + [ctypes.POINTER(_i)]),
     "cadnn_net_slot": (_i, [_vp, _i, ctypes.POINTER(_vp), _i64p]),
     "cadnn_net_free": (None, [_vp]),
     "cadnn_device_status": (_i, [ctypes.POINTER(_i)]),
@@ -355,6 +357,27 @@ def cadnn_measure_alu_peak(dtype="f32", stream=None):
     v = ctypes.c_double()
     _check(_lib.cadnn_measure_alu_peak(DTYPE[dtype], ctypes.byref(v), _stream(stream)), "cadnn_measure_alu_peak")
     return float(v.value)
+
+
+def cadnn_net_persistent_plan(net, op):
+    """Planner's choice for op `op` of the persistent run, or None if the op is not part of one."""
+    arr = (ctypes.c_int * 12)()
+    st = _lib.cadnn_net_persistent_plan(net.handle, int(op), arr)
+    if st == 4:
+        return None
+    _check(st, "cadnn_net_persistent_plan")
+    keys = ("TB", "T", "G", "tiles", "groups", "L", "CIc", "cpp", "passes", "strided", "est_clk", "phase")
+    return dict(zip(keys, list(arr)))
+
+
+def cadnn_net_persistent_profile(net, cap=256):
+    """Per phase of the persistent kernel's last launch: (wall clocks, longest block clocks, mean block clocks,
+    mean clocks until the tile copies were issued, until they had landed)."""
+    arrs = [(ctypes.c_float * cap)() for _ in range(5)]
+    n = ctypes.c_int()
+    _check(_lib.cadnn_net_persistent_profile(net.handle, cap, *arrs, ctypes.byref(n)), "cadnn_net_persistent_profile")
+    k = min(cap, n.value)
+    return [tuple(float(a[i]) for a in arrs) for i in range(k)]
 
 
 def cadnn_net_slot(net, slot):

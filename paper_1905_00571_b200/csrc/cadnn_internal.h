@@ -190,6 +190,12 @@ cadnn_status read_barrier_timeouts_async(int *host_dst, cudaStream_t st);
 cadnn_status write_copy_timeouts(int value);
 cadnn_status write_barrier_timeouts(int value);
 
+// Tensor map (a CUtensorMap, 128 bytes, 64-byte aligned, written to *map) over a float matrix of
+// `rows` channel planes by `cols` floats, copied in boxes of box_rows x box_cols; elements outside
+// the matrix read as zero.  False when the driver entry point is missing or refuses the shape.
+bool encode_plane_rows_map(void *map, const void *base, unsigned long long cols, unsigned long long rows,
+                           unsigned box_cols, unsigned box_rows);
+
 // Persistent kernel over a run of planar sparse convs (persist.cu).  One entry per conv, in
 // network order; join_phase: the op reads nothing that the ops of the current phase write, so
 // it may run in the same phase as its predecessor (no grid barrier between them).
@@ -204,10 +210,16 @@ struct PersistOpDesc {
     int act = 0;
     int n = 1;
     bool join_phase = false;
+    bool dst_external = false;   // y is read by something outside the run (or is the run's result)
 };
 cadnn_status persist_create(const std::vector<PersistOpDesc> &descs, PersistPlan **out);
 cadnn_status persist_launch(const PersistPlan *plan, cudaStream_t st);
 int persist_phases(const PersistPlan *plan);
+// plan of op `op` of the run: bands per tile, bands per unit, filters per group, tiles, groups, staged floats per
+// channel, channels per chunk, chunks per pass, passes, strided, modelled clocks, phase; 0 if there is no such op
+int persist_describe(const PersistPlan *plan, int op, int out[12]);
+cadnn_status persist_profile(const PersistPlan *plan, int cap, float *wall_clk, float *busy_max_clk, float *busy_mean_clk,
+                             float *issued_clk, float *landed_clk, int *n_out);
 void persist_free(PersistPlan *plan);
 cadnn_status launch_maxpool_planar(const float *x, int n, int h, int wd, int c, int k, int stride, int pad, float *y,
                                    bool pdl, cudaStream_t st);

@@ -197,7 +197,7 @@ void plan_persistent(cadnn_net *net)
     auto owned = [&](int slot) { return slot > 0 && slot != net->out_slot && net->slots[slot].ptr != nullptr; };
     auto eligible = [&](const cadnn_op &op) {
         return op.kind == CADNN_OP_CONV && op.w && op.w->has_planar && op.w->s.kind != KK_DENSE_SMALLC &&
-               op.w->d_pl_ent && owned(op.src) && owned(op.dst) && (op.res < 0 || owned(op.res));
+               !op.w->pl_ptr.empty() && owned(op.src) && owned(op.dst) && (op.res < 0 || owned(op.res));
     };
     int best_lo = -1, best_len = 0;
     for (int i = 0; i < n_ops;) {
@@ -221,6 +221,9 @@ void plan_persistent(cadnn_net *net)
         d.bias = op.bias;
         d.act = op.act;
         d.n = net->slots[op.src].n;
+        d.dst_external = i == best_lo + best_len - 1;
+        for (int j = 0; j < n_ops; ++j)
+            if ((j < best_lo || j >= best_lo + best_len) && (net->ops[j].src == op.dst || net->ops[j].res == op.dst)) d.dst_external = true;
         bool reads_phase = false;
         for (int s : phase_dsts) reads_phase = reads_phase || s == op.src || s == op.res;
         d.join_phase = !descs.empty() && !reads_phase && getenv("CADNN_PERSIST_NO_MERGE") == nullptr;
@@ -446,8 +449,11 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
     // measured slower with them: 556 -> 608 us on ResNet-50, 367 -> 410 us on the int8 VGG-16)
     if (!net->planar && getenv("CADNN_PDL_GRAPH") == nullptr) net->pdl_graph = false;
     {
-        const char *pe = getenv("CADNN_PERSIST");   // "0" / "1"; unset: off
-        if (net->planar && pe && atoi(pe) != 0) plan_persistent(net);
+        // the persistent kernel takes the launch ramp and drain out of every layer boundary, which is
+        // what a small batch pays for; larger batches keep one tuned kernel per layer
+        const char *pe = getenv("CADNN_PERSIST");   // "0" / "1"; unset: on for batches of up to 2 images
+        const bool want = pe ? atoi(pe) != 0 : n <= 2;
+        if (net->planar && want) plan_persistent(net);
     }
     *out = net;
     return CADNN_OK;
@@ -563,6 +569,22 @@ cadnn_status cadnn_net_layer_time(cadnn_net *net, int op, const void *x, void *y
 {
     if (!net || !x || !y || !ms || reps < 1 || op < 0 || op >= (int)net->ops.size()) return CADNN_E_ARG;
     return layer_times_range(net, x, y, flush_l2, reps, ms, (size_t)op, (size_t)op + 1, (cudaStream_t)stream);
+}
+
+cadnn_status cadnn_net_persistent_plan(const cadnn_net *net, int op, int plan[12])
+{
+    if (!net || !plan) return CADNN_E_ARG;
+    if (!net->persist || op < net->persist_first || op > net->persist_last) return CADNN_E_UNSUPPORTED;
+    return persist_describe(net->persist, op - net->persist_first, plan) ? CADNN_OK : CADNN_E_ARG;
+}
+
+cadnn_status cadnn_net_persistent_profile(const cadnn_net *net, int cap, float *wall_clk, float *busy_max_clk,
+                                          float *busy_mean_clk, float *issued_clk, float *landed_clk, int *n_phases)
+{
+    if (!net || !n_phases) return CADNN_E_ARG;
+    if (!net->persist) return CADNN_E_UNSUPPORTED;
+    CADNN_CUDA_TRY(cudaDeviceSynchronize());
+    return persist_profile(net->persist, cap, wall_clk, busy_max_clk, busy_mean_clk, issued_clk, landed_clk, n_phases);
 }
 
 cadnn_status cadnn_net_slot(const cadnn_net *net, int slot, void **ptr, int64_t *bytes)

@@ -59,12 +59,42 @@ def test_resnet50_full_batch1_persistent(monkeypatch):
     _check_logits(got, want)
 
 
-@pytest.mark.parametrize("T,ksw", [(1, 1), (2, 8), (8, 2), (4, 4)])
-def test_persistent_task_shapes(T, ksw, monkeypatch):
-    """Every (bands per lane, warps per filter) shape of the task loop, ragged tiles included."""
-    monkeypatch.setenv("CADNN_PERSIST_T", str(T))
-    monkeypatch.setenv("CADNN_PERSIST_KSW", str(ksw))
+@pytest.mark.parametrize("tb,grid,tile_kb", [(1, 0, 0), (2, 0, 0), (3, 40, 0), (4, 0, 0), (6, 0, 0), (8, 0, 0),
+                                             (0, 0, 4), (2, 33, 6), (1, 1, 0)])
+def test_persistent_item_shapes(tb, grid, tile_kb, monkeypatch):
+    """Every tile size of the item planner (ragged last tiles included), fewer blocks than items
+    (several items per block and phase), and a tile buffer so small that the input channels are
+    taken in several passes with partial sums parked in shared memory."""
+    if tb:
+        monkeypatch.setenv("CADNN_PERSIST_TB", str(tb))
+    if grid:
+        monkeypatch.setenv("CADNN_PERSIST_GRID", str(grid))
+    if tile_kb:
+        monkeypatch.setenv("CADNN_PERSIST_TILE_KB", str(tile_kb))
     m = models.resnet50(width=0.25, image=64, classes=100)
     x, got, info = _run(m, 2, True, True, monkeypatch)
+    if tb not in (6, 8):   # (tiles of 6 or 8 bands exceed what a stride-2 layer of this net can stage: no plan, layered run)
+        assert info["launches"] < len(m.ops) - 40, info
+    want, _ = oracle_forward.forward(m, x)
+    _check_logits(got, want)
+
+
+@pytest.mark.parametrize("no_parity", [False, True])
+def test_persistent_stride2_layouts(no_parity, monkeypatch):
+    """Stride-2 layers read parity planes written by their producer (default), or stage whole input rows
+    and address them with a lane stride (the fallback when the producer is not part of the run)."""
+    if no_parity:
+        monkeypatch.setenv("CADNN_PERSIST_NO_PARITY", "1")
+    m = models.resnet50(width=0.5, image=96, classes=100)
+    x, got, info = _run(m, 2, True, True, monkeypatch)
+    assert info["launches"] < len(m.ops) - 40, info
+    want, _ = oracle_forward.forward(m, x)
+    _check_logits(got, want)
+
+
+def test_persistent_odd_map_sizes(monkeypatch):
+    """Odd plane sizes at stride 2 (image 72: 18 -> 9 -> 5 -> 3) through the persistent kernel."""
+    m = models.resnet50(width=0.25, image=72, classes=100)
+    x, got, info = _run(m, 1, True, True, monkeypatch)
     want, _ = oracle_forward.forward(m, x)
     _check_logits(got, want)

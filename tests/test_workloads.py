@@ -72,3 +72,18 @@ def test_vgg16_reduced_health_and_full_counts():
     # conv1 has K = 27 at 8 %: some filters keep nothing at all
     c1 = models.vgg16(width=1.0, image=32, classes=10, fc_width=64).ops[0]
     assert (c1.mask.reshape(64, -1).sum(1) == 0).any()
+
+
+def test_mobilenet_v1_counts_and_health():
+    m = models.mobilenet_v1()
+    # 4.23 M parameters without BatchNorm vectors: stem 864, depthwise 13 layers, pointwise 13 layers, fc 1.024 M
+    assert sum(o.w.size for o in m.weight_ops()) == 4209088
+    dw = [o for o in m.ops if o.kind == "conv" and o.groups > 1]
+    pw = [o for o in m.ops if o.kind == "conv" and o.k == 1]
+    assert len(dw) == 13 and all(o.mask is None for o in dw) and len(pw) == 13
+    assert [o.stride for o in dw].count(2) == 4
+    y, slots = forward.forward(m, models.make_input(m, 1))
+    for op in m.ops:
+        sd = float(slots[op.dst].std())
+        assert 0.1 < sd < 10.0, (op.name, sd)
+    assert y.shape == (1, 1000) and np.isfinite(y).all()

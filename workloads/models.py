@@ -1,5 +1,5 @@
 """Synthetic networks shaped like the paper's workloads (Section 5, Table 2, and
-the VGGNet named in Section 3): ResNet-50 v1.5, VGG-16, MobileNet-V2.
+the VGGNet named in Section 3): ResNet-50 v1.5, VGG-16, MobileNet-V2, MobileNet-V1.
 
 A network is plain data: an ordered list of ops over numbered tensor slots
 (slot 0 is the input image).  Both the CPU oracle's network walker and the CUDA
@@ -188,6 +188,28 @@ def mobilenet_v2(seed=4, density=0.25, width=1.0, image=224, classes=1000):
     dst = m.new_slot()
     m.ops.append(Op("gavgpool", "avgpool", cur, dst, c_in=head, c_out=head, in_hw=(h, h), out_hw=(1, 1)))
     _f32_fc(m, g, "fc", dst, head, classes, density)
+    return m
+
+
+def mobilenet_v1(seed=5, density=0.25, width=1.0, image=224, classes=1000):
+    """MobileNet-V1 (Table 2 of the paper lists it next to V2): stem 3x3 s2 and the 13 depthwise 3x3
+    convs dense, the 13 pointwise 1x1 convs and the classifier magnitude-pruned to `density`;
+    ReLU after every conv."""
+    g = gen.rng(seed)
+    m = Model("mobilenet_v1", "f32", (image, image, 3), seed=seed)
+    ch = lambda c: max(8, int(round(c * width / 8.0)) * 8)
+    c_in = ch(32)
+    cur, h = _f32_conv(m, g, "stem", 0, 3, c_in, 3, 2, 1, image, "relu", 1.0)
+    cfg = [(64, 1), (128, 2), (128, 1), (256, 2), (256, 1), (512, 2), (512, 1), (512, 1), (512, 1), (512, 1), (512, 1),
+           (1024, 2), (1024, 1)]
+    for i, (c, st) in enumerate(cfg):
+        c = ch(c)
+        cur, h = _f32_conv(m, g, "b%d.dw" % (i + 1), cur, c_in, c_in, 3, st, 1, h, "relu", 1.0, groups=c_in)
+        cur, _ = _f32_conv(m, g, "b%d.pw" % (i + 1), cur, c_in, c, 1, 1, 0, h, "relu", density)
+        c_in = c
+    dst = m.new_slot()
+    m.ops.append(Op("gavgpool", "avgpool", cur, dst, c_in=c_in, c_out=c_in, in_hw=(h, h), out_hw=(1, 1)))
+    _f32_fc(m, g, "fc", dst, c_in, classes, density)
     return m
 
 
