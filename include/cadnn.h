@@ -257,11 +257,13 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
  * graphs; NHWC networks use them inside graphs only with CADNN_PDL_GRAPH set, they measured
  * slower there).  In a captured graph an op whose result the next op does not read (a residual
  * block's downsample conv) becomes a parallel branch; CADNN_NO_FORK keeps one chain.
- * Planar networks run at a batch of up to 2 images execute their longest run of consecutive sparse
- * convs as ONE persistent cooperative kernel (one thread block per SM, device-wide barriers between
- * layers, every wait bounded): at such batches a layer's work is far below the cost of a kernel
- * boundary.  CADNN_PERSIST=0 / 1 in the environment at cadnn_net_create forces it off / on for any
- * batch.  The folded scale / bias vectors of those layers are read once, when the net is created.
+ * CADNN_PERSIST=1 in the environment at cadnn_net_create makes a planar network execute its longest
+ * run of consecutive sparse convs as ONE persistent cooperative kernel (one thread block per SM, host-
+ * planned work items, device-wide barriers between layers, every wait bounded).  Measured it does not beat
+ * one tuned kernel per layer (see cadnn_net_persistent_profile), so it is off by default.  The folded
+ * scale / bias vectors of those layers are read once, when the net is created, and a map whose only
+ * reader is a stride-2 layer inside that kernel is kept as parity planes only (cadnn_net_slot then
+ * shows an unwritten buffer).
  * Asynchronous on stream.
  */
 cadnn_status cadnn_forward(cadnn_net *net, const void *x, void *y, int use_graph, void *stream);

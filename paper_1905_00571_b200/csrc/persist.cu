@@ -197,7 +197,7 @@ __device__ __forceinline__ void pn_grid_barrier(unsigned *arrive, unsigned targe
 {
     // The release is cumulative: the stores of the block's other threads, ordered before this thread by
     // the block barrier, are visible device-wide before the count moves; the acquire orders everything
-    // after it.  The tiles of the next phase are read by the copy unit, hence the proxy fence.
+    // after it.  (The writers ordered their stores against the copy unit's reads with a proxy fence.)
     red_release(arrive, 1u);
     unsigned spins = 0;
     while (ld_acquire(arrive) < target) {
@@ -206,7 +206,6 @@ __device__ __forceinline__ void pn_grid_barrier(unsigned *arrive, unsigned targe
             break;
         }
     }
-    asm volatile("fence.proxy.async.global;\n" ::: "memory");
 }
 
 // multiply-adds of entries [beg, end) of a unit (pairs; both even) against the staged tile
@@ -214,66 +213,44 @@ template <int T, bool STRIDED>
 __device__ __forceinline__ void pn_mac(const unsigned char *smem, unsigned ent, int beg, int end, unsigned tile,
                                        const unsigned (&lb)[T], float (&acc)[T])
 {
-    // Software pipeline over batches of P pairs of nonzeros: the nonzeros are read with broadcast loads
-    // two batches ahead and the activations of the NEXT batch are requested before the multiply-adds of
-    // the current one, so that a warp always has 2 P T shared-memory loads in flight behind its
-    // arithmetic (with four warps per scheduler nothing else hides their latency).  Slots past the end
-    // get weight 0; their offsets stay inside the tile (they are the next entries of the record, or its
-    // zero tail), and shared memory never holds anything but finite numbers.
+    // A batch of P pairs of nonzeros is read with broadcast loads one batch ahead; the batch's
+    // activation loads are all issued before its first multiply-add.  Slots past the end get weight 0;
+    // their offsets stay inside the tile (they are the next entries of the record, or its zero tail), and
+    // shared memory never holds anything but finite numbers.  (Requesting the NEXT batch's activations
+    // before the current multiply-adds measured no faster and costs loads on short rows.)
     constexpr int P = T == 1 ? 4 : 2;
+    uint4 nx[P];
+#pragma unroll
+    for (int i = 0; i < P; ++i) nx[i] = *reinterpret_cast<const uint4 *>(smem + ent + (beg + 2 * i) * 8);
     const unsigned base0 = tile + lb[0];
-    auto load_w = [&](uint4 (&w)[P], int e) {
+    for (int e = beg; e < end; e += 2 * P) {
+        uint4 v[P];
 #pragma unroll
-        for (int i = 0; i < P; ++i) w[i] = *reinterpret_cast<const uint4 *>(smem + ent + (e + 2 * i) * 8);
-    };
-    auto mask_w = [&](uint4 (&w)[P], int e) {
+        for (int i = 0; i < P; ++i) {
+            v[i] = nx[i];
+            if (e + 2 * i >= end) v[i].x = v[i].z = 0u;
+        }
 #pragma unroll
-        for (int i = 0; i < P; ++i)
-            if (e + 2 * i >= end) w[i].x = w[i].z = 0u;
-    };
-    auto load_a = [&](float (&a)[P][2][T], const uint4 (&w)[P]) {
+        for (int i = 0; i < P; ++i) nx[i] = *reinterpret_cast<const uint4 *>(smem + ent + (e + 2 * P + 2 * i) * 8);
+        float a[P][2][T];
 #pragma unroll
         for (int i = 0; i < P; ++i)
 #pragma unroll
             for (int t = 0; t < T; ++t) {
                 if (STRIDED) {
-                    a[i][0][t] = *reinterpret_cast<const float *>(smem + tile + lb[t] + w[i].y);
-                    a[i][1][t] = *reinterpret_cast<const float *>(smem + tile + lb[t] + w[i].w);
+                    a[i][0][t] = *reinterpret_cast<const float *>(smem + tile + lb[t] + v[i].y);
+                    a[i][1][t] = *reinterpret_cast<const float *>(smem + tile + lb[t] + v[i].w);
                 } else {
-                    a[i][0][t] = *reinterpret_cast<const float *>(smem + base0 + w[i].y + t * 128);
-                    a[i][1][t] = *reinterpret_cast<const float *>(smem + base0 + w[i].w + t * 128);
+                    a[i][0][t] = *reinterpret_cast<const float *>(smem + base0 + v[i].y + t * 128);
+                    a[i][1][t] = *reinterpret_cast<const float *>(smem + base0 + v[i].w + t * 128);
                 }
             }
-    };
-    uint4 v[P], nx[P];
-    float a[P][2][T];
-    load_w(v, beg);
-    mask_w(v, beg);
-    load_w(nx, beg + 2 * P);
-    load_a(a, v);
-    for (int e = beg; e < end; e += 2 * P) {
-        uint4 vn[P];
-        float an[P][2][T];
-#pragma unroll
-        for (int i = 0; i < P; ++i) vn[i] = nx[i];
-        mask_w(vn, e + 2 * P);
-        load_w(nx, e + 4 * P);
-        load_a(an, vn);
 #pragma unroll
         for (int i = 0; i < P; ++i) {
 #pragma unroll
             for (int t = 0; t < T; ++t) acc[t] = fmaf(__uint_as_float(v[i].x), a[i][0][t], acc[t]);
 #pragma unroll
             for (int t = 0; t < T; ++t) acc[t] = fmaf(__uint_as_float(v[i].z), a[i][1][t], acc[t]);
-        }
-#pragma unroll
-        for (int i = 0; i < P; ++i) {
-            v[i] = vn[i];
-#pragma unroll
-            for (int t = 0; t < T; ++t) {
-                a[i][0][t] = an[i][0][t];
-                a[i][1][t] = an[i][1][t];
-            }
         }
     }
 }
@@ -401,21 +378,22 @@ __device__ __forceinline__ void pn_compute(const PnItem &it, unsigned char *smem
         cpar ^= all_landed;   // every chunk barrier of the pass has been armed once
         if (p + 1 < passes) __syncthreads();   // the tile is free: the control warp stages the next pass
     }
+    // the maps this warp stored are read by the copy unit in a later phase
+    asm volatile("fence.proxy.async.global;\n" ::: "memory");
 }
 
-// control thread: start the copies of one pass of an item's tile
-__device__ __forceinline__ void pn_issue_pass(const PnItem &it, const PnMaps &maps, unsigned smem32, const PnLayout &lay, int p)
+// control warp: lane c starts the copies of chunk c of one pass of an item's tile (issuing a tensor copy
+// takes a few hundred clocks; the lanes' issues overlap)
+__device__ __forceinline__ void pn_issue_pass(const PnItem &it, const PnMaps &maps, unsigned smem32, const PnLayout &lay, int p, int c)
 {
     const CUtensorMap *map = &maps.m[it.layer];
     const unsigned box_bytes = (unsigned)(it.RB * it.L * 4);
     const unsigned chunk_bytes = box_bytes * (unsigned)it.nrb;
-    for (int c = 0; c < it.cpp; ++c) {
-        const unsigned bar = smem32 + lay.bars + 16 + c * 8;
-        pn_expect_tx(bar, chunk_bytes);
-        const int row = it.row0 + (p * it.cpp + c) * it.CIc;
-        for (int b = 0; b < it.nrb; ++b)
-            pn_tensor_copy(smem32 + lay.tile + c * chunk_bytes + b * box_bytes, map, it.x0, row + b * it.RB, bar);
-    }
+    const unsigned bar = smem32 + lay.bars + 16 + c * 8;
+    pn_expect_tx(bar, chunk_bytes);
+    const int row = it.row0 + (p * it.cpp + c) * it.CIc;
+    for (int b = 0; b < it.nrb; ++b)
+        pn_tensor_copy(smem32 + lay.tile + c * chunk_bytes + b * box_bytes, map, it.x0, row + b * it.RB, bar);
 }
 
 __global__ void __launch_bounds__(kPnThreads, 1)
@@ -472,14 +450,17 @@ net_persistent_kernel(const PnItem *items, const int *blk_first, const __grid_co
                 // the whole warp walks the same path (block barriers are warp-wide); lane 0 does the work
                 for (int p = 0; p < it.passes; ++p) {
                     if (p > 0) __syncthreads();   // the compute warps are done with the previous pass
+                    if (p > 0 && lane == 0) asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // reads of the tile before the unit's writes
+                    __syncwarp();
+                    if (lane < it.cpp) pn_issue_pass(it, maps, smem32, lay, p, lane);
+                    __syncwarp();
                     if (lane == 0) {
-                        if (p > 0) asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // reads of the tile before the unit's writes
-                        pn_issue_pass(it, maps, smem32, lay, p);
                         if (prof && p == 0) prof[((size_t)ph * 4 + 1) * gridDim.x + blockIdx.x] = clock64();
                         if (p == 0) prefetch(sel ^ 1);   // those buffers were released by the block barrier that ended the previous item
                         // every copy of the pass has landed before its barriers are armed again
                         for (int c = 0; c < it.cpp; ++c) pn_mbar_wait(smem32 + lay.bars + 16 + c * 8, (cpar >> c) & 1u);
                         if (prof && p + 1 == it.passes) prof[((size_t)ph * 4 + 2) * gridDim.x + blockIdx.x] = clock64();
+
                     }
                     cpar ^= (1u << it.cpp) - 1u;
                     __syncwarp();
@@ -596,21 +577,24 @@ void tile_extent(const PersistLayer &l, int b0, int nb, int *x0, int *len)
 }
 
 // Cost model (clock cycles) of one block's item, fitted to clock samples of the kernel on a B200:
-// a tile copy takes about 1500 clocks before its first bytes arrive and then moves ~50 bytes per clock;
-// the multiply-adds are bound by one shared-memory wavefront per clock and SM, and a single warp
-// walks about 100 clocks per batch of nonzeros.
-double item_cost(const PersistLayer &l, int TB, int T, int G, int L, int passes, int cpp, double nnz_avg)
+//  * the first bytes of a tile arrive ~2000 clocks into the phase, and with every SM copying at once the
+//    copies share ~3800 bytes per clock (26 per SM); a lone SM gets ~60;
+//  * a further pass over the channels waits for every warp and then for its own copies;
+//  * the multiply-adds are bound by one shared-memory wavefront per clock and SM, and a single warp walks
+//    about 100 clocks per batch of nonzeros.
+double item_cost(const PersistLayer &l, int TB, int T, int G, int L, int passes, int cpp, double nnz_avg, int active)
 {
+    const double rate = std::min(60.0, 3800.0 / std::max(1, active));
     const double bytes_pass = (double)l.c_in * L * 4.0 / passes;
-    const double t_first = 1500.0 + bytes_pass / cpp / 50.0;                    // first chunk in place
-    const double t_fill = passes * (2200.0 + bytes_pass / 50.0) + (passes - 1) * 3500.0;   // a further pass waits for every warp, then for its copies
+    const double t_first = 2000.0 + bytes_pass / cpp / rate;                    // first chunk in place
+    const double t_fill = passes * (2000.0 + bytes_pass / rate) + (passes - 1) * 3000.0;
     const int upf = ceil_div_i(TB, T);
     const double wave = (double)G * nnz_avg * (TB + 0.5 * upf) * 1.15;
     const int batch = T == 1 ? 8 : 4;
-    const double t_unit = 250.0 + (nnz_avg / batch + 1.0 + passes * cpp * 0.5) * 100.0 + (l.d.residual ? 150.0 : 0.0);
+    const double t_unit = 300.0 + (nnz_avg / batch + 1.0 + passes * cpp * 0.5) * 110.0 + (l.d.residual ? 150.0 : 0.0);
     const double t_path = (double)ceil_div_i(G * upf, kPnWarps) * t_unit * passes;
     const double t_comp = std::max(wave, t_path);
-    return std::max(t_fill, t_first + t_comp) + 400.0;
+    return std::max(t_fill + 0.35 * t_comp, t_first + t_comp) + 400.0;
 }
 
 // choose tile, groups and chunking of a layer that may use `budget` blocks
@@ -664,8 +648,10 @@ bool plan_layer(PersistLayer &l, int budget, int n_img, int tile_cap, int rec_ca
             if (passes > 1 && (long long)G * upf * T * 128 > 16 * 1024) continue;   // partial sums between passes
             const long long n_items = items_sp * groups;
             const double rounds = std::ceil((double)n_items / std::max(1, budget));
-            if (rounds > 8.0) break;
-            const double cost = rounds * item_cost(l, TB, T, G, L, passes, cpp, nnz_avg);
+            if (rounds > 64.0) break;
+            // (a further round starts only when a block's previous item is done: it pays the copy start-up again)
+            const double cost = rounds * item_cost(l, TB, T, G, L, passes, cpp, nnz_avg, (int)std::min<long long>(n_items, budget)) +
+                                (rounds - 1.0) * 1500.0;
             if (!found || cost < best) {
                 found = true;
                 best = cost;

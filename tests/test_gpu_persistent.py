@@ -60,7 +60,7 @@ def test_resnet50_full_batch1_persistent(monkeypatch):
 
 
 @pytest.mark.parametrize("tb,grid,tile_kb", [(1, 0, 0), (2, 0, 0), (3, 40, 0), (4, 0, 0), (6, 0, 0), (8, 0, 0),
-                                             (0, 0, 4), (2, 33, 6), (1, 1, 0)])
+                                             (0, 0, 16), (2, 33, 24), (1, 5, 0)])
 def test_persistent_item_shapes(tb, grid, tile_kb, monkeypatch):
     """Every tile size of the item planner (ragged last tiles included), fewer blocks than items
     (several items per block and phase), and a tile buffer so small that the input channels are
