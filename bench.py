@@ -52,7 +52,7 @@ class ClockSampler:
             os.close(fd)
             self.out = open(self.path, "w")
             self.proc = subprocess.Popen(["nvidia-smi", "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
-                                          "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+                                          "-lms", "20"], stdout=self.out, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -145,7 +145,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "images/s", "n_gpus": args.gpus,
             "steps": steps, "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64" if model.dtype == "f32" else "int32", "data": "synthetic",
-            "config": {"workload": wname, "batch": args.batch, "full_forward_s": full_s},
+            "config": {"workload": wname, "batch_per_gpu": args.batch, "full_forward_s": full_s},
             "cpu_baseline": {"value": value, "unit": "images/s", "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -246,7 +246,13 @@ def run_ours(args):
         t = pm.layer_times(x, y, flush_l2=False, reps=20)
         per = [p + v / reps for p, v in zip(per, t)]
     peaks = roofline.measured_peaks()
-    r_alu = roofline.alu_peak_tflops(peaks["sm_max_mhz"])
+    from paper_1905_00571_b200 import binding as B
+    r_alu_derived = roofline.alu_peak_tflops(peaks["sm_max_mhz"])
+    # the plain ALUs' multiply-add rate measured on this device (a kernel of nothing but FFMA / IMAD chains):
+    # the compute-side denominator of every fraction below
+    ffma_tflops = max(B.cadnn_measure_alu_peak("f32") for _ in range(2)) / 1e12
+    imad_tops = max(B.cadnn_measure_alu_peak("s8") for _ in range(2)) / 1e12
+    r_alu = imad_tops if model.dtype == "s8" else ffma_tflops
     rows_nom = roofline.network_roofline(model, batch, r_alu, roofline.HBM_NOMINAL_GBS)
     rows_meas = roofline.network_roofline(model, batch, r_alu, peaks["hbm_gbs"])
     fam = {}
@@ -263,7 +269,8 @@ def run_ours(args):
     if alu_bound:
         achieved = ft["flops"] / (ft["ms"] * 1e-3) / 1e12
         roof = {"bound": "alu", "achieved": achieved, "peak": r_alu, "unit": "TFLOP/s", "frac": achieved / r_alu,
-                "traffic": None, "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 x %.0f MHz" % peaks["sm_max_mhz"]}
+                "traffic": None, "peak_source": "measured: %s chains on this device" % ("IMAD" if model.dtype == "s8" else "FFMA"),
+                "frac_of_derived_peak": achieved / r_alu_derived}
     else:
         achieved = ft["bytes"] / (ft["ms"] * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -281,8 +288,26 @@ def run_ours(args):
               "frac_cold": t_roof_nom / (cold_ms * 1e3), "frac_warm": t_roof_nom / (warm_ms * 1e3),
               "frac_kernel_sum": t_roof_nom / (sum(per) * 1e3),
               "frac_3x3_layers": (sum(r["t_roof_us"] for r, _ in k3) / (sum(ms for _, ms in k3) * 1e3)) if k3 else None,
-              "alu_peak_tflops": r_alu,
+              "alu_peak_tflops": r_alu, "alu_peak_source": "measured",
+              "alu_peak_ffma_tflops_measured": ffma_tflops, "alu_peak_imad_tops_measured": imad_tops,
+              "alu_peak_tflops_derived": r_alu_derived,
+              "frac_warm_of_derived_peak": sum(r["t_roof_us"] for r in roofline.network_roofline(model, batch, r_alu_derived, roofline.HBM_NOMINAL_GBS)) / (warm_ms * 1e3),
               "families": {k: {"ms": v["ms"], "launches": v["launches"], "t_roof_us": v["t_roof_us"]} for k, v in fam.items()}}
+
+    # the throughput regime beside the latency-limited batch-1 number: kernel-only fraction of the pruned 3x3
+    # layers at batch 32 (schedules from the packer's time model; per-layer times as above)
+    if rank == 0 and world == 1 and args.workload == "resnet50" and not args.no_batch32:
+        pm32 = PackedModel(model, 32, dev, autotune=False)
+        x32 = torch.from_numpy(models.make_input(model, 32, seed=7)).to(dev)
+        y32 = pm32.new_output()
+        pm32.forward(x32, y32)
+        torch.cuda.synchronize()
+        t32 = pm32.layer_times(x32, y32, flush_l2=False, reps=5)
+        rows32 = roofline.network_roofline(model, 32, r_alu, roofline.HBM_NOMINAL_GBS)
+        k32 = [(r, ms) for r, ms in zip(rows32, t32) if r["family"] == "sconv_kxk" and r["nnz"] and r["name"] not in ("conv1", "stem")]
+        sparse["frac_3x3_layers_batch32_kernel_only"] = sum(r["t_roof_us"] for r, _ in k32) / (sum(ms for _, ms in k32) * 1e3)
+        sparse["frac_network_batch32_kernel_sum"] = sum(r["t_roof_us"] for r in rows32) / (sum(t32) * 1e3)
+        del pm32, x32, y32
 
     line = None
     if rank == 0:
@@ -296,8 +321,17 @@ def run_ours(args):
                 oracle_forward.forward(model, x_np)
                 reps_cpu += 1
             dt = (time.perf_counter() - t0) / reps_cpu
-            cpu_base = {"value": batch / dt, "unit": "images/s", "cores": ref.num_threads(), "kind": "oracle",
+            cores = ref.num_threads()
+            cpu_base = {"value": batch / dt, "unit": "images/s", "cores": cores, "kind": "oracle",
                         "sample": "%d whole-network forward(s) of %d image(s), %.2f s each" % (reps_cpu, batch, dt)}
+            if not args.no_one_thread:
+                ref.set_threads(1)
+                t0 = time.perf_counter()
+                oracle_forward.forward(model, x_np)
+                dt1 = time.perf_counter() - t0
+                ref.set_threads(cores)
+                cpu_base["one_thread"] = {"value": batch / dt1, "unit": "images/s", "cores": 1,
+                                          "sample": "1 whole-network forward of %d image(s), %.2f s" % (batch, dt1)}
         value = images / (cold_ms * 1e-3)
         line = {"metric": METRIC, "value": value, "unit": "images/s", "n_gpus": world, "steps": K, "warmup": W,
                 "ms_per_step": cold_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -326,6 +360,8 @@ def main():
     ap.add_argument("--workload", default="resnet50")
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--no-autotune", action="store_true", help="use the packer's time model instead of timing schedules")
+    ap.add_argument("--no-one-thread", action="store_true", help="skip the 1-thread run of the CPU baseline")
+    ap.add_argument("--no-batch32", action="store_true", help="skip the batch-32 kernel-only fraction of the 3x3 layers")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = 5 if args.steps is None else args.steps
