@@ -2,7 +2,7 @@
 """Benchmark: whole-network forward of the synthetic pruned ResNet-50 (batch 1 per GPU).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload resnet50|vgg16|mobilenet_v2|single] [--batch B]
+                    [--workload resnet50|vgg16|mobilenet_v2|mobilenet_v1|inception_v3|single] [--batch B]
 
 One step = one pass of the whole hot path (every layer of the network) over one
 batch.  Prints ONE JSON line on rank 0.  Multi-GPU runs are independent replicas
@@ -30,6 +30,10 @@ def build_model(name):
         return models.vgg16(), "vgg16_int8_224_conv8pct_fc4pct"
     if name == "mobilenet_v2":
         return models.mobilenet_v2(), "mobilenet_v2_1.0_224_pointwise25pct"
+    if name == "inception_v3":
+        return models.inception_v3(), "inception_v3_299_conv12.5pct_fc10pct_stem_dense"
+    if name == "mobilenet_v1":
+        return models.mobilenet_v1(), "mobilenet_v1_1.0_224_pointwise25pct"
     if name == "single":
         return models.single_layer(), "conv3x3_64to64_56x56_10pct"
     raise SystemExit("unknown workload " + name)

@@ -73,7 +73,8 @@ typedef enum {
  * filter regrouping depend on the layer's spatial size, so the input size the
  * layer will run at is part of its description.
  *   conv: c_in, c_out, kh, kw, stride, pad, groups (1, or c_in == c_out for depthwise),
- *         in_h, in_w.
+ *         in_h, in_w.  pad pads rows and columns alike unless pad_w >= 0, which then pads the
+ *         columns (the 1x7 / 7x1 kernels of an Inception module pad one axis only).
  *   fc:   kh = kw = 1, stride = 1, pad = 0, groups = 1, in_h = in_w = 1, c_in = K.
  *   batch_hint: batch size the schedule is tuned for (>= 1); any batch still runs.
  */
@@ -84,6 +85,7 @@ typedef struct {
     int dtype; /* cadnn_dtype of weights and activations: CADNN_F32 or CADNN_S8 */
     int fmt;   /* cadnn_fmt, CADNN_FMT_AUTO */
     int flags; /* CADNN_PACK_HOST_ONLY, CADNN_PACK_AUTOTUNE or 0 */
+    int pad_w; /* padding of the columns; -1 = same as pad */
 } cadnn_layer_desc;
 
 typedef struct cadnn_weights cadnn_weights;
@@ -167,13 +169,20 @@ void cadnn_free_weights(cadnn_weights *w); /* the same call under the name the p
  *                residual must be NULL and ReLU6 is not defined.
  * scale, bias: device float [c_out], NULL = 1 / 0.  residual: device, same shape and
  * dtype as y, or NULL.
+ * Channel concatenation (the branches of an Inception module, Section 5 / Table 2): with
+ * out_c_total > 0, y has out_c_total channels per pixel and the layer writes channels
+ * [out_c_off, out_c_off + c_out) of it, leaving the others alone; 0 = y has exactly c_out
+ * channels.  Sparse conv layers only (E_UNSUPPORTED for fc, depthwise and stem kernels), and
+ * without a residual.
  */
 typedef struct {
     const float *scale;
     const float *bias;
     const void *residual;
-    int act;       /* cadnn_act */
-    int out_dtype; /* cadnn_dtype of y */
+    int act;         /* cadnn_act */
+    int out_dtype;   /* cadnn_dtype of y */
+    int out_c_total; /* channels per pixel of y, 0 = c_out */
+    int out_c_off;   /* first channel of y this layer writes */
 } cadnn_epilogue;
 
 /*
@@ -215,11 +224,16 @@ cadnn_status cadnn_fc(const cadnn_weights *w, const void *x, int n, void *y,
  * Max pool ignores padded taps; dtype CADNN_F32 or CADNN_S8. */
 cadnn_status cadnn_maxpool2d(const void *x, int n, int h, int wd, int c, int k, int stride, int pad,
                              int dtype, void *y, void *stream);
+/* Max or average pool (kind 0 / 1) that writes channels [out_c_off, out_c_off + c) of a y with out_c_total
+ * channels per pixel (0 = c).  The average pool is float only; taps that fall in the padding count
+ * as zeros and the divisor is always k * k. */
+cadnn_status cadnn_pool2d(const void *x, int n, int h, int wd, int c, int k, int stride, int pad, int dtype, int kind,
+                          void *y, int out_c_total, int out_c_off, void *stream);
 /* Global average pool, float: y[b][c] = mean over h*w. */
 cadnn_status cadnn_global_avgpool(const float *x, int n, int h, int wd, int c, float *y, void *stream);
 
 /* Whole network (Section 5: single-image inference of a complete model). */
-typedef enum { CADNN_OP_CONV = 0, CADNN_OP_FC = 1, CADNN_OP_MAXPOOL = 2, CADNN_OP_GAVGPOOL = 3 } cadnn_op_kind;
+typedef enum { CADNN_OP_CONV = 0, CADNN_OP_FC = 1, CADNN_OP_MAXPOOL = 2, CADNN_OP_GAVGPOOL = 3, CADNN_OP_AVGPOOL = 4 } cadnn_op_kind;
 
 typedef struct {
     int kind;                 /* cadnn_op_kind */
@@ -229,7 +243,9 @@ typedef struct {
     const float *bias;        /* device [c_out] or NULL; borrowed */
     int act;                  /* cadnn_act */
     int out_dtype;            /* cadnn_dtype of the dst slot */
-    int pool_k, pool_stride, pool_pad; /* max pool only */
+    int pool_k, pool_stride, pool_pad; /* max / average pool only */
+    int dst_c_off, dst_c_total; /* conv and pools: the op writes channels [dst_c_off, dst_c_off + c) of a dst slot
+                                   that has dst_c_total channels (channel concatenation); 0, 0 = the whole slot */
 } cadnn_op;
 
 /*
@@ -237,7 +253,8 @@ typedef struct {
  * and allocate one device buffer per intermediate slot (owned by the net).  The dst
  * slot of the last op is the network output and is written straight to the pointer
  * given to cadnn_forward.  Every slot is written by exactly one op, after which it is
- * only read.
+ * only read - or, for a concatenation, by several ops that each write their own channel
+ * window of it (dst_c_total > 0, same in all of them) before any op reads it.
  */
 cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int wd, int c, int in_dtype,
                               cadnn_net **out);

@@ -23,7 +23,7 @@ DTYPE = {"f32": F32, "s8": S8, "s32": S32}
 ACT = {"none": 0, "relu": 1, "relu6": 2, None: 0}
 PACK_HOST_ONLY = 1
 PACK_AUTOTUNE = 2
-OP_CONV, OP_FC, OP_MAXPOOL, OP_GAVGPOOL = 0, 1, 2, 3
+OP_CONV, OP_FC, OP_MAXPOOL, OP_GAVGPOOL, OP_AVGPOOL = 0, 1, 2, 3, 4
 FMT_NAMES = {1: "tiled_csr", 2: "row_csr", 3: "dense_dw", 4: "dense_smallc"}
 KIND_NAMES = {1: "sconv_spatial", 2: "sconv_linear", 3: "fc_spmv", 4: "dw", 5: "dense_smallc"}
 
@@ -31,19 +31,21 @@ KIND_NAMES = {1: "sconv_spatial", 2: "sconv_linear", 3: "fc_spmv", 4: "dw", 5: "
 class LayerDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in
                 ("c_in", "c_out", "kh", "kw", "stride", "pad", "groups", "in_h", "in_w",
-                 "batch_hint", "dtype", "fmt", "flags")]
+                 "batch_hint", "dtype", "fmt", "flags", "pad_w")]
 
 
 class Epilogue(ctypes.Structure):
     _fields_ = [("scale", ctypes.c_void_p), ("bias", ctypes.c_void_p), ("residual", ctypes.c_void_p),
-                ("act", ctypes.c_int), ("out_dtype", ctypes.c_int)]
+                ("act", ctypes.c_int), ("out_dtype", ctypes.c_int), ("out_c_total", ctypes.c_int),
+                ("out_c_off", ctypes.c_int)]
 
 
 class Op(ctypes.Structure):
     _fields_ = [("kind", ctypes.c_int), ("w", ctypes.c_void_p), ("src", ctypes.c_int), ("dst", ctypes.c_int),
                 ("res", ctypes.c_int), ("scale", ctypes.c_void_p), ("bias", ctypes.c_void_p),
                 ("act", ctypes.c_int), ("out_dtype", ctypes.c_int), ("pool_k", ctypes.c_int),
-                ("pool_stride", ctypes.c_int), ("pool_pad", ctypes.c_int)]
+                ("pool_stride", ctypes.c_int), ("pool_pad", ctypes.c_int), ("dst_c_off", ctypes.c_int),
+                ("dst_c_total", ctypes.c_int)]
 
 
 _vp, _i, _i64p = ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_int64)
@@ -61,6 +63,7 @@ _SIGS = {
     "cadnn_conv2d_planar": (_i, [_vp, _vp, _i, _vp, ctypes.POINTER(Epilogue), _vp]),
     "cadnn_fc": (_i, [_vp, _vp, _i, _vp, ctypes.POINTER(Epilogue), _vp]),
     "cadnn_maxpool2d": (_i, [_vp, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _vp]),
+    "cadnn_pool2d": (_i, [_vp, _i, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i, _i, _vp]),
     "cadnn_global_avgpool": (_i, [_vp, _i, _i, _i, _i, _vp, _vp]),
     "cadnn_net_create": (_i, [ctypes.POINTER(Op), _i, _i, _i, _i, _i, _i, ctypes.POINTER(_vp)]),
     "cadnn_forward": (_i, [_vp, _vp, _vp, _i, _vp]),
@@ -139,9 +142,9 @@ class Weights:
 
 
 def make_desc(c_in, c_out, kh=1, kw=1, stride=1, pad=0, groups=1, in_h=1, in_w=1, batch_hint=1,
-              dtype="f32", host_only=False, autotune=False):
+              dtype="f32", host_only=False, autotune=False, pad_w=-1):
     flags = (PACK_HOST_ONLY if host_only else 0) | (PACK_AUTOTUNE if autotune else 0)
-    return LayerDesc(c_in, c_out, kh, kw, stride, pad, groups, in_h, in_w, batch_hint, DTYPE[dtype], 0, flags)
+    return LayerDesc(c_in, c_out, kh, kw, stride, pad, groups, in_h, in_w, batch_hint, DTYPE[dtype], 0, flags, pad_w)
 
 
 def cadnn_pack(desc, w_ohwi, mask=None, w_scale=None):
@@ -212,18 +215,20 @@ def cadnn_weights_unpack(w):
     return dense, mask
 
 
-def _epilogue(scale, bias, residual, act, out_dtype):
+def _epilogue(scale, bias, residual, act, out_dtype, out_c_total=0, out_c_off=0):
     return Epilogue(None if scale is None else scale.data_ptr(), None if bias is None else bias.data_ptr(),
                     None if residual is None else residual.data_ptr(), ACT[act] if not isinstance(act, int) else act,
-                    DTYPE[out_dtype] if not isinstance(out_dtype, int) else out_dtype)
+                    DTYPE[out_dtype] if not isinstance(out_dtype, int) else out_dtype, out_c_total, out_c_off)
 
 
-def cadnn_conv2d(w, x, y, scale=None, bias=None, residual=None, act="none", out_dtype=None, stream=None):
-    """x, y: torch CUDA tensors, NHWC contiguous; y is written in place."""
+def cadnn_conv2d(w, x, y, scale=None, bias=None, residual=None, act="none", out_dtype=None, stream=None,
+                 out_c_total=0, out_c_off=0):
+    """x, y: torch CUDA tensors, NHWC contiguous; y is written in place (channels [out_c_off, out_c_off + c_out)
+    of it when out_c_total > 0)."""
     n, h, wd = int(x.shape[0]), int(x.shape[1]), int(x.shape[2])
     if out_dtype is None:
         out_dtype = w.desc.dtype
-    ep = _epilogue(scale, bias, residual, act, out_dtype)
+    ep = _epilogue(scale, bias, residual, act, out_dtype, out_c_total, out_c_off)
     _check(_lib.cadnn_conv2d(w.handle, _dev_ptr(x), n, h, wd, _dev_ptr(y), ctypes.byref(ep), _stream(stream)),
            "cadnn_conv2d")
     return y
@@ -253,6 +258,16 @@ def cadnn_maxpool2d(x, y, k, stride, pad=0, stream=None):
     dt = S8 if x.dtype == torch.int8 else F32
     _check(_lib.cadnn_maxpool2d(_dev_ptr(x), n, h, wd, c, k, stride, pad, dt, _dev_ptr(y), _stream(stream)),
            "cadnn_maxpool2d")
+    return y
+
+
+def cadnn_pool2d(x, y, k, stride, pad=0, kind="max", out_c_total=0, out_c_off=0, stream=None):
+    """Max / average pool of x (NHWC) into y, or into channels [out_c_off, out_c_off + c) of a wider y."""
+    import torch
+    n, h, wd, c = (int(v) for v in x.shape)
+    dt = S8 if x.dtype == torch.int8 else F32
+    _check(_lib.cadnn_pool2d(_dev_ptr(x), n, h, wd, c, k, stride, pad, dt, 1 if kind == "avg" else 0, _dev_ptr(y),
+                             out_c_total, out_c_off, _stream(stream)), "cadnn_pool2d")
     return y
 
 

@@ -45,6 +45,14 @@ cadnn_status check_epilogue(const cadnn_weights *w, const cadnn_epilogue *ep, La
     le.residual = ep->residual;
     le.act = ep->act;
     le.out_dtype = ep->out_dtype;
+    le.out_c_total = ep->out_c_total;
+    le.out_c_off = ep->out_c_off;
+    if (le.out_c_total < 0 || le.out_c_off < 0) return CADNN_E_ARG;
+    if (le.out_c_total > 0) {   // a channel window of a wider output: sparse conv kernels only, no residual
+        if (le.out_c_off + w->desc.c_out > le.out_c_total) return CADNN_E_SHAPE;
+        if (le.residual) return CADNN_E_UNSUPPORTED;
+        if (w->s.kind != KK_SCONV_SPATIAL && w->s.kind != KK_SCONV_LINEAR) return CADNN_E_UNSUPPORTED;
+    } else if (le.out_c_off != 0) return CADNN_E_ARG;
     if (le.act < CADNN_ACT_NONE || le.act > CADNN_ACT_RELU6) return CADNN_E_ARG;
     if (dt == CADNN_F32) {
         if (le.out_dtype != CADNN_F32) return CADNN_E_DTYPE;
@@ -59,7 +67,7 @@ cadnn_status check_epilogue(const cadnn_weights *w, const cadnn_epilogue *ep, La
 
 }  // namespace
 
-cadnn_status check_layer_call(const cadnn_weights *w, bool has_residual, int act, int out_dtype)
+cadnn_status check_layer_call(const cadnn_weights *w, bool has_residual, int act, int out_dtype, int out_c_total, int out_c_off)
 {
     if (!w || !w->on_device) return CADNN_E_ARG;
     int dev = -1;
@@ -68,7 +76,7 @@ cadnn_status check_layer_call(const cadnn_weights *w, bool has_residual, int act
     cadnn_epilogue ep;
     alignas(16) static const char some_residual[16] = {0};   // only its presence matters here
     ep.scale = nullptr; ep.bias = nullptr; ep.residual = has_residual ? some_residual : nullptr;
-    ep.act = act; ep.out_dtype = out_dtype;
+    ep.act = act; ep.out_dtype = out_dtype; ep.out_c_total = out_c_total; ep.out_c_off = out_c_off;
     LaunchEpilogue le;
     return check_epilogue(w, &ep, le);
 }
@@ -130,6 +138,19 @@ cadnn_status cadnn_maxpool2d(const void *x, int n, int h, int wd, int c, int k, 
     if (pad >= k || h + 2 * pad < k || wd + 2 * pad < k) return CADNN_E_SHAPE;
     if (dtype != CADNN_F32 && dtype != CADNN_S8) return CADNN_E_DTYPE;
     return launch_maxpool(x, n, h, wd, c, k, stride, pad, dtype, y, false, (cudaStream_t)stream);
+}
+
+cadnn_status cadnn_pool2d(const void *x, int n, int h, int wd, int c, int k, int stride, int pad, int dtype, int kind,
+                          void *y, int out_c_total, int out_c_off, void *stream)
+{
+    if (!x || !y || n < 0 || h < 1 || wd < 1 || c < 1 || k < 1 || stride < 1 || pad < 0 || out_c_total < 0 || out_c_off < 0)
+        return CADNN_E_ARG;
+    if (kind != 0 && kind != 1) return CADNN_E_ARG;
+    if (pad >= k || h + 2 * pad < k || wd + 2 * pad < k) return CADNN_E_SHAPE;
+    if (out_c_total > 0 ? out_c_off + c > out_c_total : out_c_off != 0) return CADNN_E_SHAPE;
+    if (dtype != CADNN_F32 && dtype != CADNN_S8) return CADNN_E_DTYPE;
+    if (kind == 1 && dtype != CADNN_F32) return CADNN_E_DTYPE;
+    return launch_pool_window(x, n, h, wd, c, k, stride, pad, dtype, kind, y, out_c_total, out_c_off, false, (cudaStream_t)stream);
 }
 
 cadnn_status cadnn_global_avgpool(const float *x, int n, int h, int wd, int c, float *y, void *stream)

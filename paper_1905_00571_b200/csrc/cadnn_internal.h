@@ -144,6 +144,7 @@ struct LaunchEpilogue {
     bool pdl = false;   // launch as a programmatic dependent of the previous kernel (inside cadnn_forward)
     bool early_trigger = false;   // trigger dependents at kernel start instead of before the epilogue
     bool planar_out = false;   // dense stem: write the channel-planar layout instead of NHWC
+    int out_c_total = 0, out_c_off = 0;   // NHWC sparse conv: channel window of a wider output tensor (concatenation)
 };
 
 // status helpers
@@ -164,7 +165,8 @@ struct SmemLimit {
 cadnn_status raise_smem_limit(const void *kern, int smem, SmemLimit *lim);
 
 // epilogue / device checks of one layer call (no launch): what conv2d_impl would refuse
-cadnn_status check_layer_call(const cadnn_weights *w, bool has_residual, int act, int out_dtype);
+cadnn_status check_layer_call(const cadnn_weights *w, bool has_residual, int act, int out_dtype, int out_c_total = 0,
+                              int out_c_off = 0);
 
 // kernel launchers (each validates nothing; callers did)
 cadnn_status launch_sconv(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
@@ -226,6 +228,9 @@ cadnn_status launch_maxpool_planar(const float *x, int n, int h, int wd, int c, 
 cadnn_status launch_gavgpool_planar(const float *x, int n, int h, int wd, int c, float *y, bool pdl, cudaStream_t st);
 cadnn_status launch_maxpool(const void *x, int n, int h, int wd, int c, int k, int stride, int pad, int dtype,
                             void *y, bool pdl, cudaStream_t st);
+// max (kind 0) or average (kind 1, float) pool into channels [c_off, c_off + c) of a y with ldc channels per pixel
+cadnn_status launch_pool_window(const void *x, int n, int h, int wd, int c, int k, int stride, int pad, int dtype, int kind,
+                                void *y, int ldc, int c_off, bool pdl, cudaStream_t st);
 cadnn_status launch_gavgpool(const float *x, int n, int h, int wd, int c, float *y, bool pdl, cudaStream_t st);
 
 // layer entry shared by the public calls and the network runner

@@ -18,7 +18,7 @@ struct DwParams {
     const float *scale;
     const float *bias;
     const float *residual;
-    int n, h, w, c, h_out, w_out, kh, kw, stride, pad, act;
+    int n, h, w, c, h_out, w_out, kh, kw, stride, pad, pad_w, act;
     FastDiv d_cv, d_wout, d_hout;
 };
 
@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(256) dw_kernel(const DwParams p)
             const int iy = oy * p.stride + ky - p.pad;
             if (iy < 0 || iy >= p.h) continue;
             for (int kx = 0; kx < p.kw; ++kx) {
-                const int ix = ox * p.stride + kx - p.pad;
+                const int ix = ox * p.stride + kx - p.pad_w;
                 if (ix < 0 || ix >= p.w) continue;
                 const float *xs = p.x + (((size_t)b * p.h + iy) * p.w + ix) * p.c + c0;
                 const float *ws = p.wt + (size_t)(ky * p.kw + kx) * p.c + c0;
@@ -92,7 +92,7 @@ struct StemParams {
     const float *scale;
     const float *bias;
     const float *residual;
-    int n, h, w, c_in, c_out, h_out, w_out, kh, kw, stride, pad, act;
+    int n, h, w, c_in, c_out, h_out, w_out, kh, kw, stride, pad, pad_w, act;
     int tiles_x, tiles_y, in_rows, in_cols, taps, co_blocks;
     int planar_out, halo;   // write [n][c][h_out + 2 halo][w_out + 2 halo] instead of NHWC
 };
@@ -121,7 +121,7 @@ __global__ void __launch_bounds__(256) stem_kernel(const StemParams p)
     }
     grid_dep_wait();
     grid_dep_trigger();
-    const int iy0 = oy0 * p.stride - p.pad, ix0 = ox0 * p.stride - p.pad;
+    const int iy0 = oy0 * p.stride - p.pad, ix0 = ox0 * p.stride - p.pad_w;
     const int row_words = p.in_cols * p.c_in;
     for (int i = tid; i < p.in_rows * row_words; i += blockDim.x) {
         const int r = i / row_words, rem = i - r * row_words;
@@ -246,7 +246,7 @@ __global__ void __launch_bounds__(128) stem2_kernel(const StemParams p)
     }
     grid_dep_wait();
     grid_dep_trigger();
-    const int iy0 = oy0 * STRIDE - p.pad, ix0 = ox0 * STRIDE - p.pad;
+    const int iy0 = oy0 * STRIDE - p.pad, ix0 = ox0 * STRIDE - p.pad_w;
     // input rows: IN_COLS * CIN consecutive floats of the NHWC image each; warp r mod 4 takes row r
     for (int r = wc; r < IN_ROWS; r += 4) {
         const int iy = iy0 + r;
@@ -357,7 +357,7 @@ cadnn_status launch_dw(const cadnn_weights *w, const void *x, int n, void *y, co
     p.x = (const float *)x; p.y = (float *)y; p.wt = w->d_dense;
     p.scale = ep.scale; p.bias = ep.bias; p.residual = (const float *)ep.residual;
     p.n = n; p.h = d.in_h; p.w = d.in_w; p.c = d.c_out; p.h_out = w->h_out; p.w_out = w->w_out;
-    p.kh = d.kh; p.kw = d.kw; p.stride = d.stride; p.pad = d.pad; p.act = ep.act;
+    p.kh = d.kh; p.kw = d.kw; p.stride = d.stride; p.pad = d.pad; p.pad_w = d.pad_w; p.act = ep.act;
     const bool v4 = d.c_out % 4 == 0;
     long long total = (long long)n * w->h_out * w->w_out * (v4 ? d.c_out / 4 : d.c_out);
     if (total <= 0) return CADNN_OK;
@@ -379,7 +379,7 @@ cadnn_status launch_dense_smallc(const cadnn_weights *w, const void *x, int n, v
     p.x = (const float *)x; p.y = (float *)y; p.wt = w->d_dense;
     p.scale = ep.scale; p.bias = ep.bias; p.residual = (const float *)ep.residual;
     p.n = n; p.h = d.in_h; p.w = d.in_w; p.c_in = d.c_in; p.c_out = d.c_out;
-    p.h_out = w->h_out; p.w_out = w->w_out; p.kh = d.kh; p.kw = d.kw; p.stride = d.stride; p.pad = d.pad;
+    p.h_out = w->h_out; p.w_out = w->w_out; p.kh = d.kh; p.kw = d.kw; p.stride = d.stride; p.pad = d.pad; p.pad_w = d.pad_w;
     p.act = ep.act;
     p.planar_out = ep.planar_out ? 1 : 0;
     p.halo = kPlanarHalo;

@@ -128,8 +128,11 @@ cadnn_status cadnn_forward_static(const cadnn_op *ops, int n_ops, int n, int h, 
         const cadnn_op &op = ops[i];
         const Tensor si = t[op.src];
         Tensor &so = t[op.dst];
-        if (!si.defined || so.defined) return CADNN_E_ARG;
-        so.n = si.n;
+        const bool window = op.dst_c_total > 0;
+        if (op.dst_c_total < 0 || op.dst_c_off < 0 || (!window && op.dst_c_off != 0)) return CADNN_E_ARG;
+        if (!si.defined || (so.defined && !window)) return CADNN_E_ARG;
+        Tensor sn;   // what this op produces
+        sn.n = si.n;
         if (op.kind == CADNN_OP_CONV || op.kind == CADNN_OP_FC) {
             if (!op.w || !op.w->on_device) return CADNN_E_ARG;
             const cadnn_layer_desc &d = op.w->desc;
@@ -139,34 +142,45 @@ cadnn_status cadnn_forward_static(const cadnn_op *ops, int n_ops, int n, int h, 
             } else if (si.h != d.in_h || si.w != d.in_w || si.c != d.c_in) {
                 return CADNN_E_SHAPE;
             }
-            so.h = op.w->h_out; so.w = op.w->w_out; so.c = d.c_out; so.dtype = op.out_dtype;
+            sn.h = op.w->h_out; sn.w = op.w->w_out; sn.c = d.c_out; sn.dtype = op.out_dtype;
             if (op.res >= 0) {
                 const Tensor &sr = t[op.res];
-                if (!sr.defined || sr.h != so.h || sr.w != so.w || sr.c != so.c || sr.dtype != so.dtype)
+                if (!sr.defined || sr.h != sn.h || sr.w != sn.w || sr.c != sn.c || sr.dtype != sn.dtype)
                     return CADNN_E_SHAPE;
             }
             // everything the layer call itself would refuse is refused here, before the first launch:
             // the epilogue combination, weights packed on another GPU, an input beyond the staging limit
-            cadnn_status cs = check_layer_call(op.w, op.res >= 0, op.act, op.out_dtype);
+            cadnn_status cs = check_layer_call(op.w, op.res >= 0, op.act, op.out_dtype, op.dst_c_total, op.dst_c_off);
             if (cs != CADNN_OK) return cs;
             if ((long long)si.n * si.h * si.w * si.c * dtype_size(si.dtype) >= (1LL << 34)) return CADNN_E_UNSUPPORTED;
-        } else if (op.kind == CADNN_OP_MAXPOOL) {
+        } else if (op.kind == CADNN_OP_MAXPOOL || op.kind == CADNN_OP_AVGPOOL) {
             if (op.pool_k < 1 || op.pool_stride < 1 || op.pool_pad < 0 || op.pool_pad >= op.pool_k ||
                 si.h + 2 * op.pool_pad < op.pool_k || si.w + 2 * op.pool_pad < op.pool_k)
                 return CADNN_E_SHAPE;
-            so.h = (si.h + 2 * op.pool_pad - op.pool_k) / op.pool_stride + 1;
-            so.w = (si.w + 2 * op.pool_pad - op.pool_k) / op.pool_stride + 1;
-            so.c = si.c; so.dtype = si.dtype;
+            if (op.kind == CADNN_OP_AVGPOOL && si.dtype != CADNN_F32) return CADNN_E_DTYPE;
+            sn.h = (si.h + 2 * op.pool_pad - op.pool_k) / op.pool_stride + 1;
+            sn.w = (si.w + 2 * op.pool_pad - op.pool_k) / op.pool_stride + 1;
+            sn.c = si.c; sn.dtype = si.dtype;
         } else if (op.kind == CADNN_OP_GAVGPOOL) {
+            if (window) return CADNN_E_UNSUPPORTED;
             if (si.dtype != CADNN_F32) return CADNN_E_DTYPE;
-            so.h = 1; so.w = 1; so.c = si.c; so.dtype = CADNN_F32;
+            sn.h = 1; sn.w = 1; sn.c = si.c; sn.dtype = CADNN_F32;
         } else {
             return CADNN_E_ARG;
         }
-        so.defined = true;
-        so.bytes = ((size_t)so.n * so.h * so.w * so.c * dtype_size(so.dtype) + 255) / 256 * 256;
         t[op.src].last_use = i;
         if (op.res >= 0) t[op.res].last_use = i;
+        if (window) {
+            if (op.dst_c_off + sn.c > op.dst_c_total) return CADNN_E_SHAPE;
+            sn.c = op.dst_c_total;
+            if (so.defined) {   // a later writer of the same concatenation
+                if (so.h != sn.h || so.w != sn.w || so.c != sn.c || so.dtype != sn.dtype || so.n != sn.n) return CADNN_E_SHAPE;
+                continue;
+            }
+        }
+        so.n = sn.n; so.h = sn.h; so.w = sn.w; so.c = sn.c; so.dtype = sn.dtype;
+        so.defined = true;
+        so.bytes = ((size_t)so.n * so.h * so.w * so.c * dtype_size(so.dtype) + 255) / 256 * 256;
     }
 
     // ---- place the intermediate tensors: first fit, a region returns to the free list once
@@ -177,7 +191,7 @@ cadnn_status cadnn_forward_static(const cadnn_op *ops, int n_ops, int n, int h, 
     for (int i = 0; i <= max_slot; ++i) placed_at[i] = -1;
     for (int i = 0; i < n_ops; ++i) {
         const cadnn_op &op = ops[i];
-        if (op.dst != out_slot) {
+        if (op.dst != out_slot && placed_at[op.dst] < 0) {   // (a concatenation is placed by its first writer)
             // does not fit the fixed workspace: refuse rather than allocate
             if (!arena_take(fl, t[op.dst].bytes, &t[op.dst].off)) return CADNN_E_UNSUPPORTED;
             placed_at[op.dst] = i;
@@ -212,10 +226,13 @@ cadnn_status cadnn_forward_static(const cadnn_op *ops, int n_ops, int n, int h, 
             ep.residual = op.res >= 0 ? ptr_of(op.res) : nullptr;
             ep.act = op.act;
             ep.out_dtype = op.out_dtype;
+            ep.out_c_total = op.dst_c_total;
+            ep.out_c_off = op.dst_c_off;
             if (op.kind == CADNN_OP_FC) rc = conv2d_impl(op.w, src, si.n, 1, 1, dst, &ep, false, st);
             else rc = conv2d_impl(op.w, src, si.n, si.h, si.w, dst, &ep, false, st);
-        } else if (op.kind == CADNN_OP_MAXPOOL) {
-            rc = launch_maxpool(src, si.n, si.h, si.w, si.c, op.pool_k, op.pool_stride, op.pool_pad, si.dtype, dst, false, st);
+        } else if (op.kind == CADNN_OP_MAXPOOL || op.kind == CADNN_OP_AVGPOOL) {
+            rc = launch_pool_window(src, si.n, si.h, si.w, si.c, op.pool_k, op.pool_stride, op.pool_pad, si.dtype,
+                                    op.kind == CADNN_OP_AVGPOOL ? 1 : 0, dst, op.dst_c_total, op.dst_c_off, false, st);
         } else {
             rc = launch_gavgpool((const float *)src, si.n, si.h, si.w, si.c, (float *)dst, false, st);
         }

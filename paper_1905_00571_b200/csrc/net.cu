@@ -92,11 +92,14 @@ cadnn_status run_op(cadnn_net *net, const cadnn_op &op, const void *x, void *y, 
         ep.residual = op.res >= 0 ? slot_ptr(net, op.res, x, y) : nullptr;
         ep.act = op.act;
         ep.out_dtype = op.out_dtype;
+        ep.out_c_total = op.dst_c_total;
+        ep.out_c_off = op.dst_c_off;
         if (op.kind == CADNN_OP_FC) return conv2d_impl(op.w, src, si.n, 1, 1, dst, &ep, pdl, st);
         return conv2d_impl(op.w, src, si.n, si.h, si.w, dst, &ep, pdl, st);
     }
-    if (op.kind == CADNN_OP_MAXPOOL)
-        return launch_maxpool(src, si.n, si.h, si.w, si.c, op.pool_k, op.pool_stride, op.pool_pad, si.dtype, dst, pdl, st);
+    if (op.kind == CADNN_OP_MAXPOOL || op.kind == CADNN_OP_AVGPOOL)
+        return launch_pool_window(src, si.n, si.h, si.w, si.c, op.pool_k, op.pool_stride, op.pool_pad, si.dtype,
+                                  op.kind == CADNN_OP_AVGPOOL ? 1 : 0, dst, op.dst_c_total, op.dst_c_off, pdl, st);
     if (op.kind == CADNN_OP_GAVGPOOL)
         return launch_gavgpool((const float *)src, si.n, si.h, si.w, si.c, (float *)dst, pdl, st);
     return CADNN_E_ARG;
@@ -345,6 +348,7 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
         std::vector<char> flat(max_slot + 1, 0);   // slot holds a dense [n][c] vector
         for (int i = 0; i < n_ops && planar; ++i) {
             const cadnn_op &op = ops[i];
+            if (op.dst_c_total > 0 || op.kind == CADNN_OP_AVGPOOL) { planar = false; break; }   // concatenations stay NHWC
             if (op.kind == CADNN_OP_CONV) {
                 if (!op.w) { planar = false; break; }
                 const bool stem = op.w->s.kind == KK_DENSE_SMALLC && op.src == 0 && op.res < 0;
@@ -382,8 +386,12 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
         const cadnn_op &op = ops[i];
         const SlotInfo si = net->slots[op.src];
         SlotInfo &so = net->slots[op.dst];
-        if (!si.defined || so.defined) { st = CADNN_E_ARG; break; }
-        so.n = si.n;
+        const bool window = op.dst_c_total > 0;
+        if (op.dst_c_total < 0 || op.dst_c_off < 0 || (!window && op.dst_c_off != 0)) { st = CADNN_E_ARG; break; }
+        // a slot has one writer, or several that each fill a channel window of it
+        if (!si.defined || (so.defined && !window)) { st = CADNN_E_ARG; break; }
+        SlotInfo sn;   // what this op produces
+        sn.n = si.n;
         if (op.kind == CADNN_OP_CONV || op.kind == CADNN_OP_FC) {
             if (!op.w || !op.w->on_device) { st = CADNN_E_ARG; break; }
             const cadnn_layer_desc &d = op.w->desc;
@@ -391,27 +399,38 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
             if (op.kind == CADNN_OP_FC) {
                 if ((long long)si.h * si.w * si.c != d.c_in) { st = CADNN_E_SHAPE; break; }
             } else if (si.h != d.in_h || si.w != d.in_w || si.c != d.c_in) { st = CADNN_E_SHAPE; break; }
-            so.h = op.w->h_out; so.w = op.w->w_out; so.c = d.c_out; so.dtype = op.out_dtype;
+            sn.h = op.w->h_out; sn.w = op.w->w_out; sn.c = d.c_out; sn.dtype = op.out_dtype;
             if (op.res >= 0) {
                 const SlotInfo &sr = net->slots[op.res];
-                if (!sr.defined || sr.h != so.h || sr.w != so.w || sr.c != so.c || sr.dtype != so.dtype) {
+                if (!sr.defined || sr.h != sn.h || sr.w != sn.w || sr.c != sn.c || sr.dtype != sn.dtype) {
                     st = CADNN_E_SHAPE;
                     break;
                 }
             }
             // what the layer call would refuse (epilogue combination, weights of another GPU) is refused now
-            st = check_layer_call(op.w, op.res >= 0, op.act, op.out_dtype);
+            st = check_layer_call(op.w, op.res >= 0, op.act, op.out_dtype, op.dst_c_total, op.dst_c_off);
             if (st != CADNN_OK) break;
-        } else if (op.kind == CADNN_OP_MAXPOOL) {
+        } else if (op.kind == CADNN_OP_MAXPOOL || op.kind == CADNN_OP_AVGPOOL) {
             if (op.pool_k < 1 || op.pool_stride < 1 || op.pool_pad < 0 || op.pool_pad >= op.pool_k ||
                 si.h + 2 * op.pool_pad < op.pool_k || si.w + 2 * op.pool_pad < op.pool_k) { st = CADNN_E_SHAPE; break; }
-            so.h = (si.h + 2 * op.pool_pad - op.pool_k) / op.pool_stride + 1;
-            so.w = (si.w + 2 * op.pool_pad - op.pool_k) / op.pool_stride + 1;
-            so.c = si.c; so.dtype = si.dtype;
+            if (op.kind == CADNN_OP_AVGPOOL && si.dtype != CADNN_F32) { st = CADNN_E_DTYPE; break; }
+            sn.h = (si.h + 2 * op.pool_pad - op.pool_k) / op.pool_stride + 1;
+            sn.w = (si.w + 2 * op.pool_pad - op.pool_k) / op.pool_stride + 1;
+            sn.c = si.c; sn.dtype = si.dtype;
         } else if (op.kind == CADNN_OP_GAVGPOOL) {
-            if (si.dtype != CADNN_F32) { st = CADNN_E_DTYPE; break; }
-            so.h = 1; so.w = 1; so.c = si.c; so.dtype = CADNN_F32;
+            if (si.dtype != CADNN_F32 || window) { st = window ? CADNN_E_UNSUPPORTED : CADNN_E_DTYPE; break; }
+            sn.h = 1; sn.w = 1; sn.c = si.c; sn.dtype = CADNN_F32;
         } else { st = CADNN_E_ARG; break; }
+        if (window) {
+            if (op.dst_c_off + sn.c > op.dst_c_total) { st = CADNN_E_SHAPE; break; }
+            sn.c = op.dst_c_total;
+            if (so.defined) {   // a later writer of the same concatenation: same shape, nothing more to allocate
+                if (so.h != sn.h || so.w != sn.w || so.c != sn.c || so.dtype != sn.dtype || so.n != sn.n) st = CADNN_E_SHAPE;
+                if (st != CADNN_OK) break;
+                continue;
+            }
+        }
+        so.n = sn.n; so.h = sn.h; so.w = sn.w; so.c = sn.c; so.dtype = sn.dtype;
         so.defined = true;
         so.bytes = (int64_t)so.n * so.h * so.w * so.c * dtype_size(so.dtype);
         const bool padded = net->planar && (op.kind == CADNN_OP_CONV || op.kind == CADNN_OP_MAXPOOL);

@@ -558,7 +558,7 @@ void build_planar_image(cadnn_weights *h, const Src &src, const std::vector<int6
 {
     const cadnn_layer_desc &d = h->desc;
     const int halo = kPlanarHalo;
-    if (src.s8 || d.groups != 1 || d.pad > halo || d.kh - 1 - d.pad > halo || d.kw - 1 - d.pad > halo) return;
+    if (src.s8 || d.groups != 1 || d.pad_w != d.pad || d.pad > halo || d.kh - 1 - d.pad > halo || d.kw - 1 - d.pad > halo) return;
     const long long plane = planar_pitch(d.in_h, d.in_w);
     if (plane * d.c_in >= (1LL << 31)) return;
     const int wp = d.in_w + 2 * halo;
@@ -690,7 +690,7 @@ struct PsRows {
 
 bool ps_eligible(const cadnn_layer_desc &d, bool s8)
 {
-    if (s8 || d.groups != 1 || (d.stride != 1 && d.stride != 2) || d.kh != d.kw || 2 * d.pad != d.kh - 1 || d.pad > kPlanarHalo) return false;
+    if (s8 || d.groups != 1 || (d.stride != 1 && d.stride != 2) || d.kh != d.kw || d.pad_w != d.pad || 2 * d.pad != d.kh - 1 || d.pad > kPlanarHalo) return false;
     return (long long)planar_pitch(d.in_h, d.in_w) * d.c_in < (1LL << 31);
 }
 
@@ -1032,7 +1032,7 @@ uint64_t tune_key(const cadnn_layer_desc &d, const std::vector<int64_t> &row_nnz
             hsh *= 1099511628211ull;
         }
     };
-    for (int v : {d.c_in, d.c_out, d.kh, d.kw, d.stride, d.pad, d.groups, d.in_h, d.in_w, std::max(1, d.batch_hint), (int)d.dtype})
+    for (int v : {d.c_in, d.c_out, d.kh, d.kw, d.stride, d.pad, d.pad_w, d.groups, d.in_h, d.in_w, std::max(1, d.batch_hint), (int)d.dtype})
         mix((uint64_t)(int64_t)v);
     mix(sizeof(Schedule));
     mix(sizeof(PsSchedule));
@@ -1162,7 +1162,7 @@ void pack_ps(cadnn_weights *h, const Src &src, const std::vector<int64_t> &row_n
 cadnn_status pack_sconv(cadnn_weights *h, const Src &src)
 {
     const cadnn_layer_desc &d = h->desc;
-    const bool linear = (d.kh == 1 && d.kw == 1 && d.pad == 0);
+    const bool linear = (d.kh == 1 && d.kw == 1 && d.pad == 0 && d.pad_w == 0);
     const int K = d.kh * d.kw * d.c_in;
     int bh = std::max(1, d.batch_hint);
     std::vector<int64_t> row_nnz(d.c_out, 0);
@@ -1273,15 +1273,17 @@ cadnn_status pack_dense(cadnn_weights *h, const Src &src, int kind)
 cadnn_status pack_common(const cadnn_layer_desc *desc, const Src &src, cadnn_weights **out)
 {
     if (!desc || !out || (!src.f && !src.q)) return CADNN_E_ARG;
-    const cadnn_layer_desc &d = *desc;
+    cadnn_layer_desc dn = *desc;
+    if (dn.pad_w < 0) dn.pad_w = dn.pad;   // from here on pad = rows, pad_w = columns
+    const cadnn_layer_desc &d = dn;
     if (d.c_in < 1 || d.c_out < 1 || d.kh < 1 || d.kw < 1 || d.stride < 1 || d.pad < 0 || d.groups < 1 ||
         d.in_h < 1 || d.in_w < 1)
         return CADNN_E_ARG;
     if (d.dtype != CADNN_F32 && d.dtype != CADNN_S8) return CADNN_E_DTYPE;
     if (d.dtype == CADNN_S8 && !src.q && !src.w_scale) return CADNN_E_ARG;
     if (d.dtype == CADNN_F32 && (src.q || src.w_scale)) return CADNN_E_DTYPE;
-    if (d.in_h + 2 * d.pad < d.kh || d.in_w + 2 * d.pad < d.kw) return CADNN_E_SHAPE;
-    if (d.pad >= d.kh || d.pad >= d.kw) return CADNN_E_UNSUPPORTED;
+    if (d.in_h + 2 * d.pad < d.kh || d.in_w + 2 * d.pad_w < d.kw) return CADNN_E_SHAPE;
+    if (d.pad >= d.kh || d.pad_w >= d.kw) return CADNN_E_UNSUPPORTED;
     const bool depthwise = d.groups > 1 && d.groups == d.c_in && d.c_in == d.c_out;
     if (d.groups != 1 && !depthwise) return CADNN_E_UNSUPPORTED;
     const long K = (long)d.kh * d.kw * d.c_in / d.groups;
@@ -1291,10 +1293,10 @@ cadnn_status pack_common(const cadnn_layer_desc *desc, const Src &src, cadnn_wei
     if (!h) return CADNN_E_ALLOC;
     h->desc = d;
     h->h_out = (d.in_h + 2 * d.pad - d.kh) / d.stride + 1;
-    h->w_out = (d.in_w + 2 * d.pad - d.kw) / d.stride + 1;
+    h->w_out = (d.in_w + 2 * d.pad_w - d.kw) / d.stride + 1;
     cadnn_status st;
     try {
-        const bool is_fc = d.kh == 1 && d.kw == 1 && d.in_h == 1 && d.in_w == 1 && d.pad == 0;
+        const bool is_fc = d.kh == 1 && d.kw == 1 && d.in_h == 1 && d.in_w == 1 && d.pad == 0 && d.pad_w == 0;
         // a float layer with <= 4 input channels whose mask keeps (nearly) everything is a dense stem
         bool dense_stem = false;
         if (!depthwise && d.dtype == CADNN_F32 && d.c_in <= 4 && (d.kh > 1 || d.kw > 1) &&

@@ -39,6 +39,43 @@ __global__ void __launch_bounds__(256) maxpool_kernel(const XT *x, XT *y, int n,
     }
 }
 
+// Max (AVG = false) or average pool into a channel window of a wider output tensor: the branches of an
+// Inception module end in one concatenated tensor, and a pooling branch writes its channels of it
+// directly.  Average: taps in the padding count as zeros, the divisor is always k * k; fp32 sum.
+template <typename XT, bool AVG>
+__global__ void __launch_bounds__(256) pool_window_kernel(const XT *x, XT *y, int n, int h, int w, int c, int h_out,
+                                                          int w_out, int k, int stride, int pad, int ldc, int c_off, float inv)
+{
+    const long long total = (long long)n * h_out * w_out * c;
+    grid_dep_wait();
+    grid_dep_trigger();
+    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int ch = (int)(idx % c);
+        long long pix = idx / c;
+        const int ox = (int)(pix % w_out);
+        long long r = pix / w_out;
+        const int oy = (int)(r % h_out);
+        const int b = (int)(r / h_out);
+        bool any = false;
+        XT best = 0;
+        float sum = 0.0f;
+        for (int ky = 0; ky < k; ++ky) {
+            const int iy = oy * stride + ky - pad;
+            if (iy < 0 || iy >= h) continue;
+            for (int kx = 0; kx < k; ++kx) {
+                const int ix = ox * stride + kx - pad;
+                if (ix < 0 || ix >= w) continue;
+                const XT v = ld_act(x + (((size_t)b * h + iy) * w + ix) * c + ch);
+                if (AVG) sum += (float)v;
+                else if (!any || v > best) best = v;
+                any = true;
+            }
+        }
+        y[(size_t)pix * ldc + c_off + ch] = AVG ? (XT)(sum * inv) : best;
+    }
+}
+
 // 16 bytes per thread: four floats, or sixteen int8 channels (per-byte signed max).
 template <bool S8>
 __global__ void __launch_bounds__(256) maxpool_vec_kernel(const uint4 *x, uint4 *y, int n, int h, int w, int cv,
@@ -121,6 +158,28 @@ cadnn_status launch_maxpool(const void *x, int n, int h, int wd, int c, int k, i
                              wd, c, h_out, w_out, k, stride, pad);
     return launch_kernel(maxpool_kernel<float>, (int)blocks, 256, 0, pdl, st, (const float *)x, (float *)y, n, h, wd, c,
                          h_out, w_out, k, stride, pad);
+}
+
+cadnn_status launch_pool_window(const void *x, int n, int h, int wd, int c, int k, int stride, int pad, int dtype, int kind,
+                                void *y, int ldc, int c_off, bool pdl, cudaStream_t st)
+{
+    if (kind == 0 && (ldc <= 0 || (ldc == c && c_off == 0))) return launch_maxpool(x, n, h, wd, c, k, stride, pad, dtype, y, pdl, st);
+    if (ldc <= 0) { ldc = c; c_off = 0; }
+    const int h_out = (h + 2 * pad - k) / stride + 1, w_out = (wd + 2 * pad - k) / stride + 1;
+    long long total = (long long)n * h_out * w_out * c;
+    if (total <= 0) return CADNN_OK;
+    long long blocks = std::min((total + 255) / 256, 148LL * 64);
+    const float inv = 1.0f / (float)(k * k);
+    if (kind == 1) {
+        if (dtype != CADNN_F32) return CADNN_E_DTYPE;
+        return launch_kernel(pool_window_kernel<float, true>, (int)blocks, 256, 0, pdl, st, (const float *)x, (float *)y, n, h, wd,
+                             c, h_out, w_out, k, stride, pad, ldc, c_off, inv);
+    }
+    if (dtype == CADNN_S8)
+        return launch_kernel(pool_window_kernel<signed char, false>, (int)blocks, 256, 0, pdl, st, (const signed char *)x,
+                             (signed char *)y, n, h, wd, c, h_out, w_out, k, stride, pad, ldc, c_off, inv);
+    return launch_kernel(pool_window_kernel<float, false>, (int)blocks, 256, 0, pdl, st, (const float *)x, (float *)y, n, h, wd, c,
+                         h_out, w_out, k, stride, pad, ldc, c_off, inv);
 }
 
 cadnn_status launch_gavgpool(const float *x, int n, int h, int wd, int c, float *y, bool pdl, cudaStream_t st)

@@ -37,7 +37,8 @@ struct SconvParams {
     const float *bias;
     const void *residual;
     int n, h, w, c_in, h_out, w_out, c_out;
-    int stride, pad;
+    int stride, pad, pad_w;
+    int ldc, c_off;   // channels per output pixel of y and first channel written (a window of a wider tensor for concatenations)
     int BW, RB, TBX, TBY, TH, TW, pitch, half, IH_t, IW_t;
     int CIc, PPb, n_chunks, G, n_groups, stages, esz;
     int ksplit;   // thread blocks per cluster; each takes a contiguous range of the channel chunks
@@ -123,7 +124,7 @@ __device__ __forceinline__ void build_pixel_table(const SconvParams &p, int2 *pi
             pix[q] = make_int2(src, q * p.PPb);
         }
     } else {
-        const int iy0 = oy0 * p.stride - p.pad, ix0 = ox0 * p.stride - p.pad;
+        const int iy0 = oy0 * p.stride - p.pad, ix0 = ox0 * p.stride - p.pad_w;
         for (int i = tid; i < npx; i += NT) {
             int r = i / p.IW_t, col = i - r * p.IW_t;
             int iy = iy0 + r, ix = ix0 + col;
@@ -422,7 +423,7 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
     const int co_base = grp * G;
     const int gw = min(G, p.c_out - co_base);  // real channels in this block
     const bool has_res = p.residual != nullptr;
-    const bool quad = ((gw & 3) == 0) && ((p.c_out & 3) == 0);
+    const bool quad = ((gw & 3) == 0) && ((p.c_out & 3) == 0) && ((p.ldc & 3) == 0) && ((p.c_off & 3) == 0);
     const int cols = quad ? (gw >> 2) : gw;
     const bool full = quad && gw == G;   // the usual case: a precomputed divisor
     for (int idx = tid + q_lo * cols; idx < q_hi * cols; idx += blockDim.x) {
@@ -442,7 +443,8 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
         }
         const int lc = quad ? cq * 4 : cq;
         const int co = co_base + lc;
-        const size_t oi = (size_t)opix * p.c_out + co;
+        const size_t ri = (size_t)opix * p.c_out + co;              // residual: a tensor of exactly c_out channels
+        const size_t oi = (size_t)opix * p.ldc + p.c_off + co;      // output: possibly a channel window of a wider tensor
         const AT *a = sOut + q * op + lc;
         if (quad) {
             float sc[4], bi[4];
@@ -453,7 +455,7 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
             }
             if (sizeof(XT) == 4) {
                 float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (has_res) r = *reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(p.residual) + oi);
+                if (has_res) r = *reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(p.residual) + ri);
                 float4 o;
                 o.x = act_f32(fmaf((float)a[0], sc[0], bi[0]) + r.x, p.act);
                 o.y = act_f32(fmaf((float)a[1], sc[1], bi[1]) + r.y, p.act);
@@ -482,7 +484,7 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
             const float bi = sBias[lc];
             if (sizeof(XT) == 4) {
                 float z = fmaf((float)a[0], sc, bi);
-                if (has_res) z += reinterpret_cast<const float *>(p.residual)[oi];
+                if (has_res) z += reinterpret_cast<const float *>(p.residual)[ri];
                 reinterpret_cast<float *>(p.y)[oi] = act_f32(z, p.act);
             } else if (p.out_dtype == CADNN_S32) {
                 reinterpret_cast<int *>(p.y)[oi] = (int)a[0];
@@ -579,7 +581,8 @@ cadnn_status launch_sconv(const cadnn_weights *w, const void *x, int n, void *y,
     p.residual = ep.residual;
     p.n = n; p.h = d.in_h; p.w = d.in_w; p.c_in = d.c_in;
     p.h_out = w->h_out; p.w_out = w->w_out; p.c_out = d.c_out;
-    p.stride = d.stride; p.pad = d.pad;
+    p.stride = d.stride; p.pad = d.pad; p.pad_w = d.pad_w;
+    p.ldc = ep.out_c_total > 0 ? ep.out_c_total : d.c_out; p.c_off = ep.out_c_total > 0 ? ep.out_c_off : 0;
     p.BW = s.BW; p.RB = s.RB; p.TBX = s.TBX; p.TBY = s.TBY; p.TH = s.TH; p.TW = s.TW;
     p.pitch = s.pitch; p.half = s.half; p.IH_t = s.IH_t; p.IW_t = s.IW_t;
     p.CIc = s.CIc; p.PPb = s.PPb; p.n_chunks = s.n_chunks; p.G = s.G; p.n_groups = s.n_groups;

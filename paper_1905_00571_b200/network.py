@@ -10,8 +10,9 @@ from . import binding as B
 def desc_for(op, dtype, batch_hint=1, autotune=False):
     if op.kind == "fc":
         return B.make_desc(op.c_in, op.c_out, 1, 1, 1, 0, 1, 1, 1, batch_hint, dtype, autotune=autotune)
-    return B.make_desc(op.c_in, op.c_out, op.k, op.k, op.stride, op.pad, op.groups,
-                       op.in_hw[0], op.in_hw[1], batch_hint, dtype, autotune=autotune)
+    kh, kw = int(op.w.shape[1]), int(op.w.shape[2])   # rectangular kernels carry their own shape
+    return B.make_desc(op.c_in, op.c_out, kh, kw, op.stride, op.pad, op.groups,
+                       op.in_hw[0], op.in_hw[1], batch_hint, dtype, autotune=autotune, pad_w=getattr(op, "pad_w", -1))
 
 
 def pack_op(op, dtype, batch_hint=1, autotune=False):
@@ -41,12 +42,12 @@ class PackedModel:
                     self.vecs[i] = (sc, bi)
                     ops.append(B.Op(B.OP_CONV if op.kind == "conv" else B.OP_FC, w.handle, op.src, op.dst, op.res,
                                     None if sc is None else sc.data_ptr(), None if bi is None else bi.data_ptr(),
-                                    B.ACT[op.act], B.DTYPE[op.out], 0, 0, 0))
-                elif op.kind == "maxpool":
-                    ops.append(B.Op(B.OP_MAXPOOL, None, op.src, op.dst, -1, None, None, 0, B.DTYPE[model.dtype],
-                                    op.k, op.stride, op.pad))
+                                    B.ACT[op.act], B.DTYPE[op.out], 0, 0, 0, op.dst_off, op.dst_total))
+                elif op.kind in ("maxpool", "avgpool"):
+                    ops.append(B.Op(B.OP_MAXPOOL if op.kind == "maxpool" else B.OP_AVGPOOL, None, op.src, op.dst, -1, None, None,
+                                    0, B.DTYPE[model.dtype], op.k, op.stride, op.pad, op.dst_off, op.dst_total))
                 elif op.kind == "gavgpool":
-                    ops.append(B.Op(B.OP_GAVGPOOL, None, op.src, op.dst, -1, None, None, 0, B.F32, 0, 0, 0))
+                    ops.append(B.Op(B.OP_GAVGPOOL, None, op.src, op.dst, -1, None, None, 0, B.F32, 0, 0, 0, 0, 0))
                 else:
                     raise ValueError(op.kind)
             h, w_, c = model.in_shape

@@ -28,6 +28,10 @@ def build(workload, density):
         return models.mobilenet_v2(density=density)
     if workload == "vgg16":
         return models.vgg16(density=density, fc_density=min(1.0, density / 2))
+    if workload == "mobilenet_v1":
+        return models.mobilenet_v1(density=density)
+    if workload == "inception_v3":
+        return models.inception_v3(density=density, fc_density=0.10 if density < 1.0 else 1.0)
     raise SystemExit("unknown workload " + workload)
 
 
@@ -52,9 +56,11 @@ def torch_dense_ms(model, batch, tf32, reps=20):
     layers = []
     for op in model.ops:
         if op.kind == "conv":
-            w = torch.randn(op.c_out, op.c_in // op.groups, op.k, op.k, device="cuda").contiguous(memory_format=torch.channels_last)
+            kh, kw = int(op.w.shape[1]), int(op.w.shape[2])
+            pad = (op.pad, op.pad if getattr(op, "pad_w", -1) < 0 else op.pad_w)
+            w = torch.randn(op.c_out, op.c_in // op.groups, kh, kw, device="cuda").contiguous(memory_format=torch.channels_last)
             xin = torch.randn(batch, op.c_in, op.in_hw[0], op.in_hw[1], device="cuda").contiguous(memory_format=torch.channels_last)
-            layers.append((lambda xin=xin, w=w, op=op: torch.nn.functional.conv2d(xin, w, None, op.stride, op.pad, 1, op.groups)))
+            layers.append((lambda xin=xin, w=w, op=op, pad=pad: torch.nn.functional.conv2d(xin, w, None, op.stride, pad, 1, op.groups)))
         elif op.kind == "fc":
             w = torch.randn(op.c_out, op.c_in, device="cuda")
             xin = torch.randn(batch, op.c_in, device="cuda")

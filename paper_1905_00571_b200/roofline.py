@@ -50,7 +50,7 @@ def layer_work(op, batch, dtype):
         res_b = out_b if op.res >= 0 else 0
         return {"flops": flops, "wbytes": wbytes, "abytes": in_b + out_b + res_b, "nnz": nnz, "pixels": pixels}
     in_b = batch * hi * wi * op.c_in * esz
-    out_b = batch * ho * wo * op.c_out * esz
+    out_b = batch * ho * wo * op.c_out * (4 if op.kind == "gavgpool" else esz)
     return {"flops": 0.0, "wbytes": 0, "abytes": in_b + out_b, "nnz": 0, "pixels": batch * ho * wo}
 
 
@@ -65,7 +65,7 @@ def family(op):
     if op.kind == "conv":
         if op.groups > 1:
             return "dwconv"
-        return "sconv_1x1" if (op.k == 1) else "sconv_kxk"
+        return "sconv_1x1" if (op.w.shape[1] * op.w.shape[2] == 1) else "sconv_kxk"
     if op.kind == "fc":
         return "sfc"
     return op.kind

@@ -87,3 +87,27 @@ def test_mobilenet_v1_counts_and_health():
         sd = float(slots[op.dst].std())
         assert 0.1 < sd < 10.0, (op.name, sd)
     assert y.shape == (1, 1000) and np.isfinite(y).all()
+
+
+def test_inception_v3_counts_and_health():
+    m = models.inception_v3()
+    convs = [o for o in m.ops if o.kind == "conv"]
+    assert len(convs) == 94 and sum(o.kind == "fc" for o in m.ops) == 1
+    assert sum(o.w.size for o in m.weight_ops()) == 23799136
+    shapes = {(o.w.shape[1], o.w.shape[2]) for o in convs}
+    assert {(1, 7), (7, 1), (1, 3), (3, 1), (5, 5), (3, 3), (1, 1)} <= shapes
+    assert sum(o.kind == "avgpool" for o in m.ops) == 9 and sum(o.kind == "maxpool" for o in m.ops) == 4
+    # every concatenated slot is covered exactly once by its writers' windows
+    cover = {}
+    for o in m.ops:
+        if o.dst_total:
+            cover.setdefault(o.dst, []).append((o.dst_off, o.c_out, o.dst_total))
+    assert len(cover) == 11
+    for dst, wins in cover.items():
+        wins.sort()
+        assert wins[0][0] == 0 and all(a[0] + a[1] == b[0] for a, b in zip(wins, wins[1:])) and wins[-1][0] + wins[-1][1] == wins[-1][2]
+    y, slots = forward.forward(m, models.make_input(m, 1))
+    for op in m.ops:
+        sd = float(slots[op.dst].std())
+        assert 0.05 < sd < 20.0, (op.name, sd)
+    assert slots[m.ops[-3].dst].shape == (1, 8, 8, 2048) and y.shape == (1, 1000) and np.isfinite(y).all()

@@ -78,9 +78,12 @@ _GAMMA_RMS = np.sqrt(1.0 + 1.0 / 12.0)   # rms of U(0.5, 1.5)
 
 
 def _f32_conv(m, g, name, src, c_in, c_out, k, stride, pad, h, act, density,
-              groups=1, res=-1, gain=1.0, prune="magnitude"):
+              groups=1, res=-1, gain=1.0, prune="magnitude", kw=None, pad_w=None, dst=None, dst_off=0, dst_total=0):
+    """One float conv op (square k x k kernel unless kw is given; pad_w pads the columns when it
+    differs from pad).  dst / dst_off / dst_total: write a channel window of an existing slot."""
     cg = c_in // groups
-    w = gen.he_weights(g, c_out, k, k, cg)
+    kw = k if kw is None else kw
+    w = gen.he_weights(g, c_out, k, kw, cg)
     if density >= 1.0:
         mask = None
         kept = 1.0
@@ -92,10 +95,13 @@ def _f32_conv(m, g, name, src, c_in, c_out, k, stride, pad, h, act, density,
     if act == "none":
         layer_gain /= np.sqrt(2.0)
     scale, bias = gen.folded_bn(g, c_out, gain=layer_gain)
-    dst = m.new_slot()
+    if dst is None:
+        dst = m.new_slot()
     ho = _hw_out(h, k, stride, pad)
+    wo = _hw_out(h, kw, stride, pad if pad_w is None else pad_w)
     m.ops.append(Op("conv", name, src, dst, res, c_in, c_out, k, stride, pad, groups, act,
-                    w, mask, scale, bias, "f32", density, (h, h), (ho, ho)))
+                    w, mask, scale, bias, "f32", density, (h, h), (ho, wo),
+                    pad_w=-1 if pad_w is None else pad_w, dst_off=dst_off, dst_total=dst_total))
     return dst, ho
 
 
@@ -210,6 +216,119 @@ def mobilenet_v1(seed=5, density=0.25, width=1.0, image=224, classes=1000):
     dst = m.new_slot()
     m.ops.append(Op("gavgpool", "avgpool", cur, dst, c_in=c_in, c_out=c_in, in_hw=(h, h), out_hw=(1, 1)))
     _f32_fc(m, g, "fc", dst, c_in, classes, density)
+    return m
+
+
+def inception_v3(seed=6, density=0.125, fc_density=0.10, width=1.0, image=299, classes=1000):
+    """Inception-V3 (Table 2 of the paper): the 3x3 s2 stem conv dense, the other 93 convs (1x1, 3x3,
+    5x5, 1x7, 7x1, 1x3, 3x1) magnitude-pruned to `density`, the classifier to `fc_density`; every conv is
+    Conv + folded BatchNorm + ReLU.  The branches of a module write their channel windows of one
+    concatenated tensor; average pools count padded taps as zeros (divisor k*k)."""
+    g = gen.rng(seed)
+    m = Model("inception_v3", "f32", (image, image, 3), seed=seed)
+    ch = lambda c: max(8, int(round(c * width / 8.0)) * 8)
+
+    def conv(name, src, c_in, c_out, h, k=1, stride=1, pad=0, kw=None, pad_w=None, dens=density, **kwargs):
+        return _f32_conv(m, g, name, src, c_in, c_out, k, stride, pad, h, "relu", dens, kw=kw, pad_w=pad_w, **kwargs)
+
+    def pool(kind, name, src, c, h, k, stride, pad, dst=None, dst_off=0, dst_total=0):
+        if dst is None:
+            dst = m.new_slot()
+        ho = _hw_out(h, k, stride, pad)
+        m.ops.append(Op(kind, name, src, dst, k=k, stride=stride, pad=pad, c_in=c, c_out=c, in_hw=(h, h), out_hw=(ho, ho),
+                        dst_off=dst_off, dst_total=dst_total))
+        return dst, ho
+
+    cur, h = conv("conv1a", 0, 3, ch(32), image, 3, 2, 0, dens=1.0)
+    cur, h = conv("conv2a", cur, ch(32), ch(32), h, 3, 1, 0)
+    cur, h = conv("conv2b", cur, ch(32), ch(64), h, 3, 1, 1)
+    cur, h = pool("maxpool", "pool1", cur, ch(64), h, 3, 2, 0)
+    cur, h = conv("conv3b", cur, ch(64), ch(80), h, 1)
+    cur, h = conv("conv4a", cur, ch(80), ch(192), h, 3, 1, 0)
+    cur, h = pool("maxpool", "pool2", cur, ch(192), h, 3, 2, 0)
+    c_in = ch(192)
+
+    def module_a(nm, src, c_in, h, pool_features):
+        total = ch(64) + ch(64) + ch(96) + ch(pool_features)
+        out = m.new_slot()
+        off = 0
+        conv(nm + ".b1", src, c_in, ch(64), h, dst=out, dst_off=off, dst_total=total); off += ch(64)
+        t, _ = conv(nm + ".b5a", src, c_in, ch(48), h)
+        conv(nm + ".b5b", t, ch(48), ch(64), h, 5, 1, 2, dst=out, dst_off=off, dst_total=total); off += ch(64)
+        t, _ = conv(nm + ".b3a", src, c_in, ch(64), h)
+        t, _ = conv(nm + ".b3b", t, ch(64), ch(96), h, 3, 1, 1)
+        conv(nm + ".b3c", t, ch(96), ch(96), h, 3, 1, 1, dst=out, dst_off=off, dst_total=total); off += ch(96)
+        t, _ = pool("avgpool", nm + ".pool", src, c_in, h, 3, 1, 1)
+        conv(nm + ".bp", t, c_in, ch(pool_features), h, dst=out, dst_off=off, dst_total=total)
+        return out, total
+
+    def module_b(nm, src, c_in, h):
+        total = ch(384) + ch(96) + c_in
+        out = m.new_slot()
+        _, ho = conv(nm + ".b3", src, c_in, ch(384), h, 3, 2, 0, dst=out, dst_off=0, dst_total=total)
+        t, _ = conv(nm + ".bda", src, c_in, ch(64), h)
+        t, _ = conv(nm + ".bdb", t, ch(64), ch(96), h, 3, 1, 1)
+        conv(nm + ".bdc", t, ch(96), ch(96), h, 3, 2, 0, dst=out, dst_off=ch(384), dst_total=total)
+        pool("maxpool", nm + ".pool", src, c_in, h, 3, 2, 0, dst=out, dst_off=ch(384) + ch(96), dst_total=total)
+        return out, total, ho
+
+    def module_c(nm, src, c_in, h, c7):
+        c7 = ch(c7)
+        total = 4 * ch(192)
+        out = m.new_slot()
+        conv(nm + ".b1", src, c_in, ch(192), h, dst=out, dst_off=0, dst_total=total)
+        t, _ = conv(nm + ".b7a", src, c_in, c7, h)
+        t, _ = conv(nm + ".b7b", t, c7, c7, h, 1, 1, 0, kw=7, pad_w=3)
+        conv(nm + ".b7c", t, c7, ch(192), h, 7, 1, 3, kw=1, pad_w=0, dst=out, dst_off=ch(192), dst_total=total)
+        t, _ = conv(nm + ".bda", src, c_in, c7, h)
+        t, _ = conv(nm + ".bdb", t, c7, c7, h, 7, 1, 3, kw=1, pad_w=0)
+        t, _ = conv(nm + ".bdc", t, c7, c7, h, 1, 1, 0, kw=7, pad_w=3)
+        t, _ = conv(nm + ".bdd", t, c7, c7, h, 7, 1, 3, kw=1, pad_w=0)
+        conv(nm + ".bde", t, c7, ch(192), h, 1, 1, 0, kw=7, pad_w=3, dst=out, dst_off=2 * ch(192), dst_total=total)
+        t, _ = pool("avgpool", nm + ".pool", src, c_in, h, 3, 1, 1)
+        conv(nm + ".bp", t, c_in, ch(192), h, dst=out, dst_off=3 * ch(192), dst_total=total)
+        return out, total
+
+    def module_d(nm, src, c_in, h):
+        total = ch(320) + ch(192) + c_in
+        out = m.new_slot()
+        t, _ = conv(nm + ".b3a", src, c_in, ch(192), h)
+        _, ho = conv(nm + ".b3b", t, ch(192), ch(320), h, 3, 2, 0, dst=out, dst_off=0, dst_total=total)
+        t, _ = conv(nm + ".b7a", src, c_in, ch(192), h)
+        t, _ = conv(nm + ".b7b", t, ch(192), ch(192), h, 1, 1, 0, kw=7, pad_w=3)
+        t, _ = conv(nm + ".b7c", t, ch(192), ch(192), h, 7, 1, 3, kw=1, pad_w=0)
+        conv(nm + ".b7d", t, ch(192), ch(192), h, 3, 2, 0, dst=out, dst_off=ch(320), dst_total=total)
+        pool("maxpool", nm + ".pool", src, c_in, h, 3, 2, 0, dst=out, dst_off=ch(320) + ch(192), dst_total=total)
+        return out, total, ho
+
+    def module_e(nm, src, c_in, h):
+        total = ch(320) + 4 * ch(384) + ch(192)
+        out = m.new_slot()
+        off = 0
+        conv(nm + ".b1", src, c_in, ch(320), h, dst=out, dst_off=off, dst_total=total); off += ch(320)
+        t, _ = conv(nm + ".b3a", src, c_in, ch(384), h)
+        conv(nm + ".b3b", t, ch(384), ch(384), h, 1, 1, 0, kw=3, pad_w=1, dst=out, dst_off=off, dst_total=total); off += ch(384)
+        conv(nm + ".b3c", t, ch(384), ch(384), h, 3, 1, 1, kw=1, pad_w=0, dst=out, dst_off=off, dst_total=total); off += ch(384)
+        t, _ = conv(nm + ".bda", src, c_in, ch(448), h)
+        t, _ = conv(nm + ".bdb", t, ch(448), ch(384), h, 3, 1, 1)
+        conv(nm + ".bdc", t, ch(384), ch(384), h, 1, 1, 0, kw=3, pad_w=1, dst=out, dst_off=off, dst_total=total); off += ch(384)
+        conv(nm + ".bdd", t, ch(384), ch(384), h, 3, 1, 1, kw=1, pad_w=0, dst=out, dst_off=off, dst_total=total); off += ch(384)
+        t, _ = pool("avgpool", nm + ".pool", src, c_in, h, 3, 1, 1)
+        conv(nm + ".bp", t, c_in, ch(192), h, dst=out, dst_off=off, dst_total=total)
+        return out, total
+
+    cur, c_in = module_a("m5b", cur, c_in, h, 32)
+    cur, c_in = module_a("m5c", cur, c_in, h, 64)
+    cur, c_in = module_a("m5d", cur, c_in, h, 64)
+    cur, c_in, h = module_b("m6a", cur, c_in, h)
+    for nm, c7 in (("m6b", 128), ("m6c", 160), ("m6d", 160), ("m6e", 192)):
+        cur, c_in = module_c(nm, cur, c_in, h, c7)
+    cur, c_in, h = module_d("m7a", cur, c_in, h)
+    cur, c_in = module_e("m7b", cur, c_in, h)
+    cur, c_in = module_e("m7c", cur, c_in, h)
+    dst = m.new_slot()
+    m.ops.append(Op("gavgpool", "avgpool", cur, dst, c_in=c_in, c_out=c_in, in_hw=(h, h), out_hw=(1, 1)))
+    _f32_fc(m, g, "fc", dst, c_in, classes, fc_density)
     return m
 
 
