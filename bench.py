@@ -34,6 +34,8 @@ def build_model(name):
         return models.inception_v3(), "inception_v3_299_conv12.5pct_fc10pct_stem_dense"
     if name == "mobilenet_v1":
         return models.mobilenet_v1(), "mobilenet_v1_1.0_224_pointwise25pct"
+    if name == "resnet50_int8":
+        return models.resnet50_int8(), "resnet50_v1.5_int8_224_conv12.5pct_fc10pct"
     if name == "single":
         return models.single_layer(), "conv3x3_64to64_56x56_10pct"
     raise SystemExit("unknown workload " + name)

@@ -166,9 +166,12 @@ void cadnn_free_weights(cadnn_weights *w); /* the same call under the name the p
  *                scale = s_x * s_w[co] / s_y, bias = b[co] / s_y, both precomputed by
  *                the caller); ReLU; out_dtype S8: clamp to [-127,127], round half even;
  *                F32: t as is; S32: the raw accumulator (scale / bias / act ignored).
- *                residual must be NULL and ReLU6 is not defined.
- * scale, bias: device float [c_out], NULL = 1 / 0.  residual: device, same shape and
- * dtype as y, or NULL.
+ *                An int8 residual (a quantized residual block; y's shape, dtype S8) joins with a
+ *                second fused multiply-add before the ReLU: t = fmaf((float)r, residual_scale, t),
+ *                residual_scale = s_r / s_y precomputed by the caller (sparse conv layers, S8 or
+ *                F32 output).  ReLU6 is not defined.
+ * scale, bias: device float [c_out], NULL = 1 / 0.  residual: device, same shape as y and of
+ * the layer's dtype, or NULL.
  * Channel concatenation (the branches of an Inception module, Section 5 / Table 2): with
  * out_c_total > 0, y has out_c_total channels per pixel and the layer writes channels
  * [out_c_off, out_c_off + c_out) of it, leaving the others alone; 0 = y has exactly c_out
@@ -183,6 +186,7 @@ typedef struct {
     int out_dtype;   /* cadnn_dtype of y */
     int out_c_total; /* channels per pixel of y, 0 = c_out */
     int out_c_off;   /* first channel of y this layer writes */
+    float residual_scale; /* int8 layers with a residual */
 } cadnn_epilogue;
 
 /*
@@ -244,6 +248,7 @@ typedef struct {
     int act;                  /* cadnn_act */
     int out_dtype;            /* cadnn_dtype of the dst slot */
     int pool_k, pool_stride, pool_pad; /* max / average pool only */
+    float res_scale;            /* int8 conv with a residual: multiplier of the residual (s_r / s_y) */
     int dst_c_off, dst_c_total; /* conv and pools: the op writes channels [dst_c_off, dst_c_off + c) of a dst slot
                                    that has dst_c_total channels (channel concatenation); 0, 0 = the whole slot */
 } cadnn_op;

@@ -37,15 +37,15 @@ class LayerDesc(ctypes.Structure):
 class Epilogue(ctypes.Structure):
     _fields_ = [("scale", ctypes.c_void_p), ("bias", ctypes.c_void_p), ("residual", ctypes.c_void_p),
                 ("act", ctypes.c_int), ("out_dtype", ctypes.c_int), ("out_c_total", ctypes.c_int),
-                ("out_c_off", ctypes.c_int)]
+                ("out_c_off", ctypes.c_int), ("residual_scale", ctypes.c_float)]
 
 
 class Op(ctypes.Structure):
     _fields_ = [("kind", ctypes.c_int), ("w", ctypes.c_void_p), ("src", ctypes.c_int), ("dst", ctypes.c_int),
                 ("res", ctypes.c_int), ("scale", ctypes.c_void_p), ("bias", ctypes.c_void_p),
                 ("act", ctypes.c_int), ("out_dtype", ctypes.c_int), ("pool_k", ctypes.c_int),
-                ("pool_stride", ctypes.c_int), ("pool_pad", ctypes.c_int), ("dst_c_off", ctypes.c_int),
-                ("dst_c_total", ctypes.c_int)]
+                ("pool_stride", ctypes.c_int), ("pool_pad", ctypes.c_int), ("res_scale", ctypes.c_float),
+                ("dst_c_off", ctypes.c_int), ("dst_c_total", ctypes.c_int)]
 
 
 _vp, _i, _i64p = ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_int64)
@@ -215,20 +215,21 @@ def cadnn_weights_unpack(w):
     return dense, mask
 
 
-def _epilogue(scale, bias, residual, act, out_dtype, out_c_total=0, out_c_off=0):
+def _epilogue(scale, bias, residual, act, out_dtype, out_c_total=0, out_c_off=0, residual_scale=0.0):
     return Epilogue(None if scale is None else scale.data_ptr(), None if bias is None else bias.data_ptr(),
                     None if residual is None else residual.data_ptr(), ACT[act] if not isinstance(act, int) else act,
-                    DTYPE[out_dtype] if not isinstance(out_dtype, int) else out_dtype, out_c_total, out_c_off)
+                    DTYPE[out_dtype] if not isinstance(out_dtype, int) else out_dtype, out_c_total, out_c_off,
+                    float(residual_scale))
 
 
 def cadnn_conv2d(w, x, y, scale=None, bias=None, residual=None, act="none", out_dtype=None, stream=None,
-                 out_c_total=0, out_c_off=0):
+                 out_c_total=0, out_c_off=0, residual_scale=0.0):
     """x, y: torch CUDA tensors, NHWC contiguous; y is written in place (channels [out_c_off, out_c_off + c_out)
     of it when out_c_total > 0)."""
     n, h, wd = int(x.shape[0]), int(x.shape[1]), int(x.shape[2])
     if out_dtype is None:
         out_dtype = w.desc.dtype
-    ep = _epilogue(scale, bias, residual, act, out_dtype, out_c_total, out_c_off)
+    ep = _epilogue(scale, bias, residual, act, out_dtype, out_c_total, out_c_off, residual_scale)
     _check(_lib.cadnn_conv2d(w.handle, _dev_ptr(x), n, h, wd, _dev_ptr(y), ctypes.byref(ep), _stream(stream)),
            "cadnn_conv2d")
     return y

@@ -47,6 +47,7 @@ cadnn_status check_epilogue(const cadnn_weights *w, const cadnn_epilogue *ep, La
     le.out_dtype = ep->out_dtype;
     le.out_c_total = ep->out_c_total;
     le.out_c_off = ep->out_c_off;
+    le.res_scale = ep->residual_scale;
     if (le.out_c_total < 0 || le.out_c_off < 0) return CADNN_E_ARG;
     if (le.out_c_total > 0) {   // a channel window of a wider output: sparse conv kernels only, no residual
         if (le.out_c_off + w->desc.c_out > le.out_c_total) return CADNN_E_SHAPE;
@@ -58,7 +59,9 @@ cadnn_status check_epilogue(const cadnn_weights *w, const cadnn_epilogue *ep, La
         if (le.out_dtype != CADNN_F32) return CADNN_E_DTYPE;
     } else {
         if (le.out_dtype != CADNN_S8 && le.out_dtype != CADNN_S32 && le.out_dtype != CADNN_F32) return CADNN_E_DTYPE;
-        if (le.residual) return CADNN_E_UNSUPPORTED;
+        // an int8 residual joins the requantization in the sparse conv kernels only, and never a raw accumulator
+        if (le.residual && (le.out_dtype == CADNN_S32 || (w->s.kind != KK_SCONV_SPATIAL && w->s.kind != KK_SCONV_LINEAR)))
+            return CADNN_E_UNSUPPORTED;
         if (le.act == CADNN_ACT_RELU6) return CADNN_E_UNSUPPORTED;
     }
     if (le.residual && !aligned16(le.residual)) return CADNN_E_ARG;
@@ -76,7 +79,7 @@ cadnn_status check_layer_call(const cadnn_weights *w, bool has_residual, int act
     cadnn_epilogue ep;
     alignas(16) static const char some_residual[16] = {0};   // only its presence matters here
     ep.scale = nullptr; ep.bias = nullptr; ep.residual = has_residual ? some_residual : nullptr;
-    ep.act = act; ep.out_dtype = out_dtype; ep.out_c_total = out_c_total; ep.out_c_off = out_c_off;
+    ep.act = act; ep.out_dtype = out_dtype; ep.out_c_total = out_c_total; ep.out_c_off = out_c_off; ep.residual_scale = 0.0f;
     LaunchEpilogue le;
     return check_epilogue(w, &ep, le);
 }

@@ -144,6 +144,7 @@ struct LaunchEpilogue {
     bool pdl = false;   // launch as a programmatic dependent of the previous kernel (inside cadnn_forward)
     bool early_trigger = false;   // trigger dependents at kernel start instead of before the epilogue
     bool planar_out = false;   // dense stem: write the channel-planar layout instead of NHWC
+    float res_scale = 0.0f;   // int8 layers: multiplier of the int8 residual
     int out_c_total = 0, out_c_off = 0;   // NHWC sparse conv: channel window of a wider output tensor (concatenation)
 };
 

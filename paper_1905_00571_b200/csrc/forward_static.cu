@@ -145,7 +145,8 @@ cadnn_status cadnn_forward_static(const cadnn_op *ops, int n_ops, int n, int h, 
             sn.h = op.w->h_out; sn.w = op.w->w_out; sn.c = d.c_out; sn.dtype = op.out_dtype;
             if (op.res >= 0) {
                 const Tensor &sr = t[op.res];
-                if (!sr.defined || sr.h != sn.h || sr.w != sn.w || sr.c != sn.c || sr.dtype != sn.dtype)
+                const int want_dt = d.dtype == CADNN_S8 ? CADNN_S8 : sn.dtype;   // int8 layers take an int8 residual
+                if (!sr.defined || sr.h != sn.h || sr.w != sn.w || sr.c != sn.c || sr.dtype != want_dt)
                     return CADNN_E_SHAPE;
             }
             // everything the layer call itself would refuse is refused here, before the first launch:
@@ -228,6 +229,7 @@ cadnn_status cadnn_forward_static(const cadnn_op *ops, int n_ops, int n, int h, 
             ep.out_dtype = op.out_dtype;
             ep.out_c_total = op.dst_c_total;
             ep.out_c_off = op.dst_c_off;
+            ep.residual_scale = op.res_scale;
             if (op.kind == CADNN_OP_FC) rc = conv2d_impl(op.w, src, si.n, 1, 1, dst, &ep, false, st);
             else rc = conv2d_impl(op.w, src, si.n, si.h, si.w, dst, &ep, false, st);
         } else if (op.kind == CADNN_OP_MAXPOOL || op.kind == CADNN_OP_AVGPOOL) {

@@ -94,6 +94,7 @@ cadnn_status run_op(cadnn_net *net, const cadnn_op &op, const void *x, void *y, 
         ep.out_dtype = op.out_dtype;
         ep.out_c_total = op.dst_c_total;
         ep.out_c_off = op.dst_c_off;
+        ep.residual_scale = op.res_scale;
         if (op.kind == CADNN_OP_FC) return conv2d_impl(op.w, src, si.n, 1, 1, dst, &ep, pdl, st);
         return conv2d_impl(op.w, src, si.n, si.h, si.w, dst, &ep, pdl, st);
     }
@@ -402,7 +403,9 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
             sn.h = op.w->h_out; sn.w = op.w->w_out; sn.c = d.c_out; sn.dtype = op.out_dtype;
             if (op.res >= 0) {
                 const SlotInfo &sr = net->slots[op.res];
-                if (!sr.defined || sr.h != sn.h || sr.w != sn.w || sr.c != sn.c || sr.dtype != sn.dtype) {
+                // a residual has the output's shape; int8 layers take an int8 residual whatever they store
+                const int want_dt = d.dtype == CADNN_S8 ? CADNN_S8 : sn.dtype;
+                if (!sr.defined || sr.h != sn.h || sr.w != sn.w || sr.c != sn.c || sr.dtype != want_dt) {
                     st = CADNN_E_SHAPE;
                     break;
                 }

@@ -38,6 +38,7 @@ struct SconvParams {
     const void *residual;
     int n, h, w, c_in, h_out, w_out, c_out;
     int stride, pad, pad_w;
+    float res_scale;  // int8 layers: multiplier of the int8 residual
     int ldc, c_off;   // channels per output pixel of y and first channel written (a window of a wider tensor for concatenations)
     int BW, RB, TBX, TBY, TH, TW, pitch, half, IH_t, IW_t;
     int CIc, PPb, n_chunks, G, n_groups, stages, esz;
@@ -73,16 +74,18 @@ __device__ __forceinline__ float act_f32(float z, int act)
     return z;
 }
 
-// int8 layer: one fused multiply-add on the converted accumulator, ReLU
-__device__ __forceinline__ float requant_f32(int acc, float m, float b, int act)
+// int8 layer: one fused multiply-add on the converted accumulator, a second one for the int8 residual
+// of a quantized residual block (r * residual_scale joins before the activation), ReLU
+__device__ __forceinline__ float requant_f32(int acc, float m, float b, int act, bool has_res = false, int r = 0, float rs = 0.0f)
 {
     float t = __fmaf_rn(__int2float_rn(acc), m, b);
+    if (has_res) t = __fmaf_rn(__int2float_rn(r), rs, t);
     if (act == CADNN_ACT_RELU) t = t > 0.0f ? t : 0.0f;
     return t;
 }
-__device__ __forceinline__ int requant_s8(int acc, float m, float b, int act)
+__device__ __forceinline__ int requant_s8(int acc, float m, float b, int act, bool has_res = false, int r = 0, float rs = 0.0f)
 {
-    float t = requant_f32(acc, m, b, act);
+    float t = requant_f32(acc, m, b, act, has_res, r, rs);
     t = fminf(fmaxf(t, -127.0f), 127.0f);
     return __float2int_rn(t);
 }
@@ -465,18 +468,22 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
             } else if (p.out_dtype == CADNN_S32) {
                 *reinterpret_cast<int4 *>(reinterpret_cast<int *>(p.y) + oi) = make_int4((int)a[0], (int)a[1], (int)a[2], (int)a[3]);
             } else if (p.out_dtype == CADNN_F32) {
+                char4 r = make_char4(0, 0, 0, 0);
+                if (has_res) r = *reinterpret_cast<const char4 *>(reinterpret_cast<const int8_t *>(p.residual) + ri);
                 float4 o;
-                o.x = requant_f32((int)a[0], sc[0], bi[0], p.act);
-                o.y = requant_f32((int)a[1], sc[1], bi[1], p.act);
-                o.z = requant_f32((int)a[2], sc[2], bi[2], p.act);
-                o.w = requant_f32((int)a[3], sc[3], bi[3], p.act);
+                o.x = requant_f32((int)a[0], sc[0], bi[0], p.act, has_res, r.x, p.res_scale);
+                o.y = requant_f32((int)a[1], sc[1], bi[1], p.act, has_res, r.y, p.res_scale);
+                o.z = requant_f32((int)a[2], sc[2], bi[2], p.act, has_res, r.z, p.res_scale);
+                o.w = requant_f32((int)a[3], sc[3], bi[3], p.act, has_res, r.w, p.res_scale);
                 *reinterpret_cast<float4 *>(reinterpret_cast<float *>(p.y) + oi) = o;
             } else {
+                char4 r = make_char4(0, 0, 0, 0);
+                if (has_res) r = *reinterpret_cast<const char4 *>(reinterpret_cast<const int8_t *>(p.residual) + ri);
                 char4 o;
-                o.x = (signed char)requant_s8((int)a[0], sc[0], bi[0], p.act);
-                o.y = (signed char)requant_s8((int)a[1], sc[1], bi[1], p.act);
-                o.z = (signed char)requant_s8((int)a[2], sc[2], bi[2], p.act);
-                o.w = (signed char)requant_s8((int)a[3], sc[3], bi[3], p.act);
+                o.x = (signed char)requant_s8((int)a[0], sc[0], bi[0], p.act, has_res, r.x, p.res_scale);
+                o.y = (signed char)requant_s8((int)a[1], sc[1], bi[1], p.act, has_res, r.y, p.res_scale);
+                o.z = (signed char)requant_s8((int)a[2], sc[2], bi[2], p.act, has_res, r.z, p.res_scale);
+                o.w = (signed char)requant_s8((int)a[3], sc[3], bi[3], p.act, has_res, r.w, p.res_scale);
                 *reinterpret_cast<char4 *>(reinterpret_cast<int8_t *>(p.y) + oi) = o;
             }
         } else {
@@ -488,10 +495,12 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
                 reinterpret_cast<float *>(p.y)[oi] = act_f32(z, p.act);
             } else if (p.out_dtype == CADNN_S32) {
                 reinterpret_cast<int *>(p.y)[oi] = (int)a[0];
-            } else if (p.out_dtype == CADNN_F32) {
-                reinterpret_cast<float *>(p.y)[oi] = requant_f32((int)a[0], sc, bi, p.act);
             } else {
-                reinterpret_cast<int8_t *>(p.y)[oi] = (int8_t)requant_s8((int)a[0], sc, bi, p.act);
+                const int r = has_res ? (int)reinterpret_cast<const int8_t *>(p.residual)[ri] : 0;
+                if (p.out_dtype == CADNN_F32)
+                    reinterpret_cast<float *>(p.y)[oi] = requant_f32((int)a[0], sc, bi, p.act, has_res, r, p.res_scale);
+                else
+                    reinterpret_cast<int8_t *>(p.y)[oi] = (int8_t)requant_s8((int)a[0], sc, bi, p.act, has_res, r, p.res_scale);
             }
         }
     }
@@ -582,6 +591,7 @@ cadnn_status launch_sconv(const cadnn_weights *w, const void *x, int n, void *y,
     p.n = n; p.h = d.in_h; p.w = d.in_w; p.c_in = d.c_in;
     p.h_out = w->h_out; p.w_out = w->w_out; p.c_out = d.c_out;
     p.stride = d.stride; p.pad = d.pad; p.pad_w = d.pad_w;
+    p.res_scale = ep.res_scale;
     p.ldc = ep.out_c_total > 0 ? ep.out_c_total : d.c_out; p.c_off = ep.out_c_total > 0 ? ep.out_c_off : 0;
     p.BW = s.BW; p.RB = s.RB; p.TBX = s.TBX; p.TBY = s.TBY; p.TH = s.TH; p.TW = s.TW;
     p.pitch = s.pitch; p.half = s.half; p.IH_t = s.IH_t; p.IW_t = s.IW_t;

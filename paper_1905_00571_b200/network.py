@@ -16,6 +16,7 @@ def desc_for(op, dtype, batch_hint=1, autotune=False):
 
 
 def pack_op(op, dtype, batch_hint=1, autotune=False):
+    dtype = "s8" if op.w.dtype == np.int8 else "f32"   # (an int8 network may end in float layers)
     d = desc_for(op, dtype, batch_hint, autotune)
     if op.w.dtype == np.int8:
         return B.cadnn_pack_q8(d, op.w, op.mask)
@@ -42,12 +43,12 @@ class PackedModel:
                     self.vecs[i] = (sc, bi)
                     ops.append(B.Op(B.OP_CONV if op.kind == "conv" else B.OP_FC, w.handle, op.src, op.dst, op.res,
                                     None if sc is None else sc.data_ptr(), None if bi is None else bi.data_ptr(),
-                                    B.ACT[op.act], B.DTYPE[op.out], 0, 0, 0, op.dst_off, op.dst_total))
+                                    B.ACT[op.act], B.DTYPE[op.out], 0, 0, 0, float(op.res_scale), op.dst_off, op.dst_total))
                 elif op.kind in ("maxpool", "avgpool"):
                     ops.append(B.Op(B.OP_MAXPOOL if op.kind == "maxpool" else B.OP_AVGPOOL, None, op.src, op.dst, -1, None, None,
-                                    0, B.DTYPE[model.dtype], op.k, op.stride, op.pad, op.dst_off, op.dst_total))
+                                    0, B.DTYPE[model.dtype], op.k, op.stride, op.pad, 0.0, op.dst_off, op.dst_total))
                 elif op.kind == "gavgpool":
-                    ops.append(B.Op(B.OP_GAVGPOOL, None, op.src, op.dst, -1, None, None, 0, B.F32, 0, 0, 0, 0, 0))
+                    ops.append(B.Op(B.OP_GAVGPOOL, None, op.src, op.dst, -1, None, None, 0, B.F32, 0, 0, 0, 0.0, 0, 0))
                 else:
                     raise ValueError(op.kind)
             h, w_, c = model.in_shape

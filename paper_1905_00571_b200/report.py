@@ -28,6 +28,8 @@ def build(workload, density):
         return models.mobilenet_v2(density=density)
     if workload == "vgg16":
         return models.vgg16(density=density, fc_density=min(1.0, density / 2))
+    if workload == "resnet50_int8":
+        return models.resnet50_int8(density=density, fc_density=0.10 if density < 1.0 else 1.0)
     if workload == "mobilenet_v1":
         return models.mobilenet_v1(density=density)
     if workload == "inception_v3":

@@ -170,3 +170,48 @@ def test_mobilenet_v1_full_batch1():
     assert B.cadnn_net_layout(pm.net)["planar"]
     want, _ = oracle_forward.forward(m, x)
     _check_logits(got, want)
+
+
+@pytest.mark.parametrize("out", ["s8", "f32"])
+@pytest.mark.parametrize("c_out", [64, 30])
+def test_int8_conv_with_int8_residual_bit_exact(out, c_out):
+    """The shortcut of a quantized residual block: a second fused multiply-add on the int8 residual before the ReLU."""
+    from paper_1905_00571_b200 import binding as B
+    g = gen.rng(300 + c_out)
+    x = gen.int8_relu_activation(g, (2, 9, 10, 48))
+    q = gen.int8_weights(g, (c_out, 3, 3, 48))
+    mask = gen.random_mask(g, q.shape, 0.15)
+    r = gen.int8_relu_activation(g, (2, 9, 10, c_out))
+    m = (g.uniform(0.5, 1.5, size=c_out) * 3e-4).astype(np.float32)
+    b = (g.standard_normal(c_out) * 3).astype(np.float32)
+    want = ref.conv2d_s8(x, q, mask, 1, 1, 1, m, b, "relu", out, r, 0.6)
+    wh = B.cadnn_pack_q8(B.make_desc(48, c_out, 3, 3, 1, 1, 1, 9, 10, 2, "s8"), q, mask)
+    y = torch.zeros(want.shape, dtype=torch.int8 if out == "s8" else torch.float32, device=DEV)
+    dev = lambda a: torch.from_numpy(a).to(DEV)
+    B.cadnn_conv2d(wh, dev(x), y, dev(m), dev(b), dev(r), "relu", out_dtype=out, residual_scale=0.6)
+    torch.cuda.synchronize()
+    assert_exact(y.cpu().numpy(), want, "int8 residual")
+    assert not np.array_equal(want, ref.conv2d_s8(x, q, mask, 1, 1, 1, m, b, "relu", out))
+
+
+@pytest.mark.parametrize("batch", [1, 2])
+def test_resnet50_int8_reduced(batch):
+    from paper_1905_00571_b200 import binding as B
+    m = models.resnet50_int8(width=0.25, image=64, classes=100)
+    x, got, pm = _run(m, batch)
+    want, slots = oracle_forward.forward(m, x)
+    _check_logits(got, want)
+    # everything up to the float tail is integer work: the last int8 tensor matches bit for bit
+    import ctypes
+    last_q = [op for op in m.ops if op.out == "s8"][-1]
+    ptr, nbytes = B.cadnn_net_slot(pm.net, last_q.dst)
+    host = np.empty(nbytes, np.int8)
+    assert ctypes.CDLL("libcudart.so").cudaMemcpy(ctypes.c_void_p(host.ctypes.data), ctypes.c_void_p(ptr), ctypes.c_size_t(nbytes), 2) == 0
+    assert_exact(host[:slots[last_q.dst].size].reshape(slots[last_q.dst].shape), slots[last_q.dst], last_q.name)
+
+
+def test_resnet50_int8_full_batch1():
+    m = models.resnet50_int8()
+    x, got, _ = _run(m, 1)
+    want, _ = oracle_forward.forward(m, x)
+    _check_logits(got, want)

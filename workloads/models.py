@@ -341,7 +341,8 @@ _M2_RELU = 0.5 * _T_RMS ** 2
 _M2_POOLED = 1.3 * _T_RMS ** 2
 
 
-def _s8_layer(m, g, kind, name, src, c_in, c_out, k, pad, h, act, density, m2_in, out="s8"):
+def _s8_layer(m, g, kind, name, src, c_in, c_out, k, pad, h, act, density, m2_in, out="s8", stride=1, res=-1,
+              res_scale=0.0, gain=1.0):
     shape = (c_out, k, k, c_in)
     q = gen.int8_weights(g, shape)
     mask = None if density >= 1.0 else gen.random_mask(g, shape, density)
@@ -350,12 +351,12 @@ def _s8_layer(m, g, kind, name, src, c_in, c_out, k, pad, h, act, density, m2_in
         qq = qq * mask
     row_energy = qq.reshape(c_out, -1).sum(axis=1)
     mult = np.where(row_energy > 0, _T_RMS / np.sqrt(np.maximum(row_energy, 1.0) * m2_in), 1.0)
-    mult = (mult * g.uniform(0.8, 1.25, size=c_out)).astype(np.float32)
+    mult = (mult * gain * g.uniform(0.8, 1.25, size=c_out)).astype(np.float32)
     offs = (g.standard_normal(c_out) * 0.1 * _T_RMS).astype(np.float32)
     dst = m.new_slot()
-    ho = _hw_out(h, k, 1, pad)
-    m.ops.append(Op(kind, name, src, dst, -1, c_in, c_out, k, 1, pad, 1, act, q, mask,
-                    mult, offs, out, density, (h, h), (ho, ho)))
+    ho = _hw_out(h, k, stride, pad)
+    m.ops.append(Op(kind, name, src, dst, res, c_in, c_out, k, stride, pad, 1, act, q, mask,
+                    mult, offs, out, density, (h, h), (ho, ho), res_scale=res_scale))
     return dst
 
 
@@ -384,6 +385,55 @@ def vgg16(seed=3, density=0.08, fc_density=0.04, width=1.0, image=224, classes=1
     cur = _s8_layer(m, g, "fc", "fc6", cur, k_in, fc_width, 1, 0, 1, "relu", fc_density, _M2_POOLED)
     cur = _s8_layer(m, g, "fc", "fc7", cur, fc_width, fc_width, 1, 0, 1, "relu", fc_density, _M2_RELU)
     _s8_layer(m, g, "fc", "fc8", cur, fc_width, classes, 1, 0, 1, "none", fc_density, _M2_RELU, out="f32")
+    return m
+
+
+def resnet50_int8(seed=7, density=0.125, fc_density=0.10, width=1.0, image=224, classes=1000):
+    """ResNet-50 v1.5 with int8 weights and activations (the int8 counterpart of the pruned ResNet-50): dense
+    int8 7x7 stem, every other conv an exactly-k random mask at `density`, an int8 3x3 max pool, the shortcut of
+    a block joining the last conv's requantization as an int8 residual (two fused multiply-adds, then ReLU).
+    The last block stores float32 (no rounding), which feeds a float global average pool and a pruned
+    float classifier."""
+    g = gen.rng(seed)
+    m = Model("resnet50_int8", "s8", (image, image, 3), seed=seed)
+    ch = lambda c: max(8, int(round(c * width)))
+    cur = _s8_layer(m, g, "conv", "conv1", 0, 3, ch(64), 7, 3, image, "relu", 1.0, _M2_IMAGE, stride=2)
+    h = _hw_out(image, 7, 2, 3)
+    dst = m.new_slot()
+    ho = _hw_out(h, 3, 2, 1)
+    m.ops.append(Op("maxpool", "pool1", cur, dst, k=3, stride=2, pad=1, c_in=ch(64), c_out=ch(64),
+                    in_hw=(h, h), out_hw=(ho, ho), out="s8"))
+    cur, h, c_in = dst, ho, ch(64)
+    m2 = _M2_POOLED
+    stages = [(64, 3, 1), (128, 4, 2), (256, 6, 2), (512, 3, 2)]
+    for si, (mid, blocks, stride) in enumerate(stages):
+        mid = ch(mid)
+        out = mid * 4
+        for b in range(blocks):
+            s = stride if b == 0 else 1
+            nm = "s%db%d" % (si + 2, b)
+            last = si == len(stages) - 1 and b == blocks - 1
+            if b == 0:
+                short = _s8_layer(m, g, "conv", nm + ".ds", cur, c_in, out, 1, 0, h, "none", density, m2, stride=s)
+            else:
+                short = cur
+            t = _s8_layer(m, g, "conv", nm + ".c1", cur, c_in, mid, 1, 0, h, "relu", density, m2)
+            t = _s8_layer(m, g, "conv", nm + ".c2", t, mid, mid, 3, 1, h, "relu", density, _M2_RELU, stride=s)
+            h2 = _hw_out(h, 3, s, 1)
+            cur = _s8_layer(m, g, "conv", nm + ".c3", t, mid, out, 1, 0, h2, "relu", density, _M2_RELU,
+                            out="f32" if last else "s8", res=short, res_scale=0.6, gain=0.6)
+            h, c_in, m2 = h2, out, 1.1 * _T_RMS ** 2
+    dst = m.new_slot()
+    m.ops.append(Op("gavgpool", "avgpool", cur, dst, c_in=c_in, c_out=c_in, in_hw=(h, h), out_hw=(1, 1)))
+    # float classifier on the pooled float features (in code units: ~T_RMS)
+    w = gen.he_weights(g, classes, 1, 1, c_in)
+    mask = None if fc_density >= 1.0 else gen.magnitude_mask(w, fc_density)
+    kept = 1.0 if mask is None else gen.kept_energy(w, mask)
+    scale = np.full(classes, 1.0 / (_T_RMS * np.sqrt(2.0 * kept)), np.float32)
+    bias = (g.standard_normal(classes) * 0.1).astype(np.float32)
+    out_slot = m.new_slot()
+    m.ops.append(Op("fc", "fc", dst, out_slot, -1, c_in, classes, 1, 1, 0, 1, "none", w, mask, scale, bias, "f32",
+                    fc_density, (1, 1), (1, 1)))
     return m
 
 
