@@ -55,7 +55,12 @@ typedef enum {
     CADNN_FMT_TILED_CSR = 1,   /* conv: per channel-chunk CSR by output channel, filters regrouped */
     CADNN_FMT_ROW_CSR = 2,     /* fc at small batch: CSR by output channel, rows sorted by length */
     CADNN_FMT_DENSE_DW = 3,    /* dense depthwise filters, tap-major */
-    CADNN_FMT_DENSE_SMALLC = 4 /* dense conv with very few input channels (network stem) */
+    CADNN_FMT_DENSE_SMALLC = 4, /* dense conv with very few input channels (network stem) */
+    CADNN_FMT_GROUPED = 5      /* int8 stride-1 conv with block structure (ask for it in cadnn_layer_desc.fmt): the
+                                  64 output channels x 64 input channels x one tap blocks of which the mask keeps at
+                                  least CADNN_BLOCK_DENSITY (environment, default 0.5) are stored dense and multiplied
+                                  on the tensor cores, the rest stays TILED_CSR; needs c_in and c_out multiples of 64 and
+                                  a caller-provided workspace (cadnn_conv2d_workspace) */
 } cadnn_fmt;
 
 #define CADNN_PACK_HOST_ONLY 1 /* build the packed image on the host only (no device needed, no compute) */
@@ -83,7 +88,7 @@ typedef struct {
     int in_h, in_w;
     int batch_hint;
     int dtype; /* cadnn_dtype of weights and activations: CADNN_F32 or CADNN_S8 */
-    int fmt;   /* cadnn_fmt, CADNN_FMT_AUTO */
+    int fmt;   /* CADNN_FMT_AUTO, or CADNN_FMT_GROUPED to ask for the block-structured int8 format */
     int flags; /* CADNN_PACK_HOST_ONLY, CADNN_PACK_AUTOTUNE or 0 */
     int pad_w; /* padding of the columns; -1 = same as pad */
 } cadnn_layer_desc;
@@ -200,6 +205,23 @@ typedef struct {
  */
 cadnn_status cadnn_conv2d(const cadnn_weights *w, const void *x, int n, int h, int wd, void *y,
                           const cadnn_epilogue *ep, void *stream);
+
+/*
+ * cadnn_conv2d_workspace / cadnn_weights_workspace_bytes - a layer packed as CADNN_FMT_GROUPED runs in two
+ * kernels (Section 1, "computation pattern transformation": structure left by pruning is executed in the form
+ * the processor runs fastest): its dense blocks on the tensor cores into int32 sums, then the sparse kernel
+ * over the remaining nonzeros, which adds those sums to its own before the requantization (integer sums are
+ * exact in any order, so the result is the one the plain sparse layer gives, bit for bit).  The int32 sums
+ * live in a workspace the caller provides: device memory of at least cadnn_weights_workspace_bytes(w, n)
+ * bytes, 16-byte aligned, used only during the call's kernels (stream order).  Other formats need none
+ * (*bytes = 0) and cadnn_conv2d_workspace then equals cadnn_conv2d.  cadnn_conv2d on a GROUPED handle
+ * returns E_ARG.
+ */
+cadnn_status cadnn_weights_workspace_bytes(const cadnn_weights *w, int n, int64_t *bytes);
+cadnn_status cadnn_conv2d_workspace(const cadnn_weights *w, const void *x, int n, int h, int wd, void *y,
+                                    const cadnn_epilogue *ep, void *workspace, int64_t workspace_bytes, void *stream);
+/* How many dense blocks the packer found and how many kept weights they hold (0, 0 for other formats). */
+cadnn_status cadnn_weights_block_info(const cadnn_weights *w, int *n_blocks, int64_t *block_nnz);
 
 /*
  * cadnn_conv2d_planar - the same layer on channel-planar activations (Section 4, "Memory

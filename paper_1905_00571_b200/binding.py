@@ -24,7 +24,8 @@ ACT = {"none": 0, "relu": 1, "relu6": 2, None: 0}
 PACK_HOST_ONLY = 1
 PACK_AUTOTUNE = 2
 OP_CONV, OP_FC, OP_MAXPOOL, OP_GAVGPOOL, OP_AVGPOOL = 0, 1, 2, 3, 4
-FMT_NAMES = {1: "tiled_csr", 2: "row_csr", 3: "dense_dw", 4: "dense_smallc"}
+FMT_NAMES = {1: "tiled_csr", 2: "row_csr", 3: "dense_dw", 4: "dense_smallc", 5: "grouped"}
+FMT_GROUPED = 5
 KIND_NAMES = {1: "sconv_spatial", 2: "sconv_linear", 3: "fc_spmv", 4: "dw", 5: "dense_smallc"}
 
 
@@ -60,6 +61,9 @@ _SIGS = {
     "cadnn_weights_free": (None, [_vp]),
     "cadnn_free_weights": (None, [_vp]),
     "cadnn_conv2d": (_i, [_vp, _vp, _i, _i, _i, _vp, ctypes.POINTER(Epilogue), _vp]),
+    "cadnn_weights_workspace_bytes": (_i, [_vp, _i, _i64p]),
+    "cadnn_conv2d_workspace": (_i, [_vp, _vp, _i, _i, _i, _vp, ctypes.POINTER(Epilogue), _vp, ctypes.c_int64, _vp]),
+    "cadnn_weights_block_info": (_i, [_vp, ctypes.POINTER(_i), _i64p]),
     "cadnn_conv2d_planar": (_i, [_vp, _vp, _i, _vp, ctypes.POINTER(Epilogue), _vp]),
     "cadnn_fc": (_i, [_vp, _vp, _i, _vp, ctypes.POINTER(Epilogue), _vp]),
     "cadnn_maxpool2d": (_i, [_vp, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _vp]),
@@ -142,9 +146,9 @@ class Weights:
 
 
 def make_desc(c_in, c_out, kh=1, kw=1, stride=1, pad=0, groups=1, in_h=1, in_w=1, batch_hint=1,
-              dtype="f32", host_only=False, autotune=False, pad_w=-1):
+              dtype="f32", host_only=False, autotune=False, pad_w=-1, fmt=0):
     flags = (PACK_HOST_ONLY if host_only else 0) | (PACK_AUTOTUNE if autotune else 0)
-    return LayerDesc(c_in, c_out, kh, kw, stride, pad, groups, in_h, in_w, batch_hint, DTYPE[dtype], 0, flags, pad_w)
+    return LayerDesc(c_in, c_out, kh, kw, stride, pad, groups, in_h, in_w, batch_hint, DTYPE[dtype], fmt, flags, pad_w)
 
 
 def cadnn_pack(desc, w_ohwi, mask=None, w_scale=None):
@@ -232,6 +236,32 @@ def cadnn_conv2d(w, x, y, scale=None, bias=None, residual=None, act="none", out_
     ep = _epilogue(scale, bias, residual, act, out_dtype, out_c_total, out_c_off, residual_scale)
     _check(_lib.cadnn_conv2d(w.handle, _dev_ptr(x), n, h, wd, _dev_ptr(y), ctypes.byref(ep), _stream(stream)),
            "cadnn_conv2d")
+    return y
+
+
+def cadnn_weights_workspace_bytes(w, n):
+    b = ctypes.c_int64()
+    _check(_lib.cadnn_weights_workspace_bytes(w.handle, int(n), ctypes.byref(b)), "cadnn_weights_workspace_bytes")
+    return int(b.value)
+
+
+def cadnn_weights_block_info(w):
+    nb, nz = ctypes.c_int(), ctypes.c_int64()
+    _check(_lib.cadnn_weights_block_info(w.handle, ctypes.byref(nb), ctypes.byref(nz)), "cadnn_weights_block_info")
+    return {"blocks": nb.value, "block_nnz": nz.value}
+
+
+def cadnn_conv2d_workspace(w, x, y, workspace, scale=None, bias=None, residual=None, act="none", out_dtype=None, stream=None,
+                           residual_scale=0.0):
+    """cadnn_conv2d for a layer packed as FMT_GROUPED: workspace is a torch CUDA tensor of at least
+    cadnn_weights_workspace_bytes(w, n) bytes (None for other formats)."""
+    n, h, wd = int(x.shape[0]), int(x.shape[1]), int(x.shape[2])
+    if out_dtype is None:
+        out_dtype = w.desc.dtype
+    ep = _epilogue(scale, bias, residual, act, out_dtype, 0, 0, residual_scale)
+    nbytes = 0 if workspace is None else int(workspace.numel() * workspace.element_size())
+    _check(_lib.cadnn_conv2d_workspace(w.handle, _dev_ptr(x), n, h, wd, _dev_ptr(y), ctypes.byref(ep), _dev_ptr(workspace),
+                                       nbytes, _stream(stream)), "cadnn_conv2d_workspace")
     return y
 
 

@@ -85,7 +85,7 @@ cadnn_status check_layer_call(const cadnn_weights *w, bool has_residual, int act
 }
 
 cadnn_status conv2d_impl(const cadnn_weights *w, const void *x, int n, int h, int wd, void *y, const cadnn_epilogue *ep,
-                         bool pdl, cudaStream_t s)
+                         bool pdl, cudaStream_t s, void *workspace, int64_t workspace_bytes)
 {
     if (!w || !x || !y || n < 0) return CADNN_E_ARG;
     if (!w->on_device) return CADNN_E_ARG;
@@ -95,6 +95,15 @@ cadnn_status conv2d_impl(const cadnn_weights *w, const void *x, int n, int h, in
     cadnn_status st = check_epilogue(w, ep, le);
     if (st != CADNN_OK) return st;
     le.pdl = pdl;
+    if (w->has_tc) {
+        // dense blocks on the tensor cores first; the sparse kernel then starts from their int32 sums
+        const int64_t need = (int64_t)n * w->h_out * w->w_out * w->desc.c_out * 4;
+        if (!workspace || !aligned16(workspace) || workspace_bytes < need) return CADNN_E_ARG;
+        st = launch_block_tc(w, x, n, (int *)workspace, s);
+        if (st != CADNN_OK) return st;
+        le.acc_in = (const int *)workspace;
+        le.pdl = false;
+    }
     switch (w->s.kind) {
         case KK_SCONV_SPATIAL:
         case KK_SCONV_LINEAR: return launch_sconv(w, x, n, y, le, s);
@@ -111,6 +120,27 @@ cadnn_status cadnn_conv2d(const cadnn_weights *w, const void *x, int n, int h, i
                           const cadnn_epilogue *ep, void *stream)
 {
     return conv2d_impl(w, x, n, h, wd, y, ep, false, (cudaStream_t)stream);
+}
+
+cadnn_status cadnn_weights_workspace_bytes(const cadnn_weights *w, int n, int64_t *bytes)
+{
+    if (!w || !bytes || n < 0) return CADNN_E_ARG;
+    *bytes = w->has_tc ? (int64_t)n * w->h_out * w->w_out * w->desc.c_out * 4 : 0;
+    return CADNN_OK;
+}
+
+cadnn_status cadnn_conv2d_workspace(const cadnn_weights *w, const void *x, int n, int h, int wd, void *y,
+                                    const cadnn_epilogue *ep, void *workspace, int64_t workspace_bytes, void *stream)
+{
+    return conv2d_impl(w, x, n, h, wd, y, ep, false, (cudaStream_t)stream, workspace, workspace_bytes);
+}
+
+cadnn_status cadnn_weights_block_info(const cadnn_weights *w, int *n_blocks, int64_t *block_nnz)
+{
+    if (!w) return CADNN_E_ARG;
+    if (n_blocks) *n_blocks = w->has_tc ? (int)(w->tc_blk.size() / 4) : 0;
+    if (block_nnz) *block_nnz = w->has_tc ? w->tc_nnz : 0;
+    return CADNN_OK;
 }
 
 cadnn_status cadnn_conv2d_planar(const cadnn_weights *w, const void *x, int n, void *y, const cadnn_epilogue *ep,
@@ -166,12 +196,14 @@ cadnn_status cadnn_device_status(int *copy_timeouts)
 {
     if (!copy_timeouts) return CADNN_E_ARG;
     CADNN_CUDA_TRY(cudaDeviceSynchronize());
-    int copies = 0, barriers = 0;
+    int copies = 0, barriers = 0, tc = 0;
     cadnn_status s = read_copy_timeouts(&copies);
     if (s != CADNN_OK) return s;
     s = read_barrier_timeouts(&barriers);
     if (s != CADNN_OK) return s;
-    *copy_timeouts = copies + barriers;
+    s = read_tc_timeouts(&tc);
+    if (s != CADNN_OK) return s;
+    *copy_timeouts = copies + barriers + tc;
     return CADNN_OK;
 }
 

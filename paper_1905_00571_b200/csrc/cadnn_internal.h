@@ -125,6 +125,19 @@ struct cadnn_weights {
     const uint32_t *d_ps_ent = nullptr;
     const int32_t *d_ps_perm = nullptr;
 
+    // tensor-core blocks of a block-structured int8 layer (blocktc.cu): the dense 64 x 64 blocks, the rest of the
+    // layer stays in the sparse image above
+    bool has_tc = false;
+    std::vector<int8_t> tc_wblk;        // [n_blocks][64 rows][64 bytes], rows = output channels, 16-byte chunks swizzled
+    std::vector<int32_t> tc_blk;        // [n_blocks][4]: column shift, row shift of the tap, first input channel, 0
+    std::vector<int32_t> tc_tile_ptr;   // [c_out / 64 + 1] blocks of every tile of 64 output channels
+    std::vector<uint8_t> tc_kept;       // [n_blocks][64][64] which positions of a block the mask kept (host only, for unpack)
+    int64_t tc_nnz = 0;                 // kept positions inside the dense blocks
+    void *d_tc_blob = nullptr;
+    const int8_t *d_tc_wblk = nullptr;
+    const int32_t *d_tc_blk = nullptr;
+    const int32_t *d_tc_tile_ptr = nullptr;
+
     // device image (one allocation)
     void *d_blob = nullptr;
     const uint32_t *d_ent = nullptr;
@@ -145,6 +158,7 @@ struct LaunchEpilogue {
     bool early_trigger = false;   // trigger dependents at kernel start instead of before the epilogue
     bool planar_out = false;   // dense stem: write the channel-planar layout instead of NHWC
     float res_scale = 0.0f;   // int8 layers: multiplier of the int8 residual
+    const int *acc_in = nullptr;   // int8 sparse conv: int32 sums [pixels][c_out] added to the accumulators before the epilogue
     int out_c_total = 0, out_c_off = 0;   // NHWC sparse conv: channel window of a wider output tensor (concatenation)
 };
 
@@ -185,6 +199,11 @@ cadnn_status launch_sconv_planar_staged(const cadnn_weights *w, const void *x, i
 bool dw_planar_ok(const cadnn_weights *w);   // a depthwise layer the planar layout can run (float, <= 9 taps, pad within the halo)
 cadnn_status launch_dw_planar(const cadnn_weights *w, const void *x, int n, void *y, const LaunchEpilogue &ep,
                               cudaStream_t st);
+// block-structured int8 layers (blocktc.cu)
+bool block_tc_extract(cadnn_weights *h, const int8_t *q, const uint8_t *mask, double threshold, std::vector<uint8_t> &rem_mask);
+cadnn_status block_tc_upload(cadnn_weights *h);
+cadnn_status launch_block_tc(const cadnn_weights *w, const void *x, int n, int *acc, cudaStream_t st);
+cadnn_status read_tc_timeouts(int *count);
 cadnn_status read_copy_timeouts(int *count);
 cadnn_status read_barrier_timeouts(int *count);
 // the same counters copied to (pinned) host memory in stream order, and overwritten (tests)
@@ -198,6 +217,11 @@ cadnn_status write_barrier_timeouts(int value);
 // the matrix read as zero.  False when the driver entry point is missing or refuses the shape.
 bool encode_plane_rows_map(void *map, const void *base, unsigned long long cols, unsigned long long rows,
                            unsigned box_cols, unsigned box_rows);
+
+// Tensor map over an int8 NHWC tensor [n][h][w][c] copied in boxes of box_h x box_w pixels x box_c (= 64) channels,
+// written to shared memory as box_h * box_w rows of 64 bytes with the 64-byte swizzle the tensor cores read;
+// pixels outside an image read as zero.
+bool encode_nhwc_s8_tiles_map(void *map, const void *base, int c, int w, int h, int n, int box_c, int box_w, int box_h);
 
 // Persistent kernel over a run of planar sparse convs (persist.cu).  One entry per conv, in
 // network order; join_phase: the op reads nothing that the ops of the current phase write, so
@@ -236,7 +260,7 @@ cadnn_status launch_gavgpool(const float *x, int n, int h, int wd, int c, float 
 
 // layer entry shared by the public calls and the network runner
 cadnn_status conv2d_impl(const cadnn_weights *w, const void *x, int n, int h, int wd, void *y, const cadnn_epilogue *ep,
-                         bool pdl, cudaStream_t st);
+                         bool pdl, cudaStream_t st, void *workspace = nullptr, int64_t workspace_bytes = 0);
 
 #ifdef __CUDACC__
 // Division by a runtime constant as multiply-high and shift (the divisor is fixed per

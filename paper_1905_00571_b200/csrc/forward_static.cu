@@ -135,6 +135,7 @@ cadnn_status cadnn_forward_static(const cadnn_op *ops, int n_ops, int n, int h, 
         sn.n = si.n;
         if (op.kind == CADNN_OP_CONV || op.kind == CADNN_OP_FC) {
             if (!op.w || !op.w->on_device) return CADNN_E_ARG;
+            if (op.w->has_tc) return CADNN_E_UNSUPPORTED;   // block-structured layers need a workspace of their own
             const cadnn_layer_desc &d = op.w->desc;
             if (d.dtype != si.dtype) return CADNN_E_DTYPE;
             if (op.kind == CADNN_OP_FC) {

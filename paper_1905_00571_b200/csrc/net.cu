@@ -39,6 +39,9 @@ struct cadnn_net {
     // device staging for cadnn_forward_host
     void *stage_x = nullptr, *stage_y = nullptr;
     int64_t in_bytes = 0, out_bytes = 0;
+    // int32 sums of block-structured layers (tensor-core blocks), shared by all such ops of the net
+    void *tc_ws = nullptr;
+    int64_t tc_ws_bytes = 0;
     // L2 flush buffer for layer timing
     void *flush = nullptr;
     size_t flush_bytes = 0;
@@ -96,7 +99,7 @@ cadnn_status run_op(cadnn_net *net, const cadnn_op &op, const void *x, void *y, 
         ep.out_c_off = op.dst_c_off;
         ep.residual_scale = op.res_scale;
         if (op.kind == CADNN_OP_FC) return conv2d_impl(op.w, src, si.n, 1, 1, dst, &ep, pdl, st);
-        return conv2d_impl(op.w, src, si.n, si.h, si.w, dst, &ep, pdl, st);
+        return conv2d_impl(op.w, src, si.n, si.h, si.w, dst, &ep, pdl, st, net->tc_ws, net->tc_ws_bytes);
     }
     if (op.kind == CADNN_OP_MAXPOOL || op.kind == CADNN_OP_AVGPOOL)
         return launch_pool_window(src, si.n, si.h, si.w, si.c, op.pool_k, op.pool_stride, op.pool_pad, si.dtype,
@@ -413,6 +416,8 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
             // what the layer call would refuse (epilogue combination, weights of another GPU) is refused now
             st = check_layer_call(op.w, op.res >= 0, op.act, op.out_dtype, op.dst_c_total, op.dst_c_off);
             if (st != CADNN_OK) break;
+            if (op.w->has_tc)
+                net->tc_ws_bytes = std::max(net->tc_ws_bytes, (int64_t)si.n * op.w->h_out * op.w->w_out * d.c_out * 4);
         } else if (op.kind == CADNN_OP_MAXPOOL || op.kind == CADNN_OP_AVGPOOL) {
             if (op.pool_k < 1 || op.pool_stride < 1 || op.pool_pad < 0 || op.pool_pad >= op.pool_k ||
                 si.h + 2 * op.pool_pad < op.pool_k || si.w + 2 * op.pool_pad < op.pool_k) { st = CADNN_E_SHAPE; break; }
@@ -456,6 +461,15 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
         return st;
     }
     net->out_bytes = net->slots[net->out_slot].bytes;
+    if (net->tc_ws_bytes > 0) {
+        cudaError_t e = cudaMalloc(&net->tc_ws, (size_t)net->tc_ws_bytes);
+        if (e != cudaSuccess) {
+            cadnn_note_cuda(e);
+            cadnn_net_free(net);
+            return e == cudaErrorMemoryAllocation ? CADNN_E_ALLOC : CADNN_E_CUDA;
+        }
+        net->workspace += net->tc_ws_bytes;
+    }
     if (cudaHostAlloc((void **)&net->status_host, 2 * sizeof(int), cudaHostAllocDefault) != cudaSuccess) {
         cudaGetLastError();
         cadnn_net_free(net);
@@ -629,6 +643,7 @@ void cadnn_net_free(cadnn_net *net)
     for (SlotInfo &s : net->slots)
         if (s.ptr) cudaFree(s.ptr);
     if (net->flush) cudaFree(net->flush);
+    if (net->tc_ws) cudaFree(net->tc_ws);
     if (net->status_host) cudaFreeHost(net->status_host);
     persist_free(net->persist);
     delete net;

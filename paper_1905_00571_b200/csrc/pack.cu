@@ -1305,11 +1305,38 @@ cadnn_status pack_common(const cadnn_layer_desc *desc, const Src &src, cadnn_wei
             for (size_t i = 0; i < numel; ++i) kept += src.kept(i);
             dense_stem = kept * 2 >= numel;
         }
-        if (depthwise) st = pack_dense(h, src, KK_DW);
+        std::vector<uint8_t> rem_mask;
+        std::vector<int8_t> q_codes;
+        if (d.fmt == CADNN_FMT_GROUPED) {
+            // block-structured int8 layer: the dense blocks go to the tensor-core image, the sparse image keeps the rest
+            if (depthwise || d.dtype != CADNN_S8) st = CADNN_E_UNSUPPORTED;
+            else {
+                const size_t numel = (size_t)d.c_out * d.kh * d.kw * d.c_in;
+                const int8_t *qp = src.q;
+                if (!qp) {
+                    q_codes.resize(numel);
+                    const size_t per = numel / d.c_out;
+                    for (size_t i = 0; i < numel; ++i) q_codes[i] = src.qval(i, (int)(i / per));
+                    qp = q_codes.data();
+                }
+                double thr = 0.5;
+                if (const char *e = getenv("CADNN_BLOCK_DENSITY")) thr = std::min(1.0, std::max(0.0, atof(e)));
+                if (!block_tc_extract(h, qp, src.mask, thr, rem_mask)) st = CADNN_E_UNSUPPORTED;
+                else {
+                    Src rest = src;
+                    rest.mask = rem_mask.data();
+                    st = pack_sconv(h, rest);
+                    h->nnz += h->tc_nnz;
+                    h->fmt = CADNN_FMT_GROUPED;
+                }
+            }
+        }
+        else if (depthwise) st = pack_dense(h, src, KK_DW);
         else if (dense_stem) st = pack_dense(h, src, KK_DENSE_SMALLC);
         else if (is_fc && std::max(1, d.batch_hint) <= 8 && d.c_in <= 65536) st = pack_fc_spmv(h, src);
         else st = pack_sconv(h, src);
         if (st == CADNN_OK) st = upload(h);
+        if (st == CADNN_OK) st = block_tc_upload(h);
         if (st == CADNN_OK && h->has_planar && h->on_device && (d.flags & CADNN_PACK_AUTOTUNE) && !h->tuned)
             autotune_planar(h, h->row_nnz);
         if (st == CADNN_OK && h->tune_key && !h->tuned && h->on_device) {   // remember what was measured
@@ -1492,6 +1519,21 @@ cadnn_status cadnn_weights_unpack(const cadnn_weights *w, float *dense, uint8_t 
             }
         }
     }
+    if (w->has_tc) {   // the dense blocks of a block-structured layer
+        const int n_nt = d.c_out / 64;
+        for (int nt = 0; nt < n_nt; ++nt)
+            for (int bi = w->tc_tile_ptr[nt]; bi < w->tc_tile_ptr[nt + 1]; ++bi) {
+                const int kx = w->tc_blk[bi * 4] + d.pad_w, ky = w->tc_blk[bi * 4 + 1] + d.pad, c0 = w->tc_blk[bi * 4 + 2];
+                for (int r = 0; r < 64; ++r)
+                    for (int c = 0; c < 64; ++c) {
+                        if (!w->tc_kept[(size_t)bi * 4096 + r * 64 + c]) continue;
+                        const size_t wi = ((((size_t)(nt * 64 + r)) * d.kh + ky) * d.kw + kx) * d.c_in + c0 + c;
+                        const int chunk = (c >> 4) ^ ((r >> 1) & 3);
+                        if (dense) dense[wi] = (float)w->tc_wblk[(size_t)bi * 4096 + r * 64 + chunk * 16 + (c & 15)];
+                        if (mask) mask[wi] = 1;
+                    }
+            }
+    }
     return CADNN_OK;
 }
 
@@ -1499,6 +1541,7 @@ void cadnn_weights_free(cadnn_weights *w)
 {
     if (!w) return;
     if (w->d_blob) cudaFree(w->d_blob);
+    if (w->d_tc_blob) cudaFree(w->d_tc_blob);
     delete w;
 }
 

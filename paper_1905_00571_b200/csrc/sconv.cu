@@ -39,6 +39,7 @@ struct SconvParams {
     int n, h, w, c_in, h_out, w_out, c_out;
     int stride, pad, pad_w;
     float res_scale;  // int8 layers: multiplier of the int8 residual
+    const int *acc_in; // int8 layers: int32 sums [pixels][c_out] added to the accumulators (tensor-core blocks), or null
     int ldc, c_off;   // channels per output pixel of y and first channel written (a window of a wider tensor for concatenations)
     int BW, RB, TBX, TBY, TH, TW, pitch, half, IH_t, IW_t;
     int CIc, PPb, n_chunks, G, n_groups, stages, esz;
@@ -448,7 +449,15 @@ __global__ void __launch_bounds__(512) sconv_kernel(const SconvParams p)
         const int co = co_base + lc;
         const size_t ri = (size_t)opix * p.c_out + co;              // residual: a tensor of exactly c_out channels
         const size_t oi = (size_t)opix * p.ldc + p.c_off + co;      // output: possibly a channel window of a wider tensor
-        const AT *a = sOut + q * op + lc;
+        const AT *a0 = sOut + q * op + lc;
+        AT a[4];
+#pragma unroll
+        for (int v = 0; v < 4; ++v) a[v] = (quad || v == 0) ? a0[v] : (AT)0;
+        if (sizeof(XT) == 1 && p.acc_in) {   // sums of the layer's dense blocks, computed on the tensor cores
+#pragma unroll
+            for (int v = 0; v < 4; ++v)
+                if (quad || v == 0) a[v] = (AT)((int)a[v] + p.acc_in[ri + v]);
+        }
         if (quad) {
             float sc[4], bi[4];
 #pragma unroll
@@ -592,6 +601,7 @@ cadnn_status launch_sconv(const cadnn_weights *w, const void *x, int n, void *y,
     p.h_out = w->h_out; p.w_out = w->w_out; p.c_out = d.c_out;
     p.stride = d.stride; p.pad = d.pad; p.pad_w = d.pad_w;
     p.res_scale = ep.res_scale;
+    p.acc_in = ep.acc_in;
     p.ldc = ep.out_c_total > 0 ? ep.out_c_total : d.c_out; p.c_off = ep.out_c_total > 0 ? ep.out_c_off : 0;
     p.BW = s.BW; p.RB = s.RB; p.TBX = s.TBX; p.TBY = s.TBY; p.TH = s.TH; p.TW = s.TW;
     p.pitch = s.pitch; p.half = s.half; p.IH_t = s.IH_t; p.IW_t = s.IW_t;

@@ -12,7 +12,8 @@ def desc_for(op, dtype, batch_hint=1, autotune=False):
         return B.make_desc(op.c_in, op.c_out, 1, 1, 1, 0, 1, 1, 1, batch_hint, dtype, autotune=autotune)
     kh, kw = int(op.w.shape[1]), int(op.w.shape[2])   # rectangular kernels carry their own shape
     return B.make_desc(op.c_in, op.c_out, kh, kw, op.stride, op.pad, op.groups,
-                       op.in_hw[0], op.in_hw[1], batch_hint, dtype, autotune=autotune, pad_w=getattr(op, "pad_w", -1))
+                       op.in_hw[0], op.in_hw[1], batch_hint, dtype, autotune=autotune, pad_w=getattr(op, "pad_w", -1),
+                       fmt=B.FMT_GROUPED if getattr(op, "fmt", "auto") == "grouped" else 0)
 
 
 def pack_op(op, dtype, batch_hint=1, autotune=False):

@@ -131,3 +131,39 @@ def test_compute_without_device_image_is_refused(B):
     ep = None
     st = B._lib.cadnn_conv2d(wh.handle, ctypes.c_void_p(256), 1, 4, 4, ctypes.c_void_p(512), ep, None)
     assert st == 1
+
+
+def test_grouped_format_finds_the_dense_blocks_and_round_trips(B, monkeypatch):
+    """Block-structured int8 layer, host-only pack: the blocks the mask keeps (nearly) whole are found, the
+    remainder stays sparse, and unpacking gives back exactly the kept weights and the mask."""
+    g = gen.rng(21)
+    shape = (128, 3, 3, 192)
+    q = gen.int8_weights(g, shape)
+    mask = gen.block_mask(g, shape, 0.25, sprinkle=0.02)
+    # one block at 60 % (taken at the default threshold of 0.5) and one at 30 % (left to the sparse image)
+    mask[0:64, 0, 0, 0:64] = (g.random((64, 64)) < 0.6)
+    mask[64:128, 2, 2, 128:192] = (g.random((64, 64)) < 0.3)
+    blocks_whole = 0
+    for nt in range(2):
+        for ky in range(3):
+            for kx in range(3):
+                for ck in range(3):
+                    blocks_whole += int(mask[nt * 64:nt * 64 + 64, ky, kx, ck * 64:ck * 64 + 64].mean() >= 0.5)
+    d = B.make_desc(192, 128, 3, 3, 1, 1, 1, 20, 20, 1, "s8", host_only=True, fmt=B.FMT_GROUPED)
+    wh = B.cadnn_pack_q8(d, q, mask)
+    info = B.cadnn_weights_info(wh)
+    bi = B.cadnn_weights_block_info(wh)
+    assert info["fmt"] == B.FMT_GROUPED and info["nnz"] == int(mask.sum())
+    assert bi["blocks"] == blocks_whole and 0 < bi["block_nnz"] < info["nnz"]
+    dense, m2 = B.cadnn_weights_unpack(wh)
+    np.testing.assert_array_equal(m2, mask)
+    np.testing.assert_array_equal(dense, q.astype(np.float32) * mask)
+    assert B.cadnn_weights_workspace_bytes(wh, 2) == 2 * 20 * 20 * 128 * 4
+    # a threshold of 1.0 leaves the 60 % block to the sparse image as well
+    monkeypatch.setenv("CADNN_BLOCK_DENSITY", "1.0")
+    wh2 = B.cadnn_pack_q8(d, q, mask)
+    assert B.cadnn_weights_block_info(wh2)["blocks"] == blocks_whole - 1
+    # shapes the format does not cover are refused
+    with pytest.raises(B.CadnnError):
+        B.cadnn_pack_q8(B.make_desc(96, 128, 3, 3, 1, 1, 1, 20, 20, 1, "s8", host_only=True, fmt=B.FMT_GROUPED),
+                        gen.int8_weights(g, (128, 3, 3, 96)), None)

@@ -64,6 +64,25 @@ def skewed_mask(g, shape, density, skew=4.0):
     return m.reshape(shape)
 
 
+def block_mask(g, shape, block_density, sprinkle=0.0, bm=64, bk=64):
+    """Block-structured mask for OHWI weights [c_out, kh, kw, c_in]: the tensor is cut into blocks of bm output
+    channels x bk input channels at one tap; exactly keep_count(block_density, blocks) blocks are kept whole,
+    and of the positions outside them a fraction `sprinkle` is kept at random."""
+    c_out, kh, kw, c_in = shape
+    nb_o, nb_i = c_out // bm, c_in // bk
+    blocks = nb_o * kh * kw * nb_i
+    k = keep_count(block_density, blocks)
+    pick = np.zeros(blocks, np.uint8)
+    pick[g.choice(blocks, size=k, replace=False)] = 1
+    pick = pick.reshape(nb_o, kh, kw, nb_i)
+    m = np.repeat(np.repeat(pick, bm, axis=0), bk, axis=3)
+    full = np.zeros(shape, np.uint8)
+    full[:nb_o * bm, :, :, :nb_i * bk] = m
+    if sprinkle > 0.0:
+        full |= ((g.random(shape) < sprinkle) & (full == 0)).astype(np.uint8)
+    return full
+
+
 def normal_weights(g, shape, std):
     return (g.standard_normal(shape) * std).astype(np.float32)
 

@@ -44,6 +44,7 @@ class Op:
     res_scale: float = 0.0         # int8 residual: s_r / s_y
     dst_off: int = 0               # first channel of dst this op writes (channel concatenation)
     dst_total: int = 0             # channels of the dst slot; 0 = the op's own c_out
+    fmt: str = "auto"              # 'grouped': ask the packer for the block-structured int8 format
 
     @property
     def nnz(self):
@@ -358,6 +359,27 @@ def _s8_layer(m, g, kind, name, src, c_in, c_out, k, pad, h, act, density, m2_in
     m.ops.append(Op(kind, name, src, dst, res, c_in, c_out, k, stride, pad, 1, act, q, mask,
                     mult, offs, out, density, (h, h), (ho, ho), res_scale=res_scale))
     return dst
+
+
+def vgg16_block(seed=8, block_density=0.25, sprinkle=0.01, width=1.0, image=224, classes=1000, fc_width=4096):
+    """VGG-16, int8, with BLOCK-structured pruning of the convs from conv2 on: of the 64 output channels x 64
+    input channels x one tap blocks of a layer exactly round(block_density * blocks) are kept whole, and a
+    further `sprinkle` of the remaining positions is kept at random (so that the sparse kernel has a
+    remainder to add).  conv1 (3 input channels) and the FC layers are pruned as in vgg16()."""
+    g = gen.rng(seed)
+    base = vgg16(seed=seed, width=width, image=image, classes=classes, fc_width=fc_width)
+    base.name = "vgg16_block"
+    for op in base.ops:
+        if op.kind != "conv" or op.c_in % 64 or op.c_out % 64:
+            continue
+        op.mask = gen.block_mask(g, op.w.shape, block_density, sprinkle)
+        op.density = float(op.mask.mean())
+        op.fmt = "grouped"
+        qq = (op.w.astype(np.float64) ** 2) * op.mask
+        row_energy = qq.reshape(op.c_out, -1).sum(axis=1)
+        mult = np.where(row_energy > 0, _T_RMS / np.sqrt(np.maximum(row_energy, 1.0) * _M2_RELU), 1.0)
+        op.scale = (mult * g.uniform(0.8, 1.25, size=op.c_out)).astype(np.float32)
+    return base
 
 
 def vgg16(seed=3, density=0.08, fc_density=0.04, width=1.0, image=224, classes=1000, fc_width=4096):
