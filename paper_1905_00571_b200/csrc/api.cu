@@ -95,11 +95,15 @@ cadnn_status conv2d_impl(const cadnn_weights *w, const void *x, int n, int h, in
     cadnn_status st = check_epilogue(w, ep, le);
     if (st != CADNN_OK) return st;
     le.pdl = pdl;
+    if (w->has_tc && w->nnz == w->tc_nnz) {
+        // every stored weight sits in a dense block: the tensor-core kernel finishes the layer
+        return launch_block_tc(w, x, n, nullptr, y, &le, s);
+    }
     if (w->has_tc) {
         // dense blocks on the tensor cores first; the sparse kernel then starts from their int32 sums
         const int64_t need = (int64_t)n * w->h_out * w->w_out * w->desc.c_out * 4;
         if (!workspace || !aligned16(workspace) || workspace_bytes < need) return CADNN_E_ARG;
-        st = launch_block_tc(w, x, n, (int *)workspace, s);
+        st = launch_block_tc(w, x, n, (int *)workspace, nullptr, nullptr, s);
         if (st != CADNN_OK) return st;
         le.acc_in = (const int *)workspace;
         le.pdl = false;
@@ -125,7 +129,7 @@ cadnn_status cadnn_conv2d(const cadnn_weights *w, const void *x, int n, int h, i
 cadnn_status cadnn_weights_workspace_bytes(const cadnn_weights *w, int n, int64_t *bytes)
 {
     if (!w || !bytes || n < 0) return CADNN_E_ARG;
-    *bytes = w->has_tc ? (int64_t)n * w->h_out * w->w_out * w->desc.c_out * 4 : 0;
+    *bytes = (w->has_tc && w->nnz != w->tc_nnz) ? (int64_t)n * w->h_out * w->w_out * w->desc.c_out * 4 : 0;
     return CADNN_OK;
 }
 

@@ -47,7 +47,7 @@ const int kTcM = 128;          // output pixels per block: 16 columns x 8 rows
 const int kTcBW = 16, kTcBH = 8;
 const int kTcN = 64;           // output channels per block
 const int kTcK = 64;           // input channels per dense block (bytes of a K-major row)
-const int kTcStages = 4;
+const int kTcStages = 8;
 const int kTcABytes = kTcM * kTcK;   // 8192
 const int kTcBBytes = kTcN * kTcK;   // 4096
 const int kTcStageBytes = kTcABytes + kTcBBytes;
@@ -57,7 +57,14 @@ struct TcParams {
     const int8_t *wblk;
     const int4 *blk;          // {column shift, row shift, first input channel, 0}
     const int *tile_ptr;
-    int *acc;                 // [n][h_out][w_out][c_out] int32
+    int *acc;                 // [n][h_out][w_out][c_out] int32 sums for the sparse kernel, or null:
+    void *y;                  // then the layer's epilogue runs here and writes the output tensor
+    const float *scale, *bias;
+    const int8_t *residual;   // [n][h_out][w_out][c_out] or null
+    float res_scale;
+    int act, out_dtype;
+    int ldc, c_off;           // channels of the output tensor and first channel of this layer's window in it
+    int vec_ok;               // the window allows 16-byte stores
     int h_out, w_out, c_out;
     int tiles_x, tiles_y, n_ntiles;
 };
@@ -176,16 +183,31 @@ __global__ void __launch_bounds__(128) block_tc_kernel(const TcParams p, const _
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     const unsigned tmem = *slot;
 
-    if (tid == 0) {
-        // producer: the stages are a ring; a stage is refilled once the tensor core has read it
-        for (int i = 0; i < n_blk; ++i) {
-            const int s = i % kTcStages;
-            if (i >= kTcStages && !tc_wait(bars + (kTcStages + s) * 8, (unsigned)((i / kTcStages - 1) & 1))) break;
-            const int4 bl = p.blk[blk_lo + i];
-            const unsigned full = bars + s * 8;
-            tc_expect_tx(full, (unsigned)kTcStageBytes);
-            tc_tensor_copy_4d(base32 + s * kTcStageBytes, &xmap, bl.z, x0 + bl.x, y0 + bl.y, img, full);
-            tc_bulk_copy(base32 + s * kTcStageBytes + kTcABytes, p.wblk + (size_t)(blk_lo + i) * kTcBBytes, (unsigned)kTcBBytes, full);
+    if (warp == 0) {
+        // producer: the stages are a ring; a stage is refilled once the tensor core has read it.  The warp reads the
+        // block list 32 entries at a time (one ahead), lane 0 waits for the stage and starts its copies.
+        const int4 zero = make_int4(0, 0, 0, 0);
+        int4 mine = lane < n_blk ? p.blk[blk_lo + lane] : zero;
+        bool alive = true;
+        for (int base = 0; base < n_blk; base += 32) {
+            const int4 ahead = base + 32 + lane < n_blk ? p.blk[blk_lo + base + 32 + lane] : zero;
+            const int cnt = min(32, n_blk - base);
+            for (int j = 0; j < cnt; ++j) {
+                const int bx = __shfl_sync(0xffffffffu, mine.x, j), by = __shfl_sync(0xffffffffu, mine.y, j);
+                const int bz = __shfl_sync(0xffffffffu, mine.z, j);
+                const int i = base + j, s = i % kTcStages;
+                if (lane == 0 && alive && i >= kTcStages)
+                    alive = tc_wait(bars + (kTcStages + s) * 8, (unsigned)((i / kTcStages - 1) & 1));
+                alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
+                if (alive && lane == 0) {
+                    const unsigned full = bars + s * 8;
+                    tc_expect_tx(full, (unsigned)kTcStageBytes);
+                    tc_tensor_copy_4d(base32 + s * kTcStageBytes, &xmap, bz, x0 + bx, y0 + by, img, full);
+                    tc_bulk_copy(base32 + s * kTcStageBytes + kTcABytes, p.wblk + (size_t)(blk_lo + i) * kTcBBytes, (unsigned)kTcBBytes, full);
+                }
+                __syncwarp();
+            }
+            mine = ahead;
         }
     } else if (tid == 32) {
         // multiply-add issuer
@@ -214,10 +236,11 @@ __global__ void __launch_bounds__(128) block_tc_kernel(const TcParams p, const _
     const int m = warp * 32 + lane;
     const int oy = y0 + m / kTcBW, ox = x0 + m % kTcBW;
     const bool inside = oy < p.h_out && ox < p.w_out;
-    int *dst = p.acc + (((size_t)img * p.h_out + oy) * p.w_out + ox) * p.c_out + nt * kTcN;
+    const size_t pix = ((size_t)img * p.h_out + oy) * p.w_out + ox;
 #pragma unroll
     for (int half = 0; half < kTcN / 32; ++half) {
         int v[32];
+        __syncwarp();   // the tensor-memory load is warp-wide
         if (have) {
             tc_ld32(tmem + ((unsigned)(warp * 32) << 16) + half * 32, v);
             asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
@@ -225,10 +248,63 @@ __global__ void __launch_bounds__(128) block_tc_kernel(const TcParams p, const _
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = 0;
         }
-        if (inside) {
+        if (!inside) continue;
+        const int c0 = nt * kTcN + half * 32;
+        if (p.acc) {
+            int *dst = p.acc + pix * p.c_out + c0;
 #pragma unroll
-            for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<int4 *>(dst + half * 32 + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+            for (int j = 0; j < 32; j += 4) *reinterpret_cast<int4 *>(dst + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+            continue;
+        }
+        // no sparse remainder: requantize here (same arithmetic as the sparse kernel's epilogue)
+        const size_t oi = pix * p.ldc + p.c_off + c0;
+        if (p.out_dtype == CADNN_S32) {
+            int *dst = reinterpret_cast<int *>(p.y) + oi;
+            if (p.vec_ok) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) *reinterpret_cast<int4 *>(dst + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) dst[j] = v[j];
+            }
+            continue;
+        }
+        const bool has_res = p.residual != nullptr;
+        union { int4 q[2]; signed char b[32]; } res;
+        res.q[0] = res.q[1] = make_int4(0, 0, 0, 0);
+        if (has_res) {
+            const int4 *rp = reinterpret_cast<const int4 *>(p.residual + pix * p.c_out + c0);
+            asm volatile("ld.global.v4.s32 {%0, %1, %2, %3}, [%4];\n" : "=r"(res.q[0].x), "=r"(res.q[0].y), "=r"(res.q[0].z), "=r"(res.q[0].w) : "l"(rp));
+            asm volatile("ld.global.v4.s32 {%0, %1, %2, %3}, [%4];\n" : "=r"(res.q[1].x), "=r"(res.q[1].y), "=r"(res.q[1].z), "=r"(res.q[1].w) : "l"(rp + 1));
+        }
+        if (p.out_dtype == CADNN_F32) {
+            float o[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                o[j] = requant_f32(v[j], p.scale ? __ldg(p.scale + c0 + j) : 1.0f, p.bias ? __ldg(p.bias + c0 + j) : 0.0f, p.act,
+                                   has_res, (int)res.b[j], p.res_scale);
+            float *dst = reinterpret_cast<float *>(p.y) + oi;
+            if (p.vec_ok) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4 *>(dst + j) = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) dst[j] = o[j];
+            }
+        } else {
+            union { int4 q[2]; signed char b[32]; } out;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                out.b[j] = (signed char)requant_s8(v[j], p.scale ? __ldg(p.scale + c0 + j) : 1.0f, p.bias ? __ldg(p.bias + c0 + j) : 0.0f,
+                                                   p.act, has_res, (int)res.b[j], p.res_scale);
+            int8_t *dst = reinterpret_cast<int8_t *>(p.y) + oi;
+            if (p.vec_ok) {
+                *reinterpret_cast<int4 *>(dst) = out.q[0];
+                *reinterpret_cast<int4 *>(dst + 16) = out.q[1];
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) dst[j] = out.b[j];
+            }
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
@@ -321,15 +397,26 @@ cadnn_status block_tc_upload(cadnn_weights *h)
     return CADNN_OK;
 }
 
-cadnn_status launch_block_tc(const cadnn_weights *w, const void *x, int n, int *acc, cudaStream_t st)
+cadnn_status launch_block_tc(const cadnn_weights *w, const void *x, int n, int *acc, void *y, const LaunchEpilogue *le, cudaStream_t st)
 {
     const cadnn_layer_desc &d = w->desc;
-    if (!w->has_tc || !w->d_tc_tile_ptr || !acc) return CADNN_E_ARG;
-    TcParams p;
+    if (!w->has_tc || !w->d_tc_tile_ptr || (!acc && !(y && le))) return CADNN_E_ARG;
+    TcParams p = {};
     p.wblk = w->d_tc_wblk;
     p.blk = (const int4 *)w->d_tc_blk;
     p.tile_ptr = w->d_tc_tile_ptr;
     p.acc = acc;
+    if (!acc) {
+        p.y = y;
+        p.scale = le->scale; p.bias = le->bias;
+        p.residual = (const int8_t *)le->residual;
+        p.res_scale = le->res_scale;
+        p.act = le->act; p.out_dtype = le->out_dtype;
+        p.ldc = le->out_c_total > 0 ? le->out_c_total : d.c_out;
+        p.c_off = le->out_c_total > 0 ? le->out_c_off : 0;
+        const int esz = le->out_dtype == CADNN_S8 ? 1 : 4;
+        p.vec_ok = (p.ldc * esz) % 16 == 0 && (p.c_off * esz) % 16 == 0;
+    }
     p.h_out = w->h_out; p.w_out = w->w_out; p.c_out = d.c_out;
     p.tiles_x = (w->w_out + kTcBW - 1) / kTcBW;
     p.tiles_y = (w->h_out + kTcBH - 1) / kTcBH;

@@ -202,7 +202,9 @@ cadnn_status launch_dw_planar(const cadnn_weights *w, const void *x, int n, void
 // block-structured int8 layers (blocktc.cu)
 bool block_tc_extract(cadnn_weights *h, const int8_t *q, const uint8_t *mask, double threshold, std::vector<uint8_t> &rem_mask);
 cadnn_status block_tc_upload(cadnn_weights *h);
-cadnn_status launch_block_tc(const cadnn_weights *w, const void *x, int n, int *acc, cudaStream_t st);
+// acc != null: int32 sums for the sparse kernel; acc == null: the layer has no sparse remainder and the kernel
+// applies the epilogue *le and writes y itself
+cadnn_status launch_block_tc(const cadnn_weights *w, const void *x, int n, int *acc, void *y, const LaunchEpilogue *le, cudaStream_t st);
 cadnn_status read_tc_timeouts(int *count);
 cadnn_status read_copy_timeouts(int *count);
 cadnn_status read_barrier_timeouts(int *count);
@@ -310,6 +312,30 @@ __device__ __forceinline__ signed char ld_act(const signed char *p)
     int v;
     asm volatile("ld.global.s8 %0, [%1];\n" : "=r"(v) : "l"(p));
     return (signed char)v;
+}
+
+// ---- epilogue arithmetic shared by the conv kernels ----
+__device__ __forceinline__ float act_f32(float z, int act)
+{
+    if (act == CADNN_ACT_RELU) return z > 0.0f ? z : 0.0f;
+    if (act == CADNN_ACT_RELU6) return fminf(z > 0.0f ? z : 0.0f, 6.0f);
+    return z;
+}
+
+// int8 layer: one fused multiply-add on the converted accumulator, a second one for the int8 residual
+// of a quantized residual block (r * residual_scale joins before the activation), ReLU
+__device__ __forceinline__ float requant_f32(int acc, float m, float b, int act, bool has_res = false, int r = 0, float rs = 0.0f)
+{
+    float t = __fmaf_rn(__int2float_rn(acc), m, b);
+    if (has_res) t = __fmaf_rn(__int2float_rn(r), rs, t);
+    if (act == CADNN_ACT_RELU) t = t > 0.0f ? t : 0.0f;
+    return t;
+}
+__device__ __forceinline__ int requant_s8(int acc, float m, float b, int act, bool has_res = false, int r = 0, float rs = 0.0f)
+{
+    float t = requant_f32(acc, m, b, act, has_res, r, rs);
+    t = fminf(fmaxf(t, -127.0f), 127.0f);
+    return __float2int_rn(t);
 }
 
 template <typename... KArgs, typename... Args>

@@ -416,7 +416,7 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
             // what the layer call would refuse (epilogue combination, weights of another GPU) is refused now
             st = check_layer_call(op.w, op.res >= 0, op.act, op.out_dtype, op.dst_c_total, op.dst_c_off);
             if (st != CADNN_OK) break;
-            if (op.w->has_tc)
+            if (op.w->has_tc && op.w->nnz != op.w->tc_nnz)
                 net->tc_ws_bytes = std::max(net->tc_ws_bytes, (int64_t)si.n * op.w->h_out * op.w->w_out * d.c_out * 4);
         } else if (op.kind == CADNN_OP_MAXPOOL || op.kind == CADNN_OP_AVGPOOL) {
             if (op.pool_k < 1 || op.pool_stride < 1 || op.pool_pad < 0 || op.pool_pad >= op.pool_k ||

@@ -463,7 +463,11 @@ __global__ void __launch_bounds__(512) sconv_planar_tma_kernel(const PsParams p,
         for (int s = 0; s < S; ++s) mbar_init(smem32 + p.bar_off + s * 8, 1);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(&tmap) : "memory");
-        for (int s = 0; s < npre; ++s) ps_tma_issue(p, &tmap, smem32, s, c_first + s, grp, 0, 0, true, false, [] {});
+    }
+    if (warp == 0) {
+        // lane s starts the copies of stage s: issuing a copy takes a few hundred clocks, and the lanes' issues overlap
+        __syncwarp();
+        if (lane < npre) ps_tma_issue(p, &tmap, smem32, lane, c_first + lane, grp, 0, 0, true, false, [] {});
     }
     const int KS = 1 << p.ks_shift;
     const int rslot = warp >> p.ks_shift, slice = warp & (KS - 1);
@@ -494,9 +498,7 @@ __global__ void __launch_bounds__(512) sconv_planar_tma_kernel(const PsParams p,
         for (int t = 0; t < T; ++t) acc[j][t] = 0.0f;
 
     grid_dep_wait();   // x (and the residual) are final from here on
-    if (tid == 0) {
-        for (int s = 0; s < npre; ++s) ps_tma_issue(p, &tmap, smem32, s, c_first + s, grp, (int)img * p.c_in, xq, false, true, [] {});
-    }
+    if (warp == 0 && lane < npre) ps_tma_issue(p, &tmap, smem32, lane, c_first + lane, grp, (int)img * p.c_in, xq, false, true, [] {});
     float sc[RPW], bi[RPW];
 #pragma unroll
     for (int j = 0; j < RPW; ++j) {

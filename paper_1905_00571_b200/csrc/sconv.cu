@@ -68,29 +68,6 @@ __device__ __forceinline__ void cp_async16(unsigned dst, const void *src)
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
-__device__ __forceinline__ float act_f32(float z, int act)
-{
-    if (act == CADNN_ACT_RELU) return z > 0.0f ? z : 0.0f;
-    if (act == CADNN_ACT_RELU6) return fminf(z > 0.0f ? z : 0.0f, 6.0f);
-    return z;
-}
-
-// int8 layer: one fused multiply-add on the converted accumulator, a second one for the int8 residual
-// of a quantized residual block (r * residual_scale joins before the activation), ReLU
-__device__ __forceinline__ float requant_f32(int acc, float m, float b, int act, bool has_res = false, int r = 0, float rs = 0.0f)
-{
-    float t = __fmaf_rn(__int2float_rn(acc), m, b);
-    if (has_res) t = __fmaf_rn(__int2float_rn(r), rs, t);
-    if (act == CADNN_ACT_RELU) t = t > 0.0f ? t : 0.0f;
-    return t;
-}
-__device__ __forceinline__ int requant_s8(int acc, float m, float b, int act, bool has_res = false, int r = 0, float rs = 0.0f)
-{
-    float t = requant_f32(acc, m, b, act, has_res, r, rs);
-    t = fminf(fmaxf(t, -127.0f), 127.0f);
-    return __float2int_rn(t);
-}
-
 template <typename XT> struct Traits;
 template <> struct Traits<float> {
     typedef float acc_t;

@@ -85,8 +85,80 @@ def torch_dense_ms(model, batch, tf32, reps=20):
     return a.elapsed_time(b) / reps
 
 
+def block_crossover(batches):
+    """Block-structured int8 layer (a VGG conv3 shape, 256 -> 256, 3x3, 56x56): the tensor-core route for its
+    64 x 64 blocks against the sparse CUDA-core kernel on the same mask, by the density INSIDE the blocks (all blocks
+    present; the tensor-core time does not depend on it, the sparse kernel's does), and by the fraction of
+    blocks kept (blocks whole)."""
+    import os
+    from workloads import gen
+    dev = "cuda:0"
+    c, hw = 256, 56
+    g = gen.rng(99)
+    q = gen.int8_weights(g, (c, 3, 3, c))
+    m = torch.full((c,), 2e-5, device=dev)
+    b = torch.zeros(c, device=dev)
+
+    def time_it(fn, reps=20):
+        # the calls are captured into one CUDA graph, so that the host's launch cost stays out of the figure
+        fn()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for _ in range(reps):
+                fn()
+        graph.replay()
+        torch.cuda.synchronize()
+        best = 1e9
+        for _ in range(3):
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record()
+            graph.replay()
+            a1.record()
+            torch.cuda.synchronize()
+            best = min(best, a0.elapsed_time(a1) / reps * 1e3)
+        return best
+
+    def both(mask, batch, threshold):
+        x = torch.from_numpy(gen.int8_image(g, (batch, hw, hw, c))).to(dev)
+        y1 = torch.zeros((batch, hw, hw, c), dtype=torch.int8, device=dev)
+        y2 = torch.zeros_like(y1)
+        os.environ["CADNN_BLOCK_DENSITY"] = str(threshold)
+        wg = B.cadnn_pack_q8(B.make_desc(c, c, 3, 3, 1, 1, 1, hw, hw, batch, "s8", fmt=B.FMT_GROUPED), q, mask)
+        os.environ.pop("CADNN_BLOCK_DENSITY", None)
+        ws = torch.empty(B.cadnn_weights_workspace_bytes(wg, batch), dtype=torch.uint8, device=dev)
+        wsp = B.cadnn_pack_q8(B.make_desc(c, c, 3, 3, 1, 1, 1, hw, hw, batch, "s8"), q, mask)
+        t_g = time_it(lambda: B.cadnn_conv2d_workspace(wg, x, y1, ws, m, b, None, "relu", out_dtype="s8"))
+        t_s = time_it(lambda: B.cadnn_conv2d(wsp, x, y2, m, b, None, "relu", out_dtype="s8"))
+        torch.cuda.synchronize()
+        assert torch.equal(y1, y2), "the two routes disagree"
+        return t_g, t_s, B.cadnn_weights_block_info(wg)["blocks"]
+
+    print("# Block-structured int8 conv 256->256 3x3 56x56: tensor-core blocks + sparse remainder vs sparse kernel alone\n")
+    print("## by density inside the blocks (every block present, all of them taken as dense blocks)\n")
+    print("| batch | density in block | blocks | tensor-core route µs | sparse kernel µs | ratio sparse / tc |")
+    print("|---|---|---|---|---|---|")
+    for batch in batches:
+        for rho in (0.05, 0.1, 0.2, 0.3, 0.5, 0.75, 1.0):
+            mask = (g.random(q.shape) < rho).astype(np.uint8) if rho < 1.0 else np.ones(q.shape, np.uint8)
+            t_g, t_s, nb = both(mask, batch, 0.0)
+            print("| %d | %.2f | %d | %.1f | %.1f | %.2f |" % (batch, rho, nb, t_g, t_s, t_s / t_g))
+            sys.stdout.flush()
+    print("\n## by fraction of blocks kept (kept blocks whole, nothing else)\n")
+    print("| batch | blocks kept | blocks | tensor-core route µs | sparse kernel µs | ratio sparse / tc |")
+    print("|---|---|---|---|---|---|")
+    for batch in batches:
+        for bd in (0.05, 0.1, 0.25, 0.5, 1.0):
+            mask = gen.block_mask(g, q.shape, bd)
+            t_g, t_s, nb = both(mask, batch, 0.5)
+            print("| %d | %.2f | %d | %.1f | %.1f | %.2f |" % (batch, bd, nb, t_g, t_s, t_s / t_g))
+            sys.stdout.flush()
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--block-crossover", action="store_true",
+                    help="time the tensor-core block route against the sparse kernel on one block-structured int8 layer")
     ap.add_argument("--workload", default="resnet50")
     ap.add_argument("--batch", type=int, nargs="+", default=[1])
     ap.add_argument("--density", type=float, nargs="+", default=[0.125])
@@ -94,6 +166,9 @@ def main():
     ap.add_argument("--no-autotune", action="store_true")
     ap.add_argument("--torch-dense", action="store_true", help="add cuDNN dense timings (context)")
     args = ap.parse_args()
+    if args.block_crossover:
+        block_crossover(args.batch)
+        return
     peaks = roofline.measured_peaks()
     r_alu = roofline.alu_peak_tflops(peaks["sm_max_mhz"])
     print("# %s: sparse-roofline report (ALU peak %.1f TFLOP/s, HBM %.0f GB/s nominal / %.0f measured)\n"
