@@ -202,15 +202,16 @@ __device__ __forceinline__ void stem_cp16(unsigned dst, const float *src)
 }
 
 // The same register tile specialised at compile time for the stems that occur (7x7x3 and 3x3x3 at
-// stride 2): a block is 4 warps (16 channels each) on ONE pair of output rows, so a 112 x 112 map
+// stride 2): a block is 4 warps of 16 channels (or 8 of 8) on ONE pair of output rows, so a 112 x 112 map
 // gives 224 blocks (the generic kernel's 112 leave a quarter of the SMs idle); the staged input
 // is split by channel and by column parity, so that lanes on consecutive output columns read
 // consecutive words whatever the tap (at stride 2 the interleaved layout is a 2-way bank
 // conflict); weights and input rows are copied without any division; the taps of one kernel
 // row are fully unrolled with constant offsets.
-template <int KH, int KW, int CIN>
-__global__ void __launch_bounds__(128) stem2_kernel(const StemParams p)
+template <int KH, int KW, int CIN, int CPW>
+__global__ void __launch_bounds__(32 * (kStemCoBlock / CPW)) stem2_kernel(const StemParams p)
 {
+    constexpr int NW = kStemCoBlock / CPW, NT = 32 * NW;   // warps (CPW channels each) and threads per block
     constexpr int STRIDE = 2;
     constexpr int IN_ROWS = STRIDE + KH;            // two output rows
     constexpr int IN_COLS = 31 * STRIDE + KW;
@@ -233,12 +234,12 @@ __global__ void __launch_bounds__(128) stem2_kernel(const StemParams p)
     // Weights of this block's 64 channels first (static data: before the grid-dependency wait).
     const unsigned sW32 = (unsigned)__cvta_generic_to_shared(sW), sIn32 = (unsigned)__cvta_generic_to_shared(sIn);
     if ((p.c_out & 3) == 0 && co0 + kStemCoBlock <= p.c_out) {
-        for (int i = tid; i < TAPS * (kStemCoBlock / 4); i += 128) {
+        for (int i = tid; i < TAPS * (kStemCoBlock / 4); i += NT) {
             const int t = i >> 4, c4 = i & 15;
             stem_cp16(sW32 + i * 16, p.wt + (size_t)t * p.c_out + co0 + c4 * 4);
         }
     } else {
-        for (int i = tid; i < TAPS * kStemCoBlock; i += 128) {
+        for (int i = tid; i < TAPS * kStemCoBlock; i += NT) {
             const int t = i >> 6, c = i & 63;
             const bool ok = co0 + c < p.c_out;
             stem_cp4(sW32 + i * 4, ok ? p.wt + (size_t)t * p.c_out + co0 + c : p.wt, ok);
@@ -247,8 +248,8 @@ __global__ void __launch_bounds__(128) stem2_kernel(const StemParams p)
     grid_dep_wait();
     grid_dep_trigger();
     const int iy0 = oy0 * STRIDE - p.pad, ix0 = ox0 * STRIDE - p.pad_w;
-    // input rows: IN_COLS * CIN consecutive floats of the NHWC image each; warp r mod 4 takes row r
-    for (int r = wc; r < IN_ROWS; r += 4) {
+    // input rows: IN_COLS * CIN consecutive floats of the NHWC image each; warp r mod NW takes row r
+    for (int r = wc; r < IN_ROWS; r += NW) {
         const int iy = iy0 + r;
         const bool row_ok = iy >= 0 && iy < p.h;
         const float *src = p.x + (((size_t)img * p.h + (row_ok ? iy : 0)) * p.w) * CIN;
@@ -270,10 +271,10 @@ __global__ void __launch_bounds__(128) stem2_kernel(const StemParams p)
     asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
     __syncthreads();
 
-    float acc0[kStemCo], acc1[kStemCo];
+    float acc0[CPW], acc1[CPW];
 #pragma unroll
-    for (int c = 0; c < kStemCo; ++c) acc0[c] = acc1[c] = 0.0f;
-    const float *w_base = sW + wc * kStemCo;
+    for (int c = 0; c < CPW; ++c) acc0[c] = acc1[c] = 0.0f;
+    const float *w_base = sW + wc * CPW;
     const float *in0 = sIn + lane;
 #pragma unroll 1
     for (int ky = 0; ky < KH; ++ky) {
@@ -288,7 +289,7 @@ __global__ void __launch_bounds__(128) stem2_kernel(const StemParams p)
                 const float a0 = r0[off], a1 = r1[off];
                 const float4 *wq = reinterpret_cast<const float4 *>(wk + (kx * CIN + ci) * kStemCoBlock);
 #pragma unroll
-                for (int q = 0; q < kStemCo / 4; ++q) {
+                for (int q = 0; q < CPW / 4; ++q) {
                     const float4 wv = wq[q];
                     acc0[4 * q + 0] = fmaf(a0, wv.x, acc0[4 * q + 0]);
                     acc0[4 * q + 1] = fmaf(a0, wv.y, acc0[4 * q + 1]);
@@ -303,7 +304,7 @@ __global__ void __launch_bounds__(128) stem2_kernel(const StemParams p)
     }
 
     const int ox = ox0 + lane;
-    const int cbase = co0 + wc * kStemCo;
+    const int cbase = co0 + wc * CPW;
     if (ox < p.w_out) {
 #pragma unroll
         for (int rr = 0; rr < 2; ++rr) {
@@ -315,7 +316,7 @@ __global__ void __launch_bounds__(128) stem2_kernel(const StemParams p)
             const size_t plane = (size_t)planar_pitch(p.h_out, p.w_out);
             const size_t opl = (size_t)img * p.c_out * plane + (size_t)(oy + p.halo) * wp + ox + p.halo;
 #pragma unroll
-            for (int c = 0; c < kStemCo; ++c) {
+            for (int c = 0; c < CPW; ++c) {
                 const int co = cbase + c;
                 if (co >= p.c_out) break;
                 float z = fmaf(acc[c], p.scale ? __ldg(p.scale + co) : 1.0f, p.bias ? __ldg(p.bias + co) : 0.0f);
@@ -339,12 +340,21 @@ cadnn_status launch_stem2(StemParams &p, int n, bool pdl, cudaStream_t st)
     if (blocks <= 0) return CADNN_OK;
     if (blocks > 2147483647LL) return CADNN_E_UNSUPPORTED;
     const size_t smem = ((size_t)KH * KW * CIN * kStemCoBlock + (size_t)IN_ROWS * CIN * 2 * HALF) * 4;
-    static bool raised = false;
-    if (!raised && smem > 48 * 1024) {
-        CADNN_CUDA_TRY(cudaFuncSetAttribute(stem2_kernel<KH, KW, CIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        raised = true;
+    // few blocks (one image): 8 warps of 8 channels keep more warps per scheduler than 4 of 16; many blocks: the
+    // larger register tile issues fewer shared-memory loads per multiply-add
+    static SmemLimit lim8, lim16;
+    if (blocks <= 4 * 148) {   // up to four blocks per multiprocessor
+        if (smem > 48 * 1024) {
+            cadnn_status rs = raise_smem_limit((const void *)stem2_kernel<KH, KW, CIN, 8>, (int)smem, &lim8);
+            if (rs != CADNN_OK) return rs;
+        }
+        return launch_kernel(stem2_kernel<KH, KW, CIN, 8>, (int)blocks, 256, smem, pdl, st, p);
     }
-    return launch_kernel(stem2_kernel<KH, KW, CIN>, (int)blocks, 128, smem, pdl, st, p);
+    if (smem > 48 * 1024) {
+        cadnn_status rs = raise_smem_limit((const void *)stem2_kernel<KH, KW, CIN, 16>, (int)smem, &lim16);
+        if (rs != CADNN_OK) return rs;
+    }
+    return launch_kernel(stem2_kernel<KH, KW, CIN, 16>, (int)blocks, 128, smem, pdl, st, p);
 }
 
 }  // namespace
