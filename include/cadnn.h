@@ -371,6 +371,22 @@ cadnn_status cadnn_net_info(const cadnn_net *net, int *n_launches, int64_t *work
 cadnn_status cadnn_net_layout(const cadnn_net *net, int *planar, int *persistent_ops);
 
 /*
+ * Stride-2 layers in a channel-planar net (Section 4: a layer's data layout is chosen for the layer that reads
+ * it).  A float conv of stride 2 (3x3 with padding 1, or 1x1) is packed in a second form as well: a stride-1
+ * layer over its input split by row and column parity (four planes of ceil(h/2) x ceil(w/2) per channel, each
+ * with its zero border; the 1x1 layer reads the (even, even) plane alone).  cadnn_net_create uses that form
+ * where the layer writing the input is a sparse conv - whose epilogue then stores the parity planes beside the
+ * tensor itself - and where it measured faster at pack time (both forms timed under CADNN_PACK_AUTOTUNE;
+ * CADNN_FORCE_PARITY_PLANES=1 in the environment takes it wherever it exists, CADNN_NO_PARITY_PLANES=1 never).
+ * The results are those of the plain form up to summation order.  *count = number of ops run this way; their
+ * indices go to ops[0 .. min(*count, cap) - 1] (ops may be NULL with cap 0).  cadnn_weights_parity_form: the
+ * second form of a layer (*form = NULL if it has none), owned by w and valid as long as w; it answers
+ * cadnn_weights_planar_schedule and cadnn_weights_info like any handle and is not to be freed.
+ */
+cadnn_status cadnn_net_parity_layers(const cadnn_net *net, int *count, int *ops, int cap);
+cadnn_status cadnn_weights_parity_form(const cadnn_weights *w, const cadnn_weights **form);
+
+/*
  * Measurement aids for the persistent kernel (E_UNSUPPORTED when the net has none).
  * cadnn_net_persistent_plan: what the host planner chose for op `op` (Section 4, "Optimization
  * parameters selection"): plan[0..11] = bands of 32 positions per tile, bands per unit, filters per

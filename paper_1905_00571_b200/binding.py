@@ -75,6 +75,8 @@ _SIGS = {
     "cadnn_forward_static": (_i, [ctypes.POINTER(Op), _i, _i, _i, _i, _i, _i, _vp, _vp, _vp]),
     "cadnn_net_info": (_i, [_vp, ctypes.POINTER(_i), _i64p]),
     "cadnn_net_layout": (_i, [_vp, ctypes.POINTER(_i), ctypes.POINTER(_i)]),
+    "cadnn_net_parity_layers": (_i, [_vp, ctypes.POINTER(_i), ctypes.POINTER(_i), _i]),
+    "cadnn_weights_parity_form": (_i, [_vp, ctypes.POINTER(_vp)]),
     "cadnn_net_layer_times": (_i, [_vp, _vp, _vp, _i, _i, ctypes.POINTER(ctypes.c_float), _vp]),
     "cadnn_net_layer_time": (_i, [_vp, _i, _vp, _vp, _i, _i, ctypes.POINTER(ctypes.c_float), _vp]),
     "cadnn_debug_set_device_status": (_i, [_i, _i]),
@@ -366,6 +368,31 @@ def cadnn_net_info(net):
     nl, ws = ctypes.c_int(), ctypes.c_int64()
     _check(_lib.cadnn_net_info(net.handle, ctypes.byref(nl), ctypes.byref(ws)), "cadnn_net_info")
     return {"launches": nl.value, "workspace_bytes": ws.value}
+
+
+def cadnn_net_parity_layers(net, ops=False):
+    """Number of stride-2 layers run in their parity-plane form (ops=True: their op indices)."""
+    c = ctypes.c_int()
+    _check(_lib.cadnn_net_parity_layers(net.handle, ctypes.byref(c), None, 0), "cadnn_net_parity_layers")
+    if not ops:
+        return c.value
+    buf = (ctypes.c_int * max(1, c.value))()
+    _check(_lib.cadnn_net_parity_layers(net.handle, ctypes.byref(c), buf, c.value), "cadnn_net_parity_layers")
+    return list(buf[: c.value])
+
+
+class _Borrowed:
+    """A handle owned by another object (never freed here)."""
+
+    def __init__(self, handle, desc):
+        self.handle = handle
+        self.desc = desc
+
+
+def cadnn_weights_parity_form(w):
+    out = ctypes.c_void_p()
+    _check(_lib.cadnn_weights_parity_form(w.handle, ctypes.byref(out)), "cadnn_weights_parity_form")
+    return _Borrowed(out, w.desc) if out.value else None
 
 
 def cadnn_net_layout(net):

@@ -133,6 +133,9 @@ struct cadnn_weights {
     std::vector<int32_t> tc_tile_ptr;   // [c_out / 64 + 1] blocks of every tile of 64 output channels
     std::vector<uint8_t> tc_kept;       // [n_blocks][64][64] which positions of a block the mask kept (host only, for unpack)
     int64_t tc_nnz = 0;                 // kept positions inside the dense blocks
+    // float stride-2 layers (3x3 pad 1, 1x1): the same layer packed as a stride-1 layer over the parity planes of its
+    // input (owned; null = none)
+    cadnn_weights *half = nullptr;
     void *d_tc_blob = nullptr;
     const int8_t *d_tc_wblk = nullptr;
     const int32_t *d_tc_blk = nullptr;
@@ -160,7 +163,33 @@ struct LaunchEpilogue {
     float res_scale = 0.0f;   // int8 layers: multiplier of the int8 residual
     const int *acc_in = nullptr;   // int8 sparse conv: int32 sums [pixels][c_out] added to the accumulators before the epilogue
     int out_c_total = 0, out_c_off = 0;   // NHWC sparse conv: channel window of a wider output tensor (concatenation)
+    // planar sparse convs: a second copy of the output split by row and column parity, for a stride-2 reader
+    // (parity_planes_bytes below gives its size); parity_mask = planes wanted, bit (row parity * 2 + column parity)
+    float *parity_y = nullptr;
+    int parity_mask = 0;
 };
+
+// Parity planes of an h x w map of c channels: plane (py * 2 + px) holds the pixels (2 i + py, 2 j + px) at (i, j) of a
+// padded plane of ceil(h / 2) x ceil(w / 2) (absent pixels of odd sizes stay zero).  Layout [image][plane][channel][pitch];
+// with mask 1 only the (even, even) plane exists.  A stride-2 3x3 (pad 1) layer over the map is a stride-1 layer over
+// the 4 c quarter planes, a stride-2 1x1 layer a stride-1 layer over plane 0.
+struct ParityPlanes {
+    float *y;        // null = none
+    int mask, planes, wp, pitch, c;
+};
+static inline ParityPlanes parity_planes(float *y, int mask, int h, int w, int c)
+{
+    ParityPlanes pp;
+    pp.y = y; pp.mask = mask; pp.planes = mask == 1 ? 1 : 4;
+    pp.wp = (w + 1) / 2 + 2 * kPlanarHalo;
+    pp.pitch = planar_pitch((h + 1) / 2, (w + 1) / 2);
+    pp.c = c;
+    return pp;
+}
+static inline int64_t parity_planes_bytes(int mask, int n, int h, int w, int c)
+{
+    return (int64_t)n * (mask == 1 ? 1 : 4) * c * planar_pitch((h + 1) / 2, (w + 1) / 2) * 4;
+}
 
 // status helpers
 cadnn_status cadnn_note_cuda(cudaError_t e);
@@ -312,6 +341,15 @@ __device__ __forceinline__ signed char ld_act(const signed char *p)
     int v;
     asm volatile("ld.global.s8 %0, [%1];\n" : "=r"(v) : "l"(p));
     return (signed char)v;
+}
+
+// value v of output pixel (row, col) (interior coordinates), channel co, image img -> its parity plane
+__device__ __forceinline__ void parity_store(const ParityPlanes &pp, unsigned img, int co, int row, int col, float v)
+{
+    const int par = (row & 1) * 2 + (col & 1);
+    if (!((pp.mask >> par) & 1)) return;
+    const int pl = pp.planes == 4 ? par : 0;
+    pp.y[(((size_t)img * pp.planes + pl) * pp.c + co) * pp.pitch + ((row >> 1) + kPlanarHalo) * pp.wp + (col >> 1) + kPlanarHalo] = v;
 }
 
 // ---- epilogue arithmetic shared by the conv kernels ----

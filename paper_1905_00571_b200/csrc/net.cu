@@ -14,6 +14,10 @@ struct SlotInfo {
     bool defined = false;
     void *ptr = nullptr;  // owned unless slot 0 or the output slot
     int64_t bytes = 0;
+    // planar nets: second copy of the tensor split by row and column parity, written by the producing sparse conv for
+    // stride-2 readers (owned); par_mask = planes present, bit (row parity * 2 + column parity)
+    void *par_ptr = nullptr;
+    int par_mask = 0;
 };
 
 struct cadnn_net {
@@ -29,6 +33,7 @@ struct cadnn_net {
     PersistPlan *persist = nullptr;
     int persist_first = -1, persist_last = -1;
     int64_t workspace = 0;
+    std::vector<char> use_half;   // per op: a stride-2 conv that runs as its stride-1 form over its input's parity planes
     // graph cache: [0] caller's device pointers, [1] the net's own staging buffers
     struct GraphCache {
         cudaGraph_t graph = nullptr;
@@ -75,6 +80,17 @@ cadnn_status run_op(cadnn_net *net, const cadnn_op &op, const void *x, void *y, 
             le.out_dtype = CADNN_F32;
             le.pdl = pdl;
             le.early_trigger = net->early_trigger;
+            const SlotInfo &so = net->slots[op.dst];
+            if (so.par_ptr) {
+                le.parity_y = (float *)so.par_ptr;
+                le.parity_mask = so.par_mask;
+            }
+            const size_t op_index = (size_t)(&op - net->ops.data());
+            if (op_index < net->use_half.size() && net->use_half[op_index]) {
+                const cadnn_weights *hw = op.w->half;
+                if (hw->has_ps && hw->use_ps) return launch_sconv_planar_staged(hw, si.par_ptr, si.n, dst, le, st);
+                return launch_sconv_planar(hw, si.par_ptr, si.n, dst, le, st);
+            }
             if (op.w->s.kind == KK_DENSE_SMALLC) {   // the stem reads the NHWC image and writes planes
                 le.planar_out = true;
                 return launch_dense_smallc(op.w, src, si.n, dst, le, st);
@@ -318,6 +334,58 @@ __global__ void flush_kernel(float *buf, size_t n)
 
 }  // namespace
 
+namespace {
+
+// Stride-2 layers of a planar net whose handle carries the stride-1 form over parity planes (cadnn_weights::half) use
+// it when the layer that writes their input is a sparse conv (its epilogue then stores the parity planes as well) and
+// the form measured faster at pack time (CADNN_FORCE_PARITY_PLANES=1: whenever it exists).  A 1x1 reader takes the
+// (even, even) plane, which is a tensor of its own only when no 3x3 reader asks for all four.
+cadnn_status plan_parity_planes(cadnn_net *net)
+{
+    const int n_ops = (int)net->ops.size();
+    net->use_half.assign(n_ops, 0);
+    const char *pe = getenv("CADNN_PERSIST");
+    if (!net->planar || getenv("CADNN_NO_PARITY_PLANES") || (pe && atoi(pe) != 0)) return CADNN_OK;
+    const bool force = getenv("CADNN_FORCE_PARITY_PLANES") != nullptr;
+    std::vector<int> writer(net->slots.size(), -1);
+    for (int i = 0; i < n_ops; ++i) writer[net->ops[i].dst] = i;
+    auto time_of = [](const cadnn_weights *w) { return (w->has_ps && w->use_ps) ? w->ps_us : w->pl_us; };
+    auto eligible = [&](int i, bool k3) {
+        const cadnn_op &op = net->ops[i];
+        if (op.kind != CADNN_OP_CONV || !op.w || !op.w->half || op.w->desc.stride != 2 || (op.w->desc.kh == 3) != k3) return false;
+        if (op.src == 0 || op.src == net->out_slot || writer[op.src] < 0) return false;
+        const cadnn_op &pr = net->ops[writer[op.src]];
+        if (pr.kind != CADNN_OP_CONV || !pr.w || !pr.w->has_planar || pr.w->s.kind == KK_DENSE_SMALLC || pr.w->s.kind == KK_DW) return false;
+        const float t_half = time_of(op.w->half), t_full = time_of(op.w);
+        return force || (t_half > 0.0f && t_full > 0.0f && t_half < t_full);
+    };
+    for (int i = 0; i < n_ops; ++i)
+        if (eligible(i, true)) {
+            net->use_half[i] = 1;
+            net->slots[net->ops[i].src].par_mask = 0xf;
+        }
+    for (int i = 0; i < n_ops; ++i)
+        if (eligible(i, false) && net->slots[net->ops[i].src].par_mask != 0xf) {
+            net->use_half[i] = 1;
+            net->slots[net->ops[i].src].par_mask = 0x1;
+        }
+    for (SlotInfo &sl : net->slots) {
+        if (!sl.par_mask) continue;
+        const size_t bytes = (size_t)parity_planes_bytes(sl.par_mask, sl.n, sl.h, sl.w, sl.c);
+        const size_t alloc = (bytes + 255) / 256 * 256;
+        cudaError_t e = cudaMalloc(&sl.par_ptr, alloc);
+        if (e == cudaSuccess) e = cudaMemset(sl.par_ptr, 0, alloc);   // borders and absent pixels read as zero
+        if (e != cudaSuccess) {
+            cadnn_note_cuda(e);
+            return e == cudaErrorMemoryAllocation ? CADNN_E_ALLOC : CADNN_E_CUDA;
+        }
+        net->workspace += (int64_t)alloc;
+    }
+    return CADNN_OK;
+}
+
+}  // namespace
+
 extern "C" {
 
 cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int wd, int c, int in_dtype,
@@ -461,6 +529,11 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
         return st;
     }
     net->out_bytes = net->slots[net->out_slot].bytes;
+    st = plan_parity_planes(net);
+    if (st != CADNN_OK) {
+        cadnn_net_free(net);
+        return st;
+    }
     if (net->tc_ws_bytes > 0) {
         cudaError_t e = cudaMalloc(&net->tc_ws, (size_t)net->tc_ws_bytes);
         if (e != cudaSuccess) {
@@ -530,6 +603,18 @@ cadnn_status cadnn_net_info(const cadnn_net *net, int *n_launches, int64_t *work
     if (!net) return CADNN_E_ARG;
     if (n_launches) *n_launches = (int)net->ops.size() - (net->persist ? net->persist_last - net->persist_first : 0);
     if (workspace_bytes) *workspace_bytes = net->workspace;
+    return CADNN_OK;
+}
+
+cadnn_status cadnn_net_parity_layers(const cadnn_net *net, int *count, int *ops, int cap)
+{
+    if (!net || !count || cap < 0 || (cap > 0 && !ops)) return CADNN_E_ARG;
+    *count = 0;
+    for (size_t i = 0; i < net->use_half.size(); ++i)
+        if (net->use_half[i]) {
+            if (*count < cap) ops[*count] = (int)i;
+            ++*count;
+        }
     return CADNN_OK;
 }
 
@@ -640,8 +725,10 @@ void cadnn_net_free(cadnn_net *net)
     drop_graph(net->cache[1]);
     if (net->stage_x) cudaFree(net->stage_x);
     if (net->stage_y) cudaFree(net->stage_y);
-    for (SlotInfo &s : net->slots)
+    for (SlotInfo &s : net->slots) {
         if (s.ptr) cudaFree(s.ptr);
+        if (s.par_ptr) cudaFree(s.par_ptr);
+    }
     if (net->flush) cudaFree(net->flush);
     if (net->tc_ws) cudaFree(net->tc_ws);
     if (net->status_host) cudaFreeHost(net->status_host);

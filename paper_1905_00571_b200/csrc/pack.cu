@@ -1395,6 +1395,46 @@ cadnn_status pack_common(const cadnn_layer_desc *desc, const Src &src, cadnn_wei
             rec.pl_us = h->pl_us; rec.ps_us = h->ps_us; rec.nhwc_us = h->nhwc_us;
             tune_store(h->tune_key, rec);
         }
+        // A float stride-2 layer (3x3 with padding 1, or 1x1) also gets the form a network uses when the layer before it
+        // writes its map split by row and column parity: input pixel (2 oy + ky - 1, 2 ox + kx - 1) is pixel
+        // (oy + dy, ox + dx) of parity plane ((ky - 1) & 1, (kx - 1) & 1) with dy = -1 for ky = 0 and 0 otherwise, so the
+        // layer is a stride-1 layer over the 4 c_in quarter planes (taps 0 and 1 of a padded 3x3 frame); a 1x1 layer
+        // reads the (even, even) plane alone.
+        const bool k3 = d.kh == 3 && d.kw == 3 && d.pad == 1 && d.pad_w == 1, k1 = d.kh == 1 && d.kw == 1 && d.pad == 0 && d.pad_w == 0;
+        if (st == CADNN_OK && d.dtype == CADNN_F32 && d.stride == 2 && d.groups == 1 && (k3 || k1) && h->has_planar && h->on_device &&
+            src.f && getenv("CADNN_NO_PARITY_PLANES") == nullptr) {
+            cadnn_layer_desc dc = d;
+            dc.stride = 1;
+            dc.in_h = (d.in_h + 1) / 2;
+            dc.in_w = (d.in_w + 1) / 2;
+            dc.c_in = k3 ? 4 * d.c_in : d.c_in;
+            const size_t per = (size_t)d.kh * d.kw * dc.c_in, numel = per * d.c_out;
+            std::vector<float> wc(numel, 0.0f);
+            std::vector<uint8_t> mc(numel, 0);
+            for (int co = 0; co < d.c_out; ++co)
+                for (int ky = 0; ky < d.kh; ++ky)
+                    for (int kx = 0; kx < d.kw; ++kx)
+                        for (int ci = 0; ci < d.c_in; ++ci) {
+                            const size_t wi = (((size_t)co * d.kh + ky) * d.kw + kx) * d.c_in + ci;
+                            if (!src.kept(wi)) continue;
+                            size_t wo = wi;
+                            if (k3) {
+                                const int par = (ky == 1 ? 0 : 2) + (kx == 1 ? 0 : 1);
+                                const int ty = ky == 0 ? 0 : 1, tx = kx == 0 ? 0 : 1;
+                                wo = (((size_t)co * 3 + ty) * 3 + tx) * dc.c_in + (size_t)par * d.c_in + ci;
+                            }
+                            wc[wo] = src.f[wi];
+                            mc[wo] = 1;
+                        }
+            Src sc;
+            sc.f = wc.data();
+            sc.mask = mc.data();
+            cadnn_weights *child = nullptr;
+            if (pack_common(&dc, sc, &child) == CADNN_OK) {
+                if (child->has_planar && child->h_out == h->h_out && child->w_out == h->w_out) h->half = child;
+                else cadnn_weights_free(child);
+            }
+        }
     } catch (const std::bad_alloc &) {
         st = CADNN_E_ALLOC;
     }
@@ -1467,6 +1507,13 @@ cadnn_status cadnn_weights_planar_schedule(const cadnn_weights *w, int sched[16]
         memcpy(v, t, sizeof(v));
     }
     memcpy(sched, v, sizeof(v));
+    return CADNN_OK;
+}
+
+cadnn_status cadnn_weights_parity_form(const cadnn_weights *w, const cadnn_weights **form)
+{
+    if (!w || !form) return CADNN_E_ARG;
+    *form = w->half;
     return CADNN_OK;
 }
 
@@ -1586,6 +1633,7 @@ cadnn_status cadnn_weights_unpack(const cadnn_weights *w, float *dense, uint8_t 
 void cadnn_weights_free(cadnn_weights *w)
 {
     if (!w) return;
+    if (w->half) cadnn_weights_free(w->half);
     if (w->d_blob) cudaFree(w->d_blob);
     if (w->d_tc_blob) cudaFree(w->d_tc_blob);
     delete w;

@@ -36,6 +36,7 @@ struct PlanarParams {
     int G, RPW, n_groups, tiles, act;
     int ksw_shift;   // log2 of the warps that share one filter (each walks a slice of its nonzeros)
     FastDiv d_wp_out, d_groups, d_tiles;
+    ParityPlanes par;   // second copy of the output for a stride-2 reader (par.y null = none)
 };
 
 __device__ __forceinline__ float pl_act(float z, int act)
@@ -155,8 +156,13 @@ __global__ void __launch_bounds__(512) sconv_planar_kernel(const PlanarParams p)
 #pragma unroll
             for (int t = 0; t < T; ++t) {
                 if (okmask & (1u << t)) {
-                    const float z = fmaf(acc[t], sc, bi) + res[t];
-                    p.y[obase + 32 * t] = pl_act(z, p.act);
+                    const float z = pl_act(fmaf(acc[t], sc, bi) + res[t], p.act);
+                    p.y[obase + 32 * t] = z;
+                    if (p.par.y) {
+                        const int q = q0 + 32 * t + lane;   // interior rows, padded columns
+                        const int oy = (int)fdiv((unsigned)q, p.d_wp_out);
+                        parity_store(p.par, img, co, oy, q - oy * p.wp_out - p.halo, z);
+                    }
                 }
             }
         }
@@ -304,6 +310,7 @@ cadnn_status launch_sconv_planar(const cadnn_weights *w, const void *x, int n, v
     p.n_groups = (d.c_out + p.G - 1) / p.G;
     p.tiles = (p.qtot + 32 * T - 1) / (32 * T);
     p.act = ep.act;
+    p.par = parity_planes(ep.parity_y, ep.parity_mask, w->h_out, w->w_out, d.c_out);
     p.d_wp_out = make_fastdiv(p.wp_out);
     p.d_groups = make_fastdiv(p.n_groups);
     p.d_tiles = make_fastdiv(p.tiles);

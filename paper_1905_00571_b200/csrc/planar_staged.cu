@@ -79,6 +79,7 @@ struct PsParams {
     int early_trigger;     // as a programmatic primary: let the next layer's prologue start at once
     int RB, nb, bar_off;   // TMA staging: rows per box, boxes per chunk, byte offset of the stage barriers
     FastDiv d_groups, d_tiles, d_wp, d_wp_out, d_l4;
+    ParityPlanes par;      // second copy of the output for a stride-2 reader (par.y null = none)
 };
 
 __device__ __forceinline__ void cp16(unsigned dst, const void *src, bool pred)
@@ -270,7 +271,13 @@ __device__ __forceinline__ void ps_block_tail(const PsParams &p, unsigned char *
                     float z = fmaf(acc[j][t], sc[j], bi[j]);
                     if (res) z += res[j][t];               // fetched before the multiply-add loop
                     else if (p.residual) z += p.residual[oi];
-                    p.y[oi] = ps_act(z, p.act);
+                    z = ps_act(z, p.act);
+                    p.y[oi] = z;
+                    if (p.par.y) {
+                        const int q = q0 + lane + 32 * t;
+                        const int row = (int)fdiv((unsigned)q, p.d_wp_out);
+                        parity_store(p.par, img, co, row - kPlanarHalo, q - row * p.wp_out - kPlanarHalo, z);
+                    }
                 }
             }
         }
@@ -664,6 +671,7 @@ cadnn_status launch_sconv_planar_staged(const cadnn_weights *w, const void *x, i
     p.ks_shift = s.KS >= 8 ? 3 : s.KS >= 4 ? 2 : s.KS >= 2 ? 1 : 0;
     p.tile_bytes = s.tile_bytes; p.stage_bytes = s.stage_bytes; p.hdr_bytes = s.hdr_bytes; p.block_bytes = s.block_bytes;
     p.act = ep.act;
+    p.par = parity_planes(ep.parity_y, ep.parity_mask, w->h_out, w->w_out, d.c_out);
     p.early_trigger = ep.early_trigger ? 1 : 0;
     p.d_groups = make_fastdiv(s.n_groups);
     p.d_tiles = make_fastdiv(s.tiles);

@@ -202,15 +202,21 @@ def main():
                 lines = ["\n## per layer: batch %d, density %.3g\n" % (batch, dens),
                          "| layer | kernel | in | c_in→c_out | k/s | nnz | µs | roofline µs | fraction | schedule |", "|---|---|---|---|---|---|---|---|---|---|"]
                 planar = B.cadnn_net_layout(pm.net)["planar"]
+                parity_ops = set(B.cadnn_net_parity_layers(pm.net, ops=True))
                 for i, (op, r, t) in enumerate(zip(model.ops, rows, per)):
                     s = B.cadnn_weights_schedule(pm.weights[i]) if i in pm.weights else None
                     ss = ("T%d rpw%d nw%d cic%d ks%d" % (s["T"], s["RPW"], s["NW"], s["CIc"], s["ksplit"])) if s and s["kind"] in (1, 2) else ""
-                    ps = B.cadnn_weights_planar_schedule(pm.weights[i]) if (planar and i in pm.weights and op.kind == "conv") else None
+                    wh = pm.weights.get(i) if op.kind == "conv" else None
+                    if wh is not None and i in parity_ops:   # the stride-1 form over the input's parity planes runs
+                        wh = B.cadnn_weights_parity_form(wh)
+                    ps = B.cadnn_weights_planar_schedule(wh) if (planar and wh is not None) else None
                     if ps and ps["variant"] == 1:
                         ss = "planar direct T%d nw%d ksw%d rpw%d d%d" % (ps["T"], ps["NW"], ps["KS"], ps["RPW"], ps["stages"])
                     elif ps and ps["variant"] == 2:
                         ss = "planar %s T%d nw%d ks%d rpw%d cic%d st%d kc%d" % ("tma" if ps["tma"] else "cp.async", ps["T"], ps["NW"], ps["KS"],
                                                                                ps["RPW"], ps["CIc"], ps["stages"], ps["KC"])
+                    if i in parity_ops:
+                        ss = "parity planes, " + ss
                     lines.append("| %s | %s | %dx%d | %d→%d | %d/%d | %d | %.1f | %.2f | %.3f | %s |" % (
                         op.name, r["family"], op.in_hw[0], op.in_hw[1], op.c_in, op.c_out, op.k, op.stride, r["nnz"],
                         t * 1e3, r["t_roof_us"], r["t_roof_us"] / (t * 1e3), ss))
