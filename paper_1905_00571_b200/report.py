@@ -34,6 +34,8 @@ def build(workload, density):
         return models.mobilenet_v1(density=density)
     if workload == "inception_v3":
         return models.inception_v3(density=density, fc_density=0.10 if density < 1.0 else 1.0)
+    if workload == "vgg16_block":   # block-structured pruning: `density` is the fraction of 64 x 64 blocks kept
+        return models.vgg16_block(block_density=density)
     raise SystemExit("unknown workload " + workload)
 
 
@@ -155,10 +157,45 @@ def block_crossover(batches):
             sys.stdout.flush()
 
 
+def persistent_profile(workload, batch):
+    """Per-phase clock profile of the persistent whole-network kernel (CADNN_PERSIST=1): wall clocks of the
+    phase, busiest and mean block, clocks until the first copy was issued and until its bytes had landed,
+    and what the host planner chose for every layer of the phase."""
+    import os
+    os.environ["CADNN_PERSIST"] = "1"
+    os.environ["CADNN_PERSIST_PROFILE"] = "1"
+    dev = "cuda:0"
+    m = build(workload, 0.125)
+    x = models.make_input(m, batch)
+    pm = PackedModel(m, batch, dev)
+    xd = torch.from_numpy(x).to(dev)
+    y = pm.new_output()
+    for _ in range(10):
+        pm.forward(xd, y)
+    torch.cuda.synchronize()
+    prof = B.cadnn_net_persistent_profile(pm.net)
+    names = {}
+    for i, op in enumerate(m.ops):
+        pl = B.cadnn_net_persistent_plan(pm.net, i)
+        if pl is not None:
+            names.setdefault(pl["phase"], []).append((op.name, pl))
+    print("# persistent kernel, %s batch %d: clocks per phase (last of 10 forwards)\n" % (workload, batch))
+    print("| phase | wall | busiest block | mean block | first copy issued | first bytes landed | layers (tile bands T, filters per item G, tiles, groups, passes) |")
+    print("|---|---|---|---|---|---|---|")
+    tot = 0.0
+    for ph, (w, bm, ba, ti, tl) in enumerate(prof):
+        tot += w
+        desc = "; ".join("%s T%d G%d t%d g%d p%d" % (n, p["T"], p["G"], p["tiles"], p["groups"], p["passes"]) for n, p in names.get(ph, []))
+        print("| %d | %.0f | %.0f | %.0f | %.0f | %.0f | %s |" % (ph, w, bm, ba, ti, tl, desc))
+    print("\ntotal %.0f clocks" % tot)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--block-crossover", action="store_true",
                     help="time the tensor-core block route against the sparse kernel on one block-structured int8 layer")
+    ap.add_argument("--persistent-profile", action="store_true",
+                    help="per-phase clock profile of the persistent kernel on the workload (first --batch value)")
     ap.add_argument("--workload", default="resnet50")
     ap.add_argument("--batch", type=int, nargs="+", default=[1])
     ap.add_argument("--density", type=float, nargs="+", default=[0.125])
@@ -166,6 +203,9 @@ def main():
     ap.add_argument("--no-autotune", action="store_true")
     ap.add_argument("--torch-dense", action="store_true", help="add cuDNN dense timings (context)")
     args = ap.parse_args()
+    if args.persistent_profile:
+        persistent_profile(args.workload, args.batch[0])
+        return
     if args.block_crossover:
         block_crossover(args.batch)
         return
