@@ -481,7 +481,9 @@ cadnn_status autotune_sconv(cadnn_weights *h, const Src &src, const Geometry &g,
         seen.push_back(key);
         pick.push_back(c);
     }
-    const size_t kMaxTimed = 80;
+    // large batches: a launch takes milliseconds, so only the model's best dozen classes are timed, with fewer launches
+    const size_t kMaxTimed = batch >= 32 ? 12 : 80;
+    const int reps = batch >= 32 ? 3 : 8;
     if (pick.size() > kMaxTimed) pick.resize(kMaxTimed);
     const size_t esz = src.s8 ? 1 : 4;
     const size_t xb = (size_t)batch * d.in_h * d.in_w * d.c_in * esz;
@@ -507,7 +509,7 @@ cadnn_status autotune_sconv(cadnn_weights *h, const Src &src, const Geometry &g,
         tmp.s = c.s;
         if (build_sconv_image(&tmp, src, g, row_nnz) != CADNN_OK) continue;
         if (upload(&tmp) != CADNN_OK) { if (tmp.d_blob) cudaFree(tmp.d_blob); continue; }
-        float us = time_schedule(&tmp, batch, x, y, st, 8);
+        float us = time_schedule(&tmp, batch, x, y, st, reps);
         if (us > 0.0f && (best_us < 0.0f || us < best_us)) {
             best_us = us;
             best = c.s;
@@ -672,6 +674,8 @@ void autotune_planar(cadnn_weights *h, const std::vector<int64_t> &row_nnz)
                   for (int dep : {1, 2, 4}) {
                     if (ksw > nw || nw > (T <= 4 ? 16 : 8)) continue;
                     if (dep > 1 && (T == 1 || dep > T)) continue;   // the kernel has no deeper variant there
+                    // large batches fill the device with whole filters per warp and wide bands: the rest is not timed
+                    if (batch >= 32 && (ksw > 1 || T < 4 || nw < 8 || dep > 2)) continue;
                     h->pl_T = T; h->pl_NW = nw; h->pl_KSW = ksw; h->pl_RPW = rpw; h->pl_D = dep;
                     planar_order(h, row_nnz);
                     if (h->pl_order.size() > order_cap) continue;
@@ -681,7 +685,8 @@ void autotune_planar(cadnn_weights *h, const std::vector<int64_t> &row_nnz)
                     cudaGraphExec_t ge = nullptr;
                     if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { cudaGetLastError(); continue; }
                     bool ok = true;
-                    for (int r = 0; r < 8 && ok; ++r) ok = launch_sconv_planar(h, x, batch, y, ep, st) == CADNN_OK;
+                    const int reps = batch >= 32 ? 3 : 8;
+                    for (int r = 0; r < reps && ok; ++r) ok = launch_sconv_planar(h, x, batch, y, ep, st) == CADNN_OK;
                     if (cudaStreamEndCapture(st, &g) != cudaSuccess) ok = false;
                     if (ok && cudaGraphInstantiate(&ge, g, 0) == cudaSuccess) {
                         cudaEvent_t e0, e1;
@@ -694,7 +699,7 @@ void autotune_planar(cadnn_weights *h, const std::vector<int64_t> &row_nnz)
                         if (cudaStreamSynchronize(st) == cudaSuccess) {
                             float ms = 0.0f;
                             cudaEventElapsedTime(&ms, e0, e1);
-                            float us = ms * 1e3f / 8.0f;
+                            float us = ms * 1e3f / (float)reps;
                             if (best_us < 0.0f || us < best_us) { best_us = us; bT = T; bNW = nw; bRPW = rpw; bKSW = ksw; bD = dep; }
                         }
                         cudaEventDestroy(e0);
