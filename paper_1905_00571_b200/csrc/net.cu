@@ -560,7 +560,7 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
     {
         // The persistent kernel trades the launch ramp and drain of every layer boundary for a device-wide
         // barrier and a copy start-up per layer.  Measured on a B200 (pruned ResNet-50, batch 1) a phase costs
-        // about 2300 clocks of barrier, 2200 clocks until the first bytes of its tile are in shared memory,
+        // about 2400 clocks of barrier and skew, 3400 clocks until its first tile is complete in shared memory,
         // and multiply-adds bound by shared-memory bandwidth: no less than one tuned kernel per layer under
         // programmatic launches.  So it stays opt-in.
         const char *pe = getenv("CADNN_PERSIST");   // "1": on; unset / "0": off
