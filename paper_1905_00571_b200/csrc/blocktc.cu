@@ -10,13 +10,16 @@
 // int32 sums to its own before the requantization.  Integer sums are exact in any order, so the
 // layer's result does not depend on which route a weight took.
 //
-// One thread block computes 128 output pixels (a 16 x 8 patch of one image) x 64 output channels:
-//   * thread 0 is the producer: per dense block one 4-D TMA tensor copy of the 16 x 8 x 64-channel
-//     input patch shifted by the block's tap (pixels outside the image read as zero: the padding)
-//     and one bulk copy of the block's 64 x 64 weights, both in the 64-byte-swizzled K-major layout,
-//     into a ring of stages, each on its own "full" mbarrier;
+// One thread block computes 128 output pixels (a 16 x 8 patch of one image) x 64 output channels.
+// The dense blocks of a tile of output channels are grouped by (chunk of 64 input channels, kernel
+// column kx): the taps (ky, kx) of a group read the same input columns, shifted by whole rows, so
+//   * one lane of warp 0 is the producer: per group ONE 4-D TMA tensor copy of the 16 x (8 + kh - 1)
+//     x 64-channel input patch at the column shift of kx (pixels outside the image read as zero: the
+//     padding) and one bulk copy per present block of its 64 x 64 weights, all in the
+//     64-byte-swizzled K-major layout, into a ring of stages, each on its own "full" mbarrier;
 //   * thread 32 issues the multiply-adds: per block two tcgen05.mma of M 128 x N 64 x K 32
-//     (s8 x s8 -> s32) whose accumulator lives in 64 columns of tensor memory, then a
+//     (s8 x s8 -> s32) on the patch rows ky .. ky + 7 (a shift of ky KB in the stage: the swizzle
+//     pattern repeats every 512 bytes), accumulator in 64 columns of tensor memory, then a
 //     tcgen05.commit that frees the stage ("empty" mbarrier) once the tensor core has read it;
 //   * after the last commit the four warps read their 32 accumulator rows with tcgen05.ld and store
 //     them as int32 [pixel][channel].
@@ -47,16 +50,18 @@ const int kTcM = 128;          // output pixels per block: 16 columns x 8 rows
 const int kTcBW = 16, kTcBH = 8;
 const int kTcN = 64;           // output channels per block
 const int kTcK = 64;           // input channels per dense block (bytes of a K-major row)
-const int kTcStages = 8;
-const int kTcABytes = kTcM * kTcK;   // 8192
-const int kTcBBytes = kTcN * kTcK;   // 4096
-const int kTcStageBytes = kTcABytes + kTcBBytes;
+const int kTcMaxStages = 8;
+const int kTcRowBytes = kTcBW * kTcK;   // one patch row of 16 pixels: 1024 bytes
+const int kTcBBytes = kTcN * kTcK;      // 4096
+const int kTcSmemBudget = 200 * 1024;
 const unsigned kTcSpin = 1u << 22;
 
 struct TcParams {
     const int8_t *wblk;
-    const int4 *blk;          // {column shift, row shift, first input channel, 0}
-    const int *tile_ptr;
+    const int4 *grp;          // {column shift, first input channel, mask of the kernel rows present, first block}
+    const int *grp_ptr;       // groups of every tile of 64 output channels
+    int kh, pad;              // kernel rows, padding above
+    int a_bytes, stage_bytes, stages;   // patch bytes, stage bytes (patch + kh blocks), ring depth
     int *acc;                 // [n][h_out][w_out][c_out] int32 sums for the sparse kernel, or null:
     void *y;                  // then the layer's epilogue runs here and writes the output tensor
     const float *scale, *bias;
@@ -153,11 +158,13 @@ __global__ void __launch_bounds__(128) block_tc_kernel(const TcParams p, const _
 {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     // stages at a 1024-byte boundary (the swizzle pattern repeats every 512 bytes)
+    const int S = p.stages;
     const unsigned base32 = ((unsigned)__cvta_generic_to_shared(smem_raw) + 1023u) & ~1023u;
-    const unsigned bars = base32 + kTcStages * kTcStageBytes;   // full[S], empty[S], done, then the TMEM address word
-    const unsigned slot32 = bars + (2 * kTcStages + 1) * 8;
+    const unsigned bars = base32 + S * p.stage_bytes;   // full[S], empty[S], done, then the TMEM address word, row masks
+    const unsigned slot32 = bars + (2 * S + 1) * 8;
     unsigned char *smem_gen = smem_raw + (base32 - (unsigned)__cvta_generic_to_shared(smem_raw));
-    volatile unsigned *slot = reinterpret_cast<volatile unsigned *>(smem_gen + kTcStages * kTcStageBytes + (2 * kTcStages + 1) * 8);
+    volatile unsigned *slot = reinterpret_cast<volatile unsigned *>(smem_gen + S * p.stage_bytes + (2 * S + 1) * 8);
+    volatile int *smask = reinterpret_cast<volatile int *>(smem_gen + S * p.stage_bytes + (2 * S + 1) * 8 + 16);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     // block -> (image, patch row, patch column, output-channel tile); channel tiles vary fastest
@@ -167,10 +174,10 @@ __global__ void __launch_bounds__(128) block_tc_kernel(const TcParams p, const _
     const int ty = b % p.tiles_y;
     const int img = b / p.tiles_y;
     const int x0 = tx * kTcBW, y0 = ty * kTcBH;
-    const int blk_lo = p.tile_ptr[nt], n_blk = p.tile_ptr[nt + 1] - blk_lo;
+    const int g_lo = p.grp_ptr[nt], n_grp = p.grp_ptr[nt + 1] - g_lo;
 
     if (tid == 0) {
-        for (int i = 0; i < 2 * kTcStages + 1; ++i) tc_mbar_init(bars + i * 8, 1);
+        for (int i = 0; i < 2 * S + 1; ++i) tc_mbar_init(bars + i * 8, 1);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(&xmap) : "memory");
     }
@@ -185,26 +192,32 @@ __global__ void __launch_bounds__(128) block_tc_kernel(const TcParams p, const _
 
     if (warp == 0) {
         // producer: the stages are a ring; a stage is refilled once the tensor core has read it.  The warp reads the
-        // block list 32 entries at a time (one ahead), lane 0 waits for the stage and starts its copies.
+        // group list 32 entries at a time (one ahead), lane 0 waits for the stage and starts its copies.
         const int4 zero = make_int4(0, 0, 0, 0);
-        int4 mine = lane < n_blk ? p.blk[blk_lo + lane] : zero;
+        int4 mine = lane < n_grp ? p.grp[g_lo + lane] : zero;
         bool alive = true;
-        for (int base = 0; base < n_blk; base += 32) {
-            const int4 ahead = base + 32 + lane < n_blk ? p.blk[blk_lo + base + 32 + lane] : zero;
-            const int cnt = min(32, n_blk - base);
+        int s = 0;
+        unsigned round = 0;   // times the ring has wrapped
+        for (int base = 0; base < n_grp; base += 32) {
+            const int4 ahead = base + 32 + lane < n_grp ? p.grp[g_lo + base + 32 + lane] : zero;
+            const int cnt = min(32, n_grp - base);
             for (int j = 0; j < cnt; ++j) {
-                const int bx = __shfl_sync(0xffffffffu, mine.x, j), by = __shfl_sync(0xffffffffu, mine.y, j);
-                const int bz = __shfl_sync(0xffffffffu, mine.z, j);
-                const int i = base + j, s = i % kTcStages;
-                if (lane == 0 && alive && i >= kTcStages)
-                    alive = tc_wait(bars + (kTcStages + s) * 8, (unsigned)((i / kTcStages - 1) & 1));
-                alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
-                if (alive && lane == 0) {
-                    const unsigned full = bars + s * 8;
-                    tc_expect_tx(full, (unsigned)kTcStageBytes);
-                    tc_tensor_copy_4d(base32 + s * kTcStageBytes, &xmap, bz, x0 + bx, y0 + by, img, full);
-                    tc_bulk_copy(base32 + s * kTcStageBytes + kTcABytes, p.wblk + (size_t)(blk_lo + i) * kTcBBytes, (unsigned)kTcBBytes, full);
+                const int xs = __shfl_sync(0xffffffffu, mine.x, j), ci0 = __shfl_sync(0xffffffffu, mine.y, j);
+                const int rows = __shfl_sync(0xffffffffu, mine.z, j), b0 = __shfl_sync(0xffffffffu, mine.w, j);
+                if (lane == 0 && alive) {
+                    if (round > 0 && !tc_wait(bars + (S + s) * 8, (round - 1) & 1u)) {
+                        alive = false;
+                    } else {
+                        const unsigned full = bars + s * 8, st32 = base32 + s * p.stage_bytes;
+                        const int nb = __popc(rows);
+                        smask[s] = rows;   // read by the issuing thread after its wait on the full barrier
+                        tc_expect_tx(full, (unsigned)(p.a_bytes + nb * kTcBBytes));
+                        tc_tensor_copy_4d(st32, &xmap, ci0, x0 + xs, y0 - p.pad, img, full);
+                        for (int k = 0; k < nb; ++k)
+                            tc_bulk_copy(st32 + p.a_bytes + k * kTcBBytes, p.wblk + (size_t)(b0 + k) * kTcBBytes, (unsigned)kTcBBytes, full);
+                    }
                 }
+                if (++s == S) { s = 0; ++round; }
                 __syncwarp();
             }
             mine = ahead;
@@ -212,25 +225,35 @@ __global__ void __launch_bounds__(128) block_tc_kernel(const TcParams p, const _
     } else if (tid == 32) {
         // multiply-add issuer
         const unsigned idesc = tc_instr_desc();
-        bool ok = true;
-        for (int i = 0; i < n_blk && ok; ++i) {
-            const int s = i % kTcStages;
-            ok = tc_wait(bars + s * 8, (unsigned)((i / kTcStages) & 1));
-            if (!ok) break;
+        int s = 0;
+        unsigned round = 0, first = 1;
+        for (int i = 0; i < n_grp; ++i) {
+            if (!tc_wait(bars + s * 8, round & 1u)) break;
             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-            const unsigned a0 = base32 + s * kTcStageBytes, b0 = a0 + kTcABytes;
+            const unsigned st32 = base32 + s * p.stage_bytes;
+            int rows = smask[s];
+            unsigned b0 = st32 + p.a_bytes;
+            while (rows) {
+                const int ky = __ffs(rows) - 1;
+                rows &= rows - 1;
+                const unsigned a0 = st32 + ky * kTcRowBytes;   // patch rows ky .. ky + 7
 #pragma unroll
-            for (int k = 0; k < kTcK / 32; ++k)
-                tc_mma_i8(tmem, tc_smem_desc(a0 + k * 32), tc_smem_desc(b0 + k * 32), idesc, (i > 0 || k > 0) ? 1u : 0u);
-            tc_commit(bars + (kTcStages + s) * 8);   // the stage is free when these multiply-adds have read it
+                for (int k = 0; k < kTcK / 32; ++k) {
+                    tc_mma_i8(tmem, tc_smem_desc(a0 + k * 32), tc_smem_desc(b0 + k * 32), idesc, first ? 0u : 1u);
+                    first = 0;
+                }
+                b0 += kTcBBytes;
+            }
+            tc_commit(bars + (S + s) * 8);   // the stage is free when these multiply-adds have read it
+            if (++s == S) { s = 0; ++round; }
         }
-        tc_commit(bars + 2 * kTcStages * 8);         // everything issued so far has completed
+        tc_commit(bars + 2 * S * 8);         // everything issued so far has completed
     }
 
     // ---- epilogue: warp w owns accumulator rows 32 w .. 32 w + 31 (thread = row = pixel) ----
     __syncwarp();
-    bool have = n_blk > 0;
-    if (have) have = tc_wait(bars + 2 * kTcStages * 8, 0u);
+    bool have = n_grp > 0;
+    if (have) have = tc_wait(bars + 2 * S * 8, 0u);
     have = __all_sync(0xffffffffu, have) != 0;   // the tensor-memory loads below are warp-wide
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     const int m = warp * 32 + lane;
@@ -327,17 +350,25 @@ bool block_tc_extract(cadnn_weights *h, const int8_t *q, const uint8_t *mask, do
     const size_t numel = (size_t)d.c_out * d.kh * d.kw * d.c_in;
     rem_mask.assign(numel, 1);
     if (mask) memcpy(rem_mask.data(), mask, numel);
+    if (d.kh > 16 || kTcRowBytes * (kTcBH + d.kh - 1) + d.kh * kTcBBytes > kTcSmemBudget / 2) return false;   // two stages must fit
     const int n_nt = d.c_out / kTcN, n_ck = d.c_in / kTcK;
     h->tc_tile_ptr.assign(n_nt + 1, 0);
+    h->tc_grp_ptr.assign(n_nt + 1, 0);
     h->tc_blk.clear();
+    h->tc_grp.clear();
     h->tc_wblk.clear();
     h->tc_kept.clear();
     h->tc_nnz = 0;
+    // blocks in the order (channel tile, input chunk, kernel column, kernel row): the blocks of one kernel column
+    // form a group that shares its staged input patch
     for (int nt = 0; nt < n_nt; ++nt) {
         h->tc_tile_ptr[nt] = (int32_t)(h->tc_blk.size() / 4);
-        for (int ky = 0; ky < d.kh; ++ky)
-            for (int kx = 0; kx < d.kw; ++kx)
-                for (int ck = 0; ck < n_ck; ++ck) {
+        h->tc_grp_ptr[nt] = (int32_t)(h->tc_grp.size() / 4);
+        for (int ck = 0; ck < n_ck; ++ck)
+            for (int kx = 0; kx < d.kw; ++kx) {
+                int rows = 0;
+                const int first_block = (int)(h->tc_blk.size() / 4);
+                for (int ky = 0; ky < d.kh; ++ky) {
                     int kept = 0;
                     for (int r = 0; r < kTcN; ++r) {
                         const size_t wi = ((((size_t)(nt * kTcN + r)) * d.kh + ky) * d.kw + kx) * d.c_in + (size_t)ck * kTcK;
@@ -366,9 +397,18 @@ bool block_tc_extract(cadnn_weights *h, const int8_t *q, const uint8_t *mask, do
                     h->tc_blk.push_back(ky - d.pad);
                     h->tc_blk.push_back(ck * kTcK);
                     h->tc_blk.push_back(0);
+                    rows |= 1 << ky;
                 }
+                if (rows) {
+                    h->tc_grp.push_back(kx - d.pad_w);
+                    h->tc_grp.push_back(ck * kTcK);
+                    h->tc_grp.push_back(rows);
+                    h->tc_grp.push_back(first_block);
+                }
+            }
     }
     h->tc_tile_ptr[n_nt] = (int32_t)(h->tc_blk.size() / 4);
+    h->tc_grp_ptr[n_nt] = (int32_t)(h->tc_grp.size() / 4);
     h->has_tc = true;
     return true;
 }
@@ -377,7 +417,7 @@ cadnn_status block_tc_upload(cadnn_weights *h)
 {
     if (!h->has_tc) return CADNN_OK;
     auto al = [](size_t v) { return (v + 255) / 256 * 256; };
-    const size_t b_w = h->tc_wblk.size(), b_b = h->tc_blk.size() * 4, b_t = h->tc_tile_ptr.size() * 4;
+    const size_t b_w = h->tc_wblk.size(), b_b = h->tc_grp.size() * 4, b_t = h->tc_grp_ptr.size() * 4;
     h->packed_bytes += (int64_t)(b_w + b_b + b_t);
     if (h->desc.flags & CADNN_PACK_HOST_ONLY) return CADNN_OK;
     const size_t total = al(b_w) + al(b_b) + al(b_t) + 256;
@@ -388,23 +428,28 @@ cadnn_status block_tc_upload(cadnn_weights *h)
     }
     char *base = (char *)h->d_tc_blob;
     if (b_w) CADNN_CUDA_TRY(cudaMemcpy(base, h->tc_wblk.data(), b_w, cudaMemcpyHostToDevice));
-    if (b_b) CADNN_CUDA_TRY(cudaMemcpy(base + al(b_w), h->tc_blk.data(), b_b, cudaMemcpyHostToDevice));
-    CADNN_CUDA_TRY(cudaMemcpy(base + al(b_w) + al(b_b), h->tc_tile_ptr.data(), b_t, cudaMemcpyHostToDevice));
+    if (b_b) CADNN_CUDA_TRY(cudaMemcpy(base + al(b_w), h->tc_grp.data(), b_b, cudaMemcpyHostToDevice));
+    CADNN_CUDA_TRY(cudaMemcpy(base + al(b_w) + al(b_b), h->tc_grp_ptr.data(), b_t, cudaMemcpyHostToDevice));
     CADNN_CUDA_TRY(cudaStreamSynchronize(cudaStreamLegacy));
     h->d_tc_wblk = (const int8_t *)base;
-    h->d_tc_blk = (const int32_t *)(base + al(b_w));
-    h->d_tc_tile_ptr = (const int32_t *)(base + al(b_w) + al(b_b));
+    h->d_tc_grp = (const int32_t *)(base + al(b_w));
+    h->d_tc_grp_ptr = (const int32_t *)(base + al(b_w) + al(b_b));
     return CADNN_OK;
 }
 
 cadnn_status launch_block_tc(const cadnn_weights *w, const void *x, int n, int *acc, void *y, const LaunchEpilogue *le, cudaStream_t st)
 {
     const cadnn_layer_desc &d = w->desc;
-    if (!w->has_tc || !w->d_tc_tile_ptr || (!acc && !(y && le))) return CADNN_E_ARG;
+    if (!w->has_tc || !w->d_tc_grp_ptr || (!acc && !(y && le))) return CADNN_E_ARG;
     TcParams p = {};
     p.wblk = w->d_tc_wblk;
-    p.blk = (const int4 *)w->d_tc_blk;
-    p.tile_ptr = w->d_tc_tile_ptr;
+    p.grp = (const int4 *)w->d_tc_grp;
+    p.grp_ptr = w->d_tc_grp_ptr;
+    p.kh = d.kh; p.pad = d.pad;
+    p.a_bytes = kTcRowBytes * (kTcBH + d.kh - 1);
+    p.stage_bytes = p.a_bytes + d.kh * kTcBBytes;
+    p.stages = std::min(kTcMaxStages, kTcSmemBudget / p.stage_bytes);
+    if (p.stages < 2) return CADNN_E_UNSUPPORTED;
     p.acc = acc;
     if (!acc) {
         p.y = y;
@@ -424,9 +469,11 @@ cadnn_status launch_block_tc(const cadnn_weights *w, const void *x, int n, int *
     const long long blocks = (long long)n * p.tiles_y * p.tiles_x * p.n_ntiles;
     if (blocks <= 0) return CADNN_OK;
     if (blocks > 2147483647LL) return CADNN_E_UNSUPPORTED;
+    // more blocks than multiprocessors: two blocks per multiprocessor with half the ring each
+    if (blocks > 148) p.stages = std::max(2, std::min(p.stages, kTcSmemBudget / 2 / p.stage_bytes));
     alignas(64) CUtensorMap map;
-    if (!encode_nhwc_s8_tiles_map(&map, x, d.c_in, d.in_w, d.in_h, n, kTcK, kTcBW, kTcBH)) return CADNN_E_UNSUPPORTED;
-    const int smem = kTcStages * kTcStageBytes + (2 * kTcStages + 1) * 8 + 16 + 1024;
+    if (!encode_nhwc_s8_tiles_map(&map, x, d.c_in, d.in_w, d.in_h, n, kTcK, kTcBW, kTcBH + d.kh - 1)) return CADNN_E_UNSUPPORTED;
+    const int smem = p.stages * p.stage_bytes + (2 * p.stages + 1) * 8 + 16 + p.stages * 4 + 1024;
     static SmemLimit lim;
     cadnn_status rs = raise_smem_limit((const void *)block_tc_kernel, smem, &lim);
     if (rs != CADNN_OK) return rs;

@@ -131,6 +131,9 @@ struct cadnn_weights {
     std::vector<int8_t> tc_wblk;        // [n_blocks][64 rows][64 bytes], rows = output channels, 16-byte chunks swizzled
     std::vector<int32_t> tc_blk;        // [n_blocks][4]: column shift, row shift of the tap, first input channel, 0
     std::vector<int32_t> tc_tile_ptr;   // [c_out / 64 + 1] blocks of every tile of 64 output channels
+    std::vector<int32_t> tc_grp;        // [n_groups][4]: blocks of one (input chunk, kernel column): column shift, first input
+                                        // channel, mask of the kernel rows present, first block
+    std::vector<int32_t> tc_grp_ptr;    // [c_out / 64 + 1] groups of every tile of 64 output channels
     std::vector<uint8_t> tc_kept;       // [n_blocks][64][64] which positions of a block the mask kept (host only, for unpack)
     int64_t tc_nnz = 0;                 // kept positions inside the dense blocks
     // float stride-2 layers (3x3 pad 1, 1x1): the same layer packed as a stride-1 layer over the parity planes of its
@@ -138,8 +141,8 @@ struct cadnn_weights {
     cadnn_weights *half = nullptr;
     void *d_tc_blob = nullptr;
     const int8_t *d_tc_wblk = nullptr;
-    const int32_t *d_tc_blk = nullptr;
-    const int32_t *d_tc_tile_ptr = nullptr;
+    const int32_t *d_tc_grp = nullptr;
+    const int32_t *d_tc_grp_ptr = nullptr;
 
     // device image (one allocation)
     void *d_blob = nullptr;

@@ -42,18 +42,37 @@ __global__ void __launch_bounds__(256) fc_spmv_kernel(const FcParams p)
     const int co = p.perm[row];
     if (co < 0) return;
     const int beg = p.ptr[row], end = p.ptr[row + 1];
-    const XT *vals = reinterpret_cast<const XT *>(p.vals);
     const XT *x = reinterpret_cast<const XT *>(p.x);
+    // rows are padded to whole quads of entries: a lane fetches four values and their four column indices per step
+    const int qbeg = beg >> 2, qend = end >> 2;
     for (int b0 = 0; b0 < p.n; b0 += NB) {
         AT acc[NB];
 #pragma unroll
         for (int b = 0; b < NB; ++b) acc[b] = 0;
-        for (int e = beg + lane; e < end; e += 32) {
-            const AT wv = (AT)vals[e];
-            const int k = p.idx[e];
+        for (int q = qbeg + lane; q < qend; q += 32) {
+            AT wv[4];
+            if (sizeof(XT) == 1) {
+                const int w4 = __ldg(reinterpret_cast<const int *>(p.vals) + q);
+                wv[0] = (AT)(signed char)(w4 & 0xff);
+                wv[1] = (AT)(signed char)((w4 >> 8) & 0xff);
+                wv[2] = (AT)(signed char)((w4 >> 16) & 0xff);
+                wv[3] = (AT)(signed char)((w4 >> 24) & 0xff);
+            } else {
+                const float4 w4 = __ldg(reinterpret_cast<const float4 *>(p.vals) + q);
+                wv[0] = (AT)w4.x; wv[1] = (AT)w4.y; wv[2] = (AT)w4.z; wv[3] = (AT)w4.w;
+            }
+            const uint2 i4 = __ldg(reinterpret_cast<const uint2 *>(p.idx) + q);
+            const int k[4] = {(int)(i4.x & 0xffffu), (int)(i4.x >> 16), (int)(i4.y & 0xffffu), (int)(i4.y >> 16)};
 #pragma unroll
             for (int b = 0; b < NB; ++b)
-                if (b0 + b < p.n) acc[b] += wv * (AT)ld_act(x + (size_t)(b0 + b) * p.k + k);
+                if (b0 + b < p.n) {
+                    const XT *xb = x + (size_t)(b0 + b) * p.k;
+                    XT xv[4];
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) xv[v] = ld_act(xb + k[v]);
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) acc[b] += wv[v] * (AT)xv[v];
+                }
         }
 #pragma unroll
         for (int b = 0; b < NB; ++b)

@@ -1277,23 +1277,36 @@ cadnn_status pack_fc_spmv(cadnn_weights *h, const Src &src)
     std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return row_nnz[a] > row_nnz[b]; });
     h->perm.assign(h->c_pad, -1);
     for (int i = 0; i < d.c_out; ++i) h->perm[i] = order[i];
+    // rows are padded to a multiple of 4 entries (weight 0 at column 0), so that a lane fetches four values and four
+    // column indices with one load each; cnt keeps the real lengths
     h->ptr.assign(h->c_pad + 1, 0);
+    h->cnt.assign(h->c_pad, 0);
     int32_t running = 0;
+    int64_t real = 0;
     for (int r = 0; r < h->c_pad; ++r) {
         h->ptr[r] = running;
         int co = h->perm[r];
         if (co < 0) continue;
+        int len = 0;
         for (int k = 0; k < K; ++k) {
             size_t wi = (size_t)co * K + k;
             if (!src.kept(wi)) continue;
             h->offs.push_back((uint16_t)k);
             if (src.s8) h->vals_q.push_back(src.qval(wi, co));
             else h->vals_f.push_back(src.fval(wi));
-            ++running;
+            ++len;
         }
+        h->cnt[r] = len;
+        real += len;
+        for (; len & 3; ++len) {
+            h->offs.push_back(0);
+            if (src.s8) h->vals_q.push_back(0);
+            else h->vals_f.push_back(0.0f);
+        }
+        running += len;
     }
     h->ptr[h->c_pad] = running;
-    h->nnz = running;
+    h->nnz = real;
     h->fmt = CADNN_FMT_ROW_CSR;
     return CADNN_OK;
 }
@@ -1538,7 +1551,7 @@ cadnn_status cadnn_weights_warp_loads(const cadnn_weights *w, int64_t *loads, in
         int64_t tot = 0;
         for (int c = 0; c < chunks; ++c) {
             if (s.kind == KK_FC_SPMV) {
-                tot += w->ptr[(i + 1) * s.RPW] - w->ptr[i * s.RPW];
+                for (int j = 0; j < s.RPW; ++j) tot += w->cnt[(size_t)i * s.RPW + j];   // real entries, without row padding
             } else {
                 for (int j = 0; j < s.RPW; ++j) tot += w->cnt[(size_t)c * w->c_pad + i * s.RPW + j];
             }
@@ -1570,7 +1583,7 @@ cadnn_status cadnn_weights_unpack(const cadnn_weights *w, float *dense, uint8_t 
         for (int r = 0; r < w->c_pad; ++r) {
             int co = w->perm[r];
             if (co < 0) continue;
-            for (int e = w->ptr[r]; e < w->ptr[r + 1]; ++e) {
+            for (int e = w->ptr[r]; e < w->ptr[r] + w->cnt[r]; ++e) {   // the rest of the row is padding
                 size_t wi = (size_t)co * K + w->offs[e];
                 if (dense) dense[wi] = val(e);
                 if (mask) mask[wi] = 1;
