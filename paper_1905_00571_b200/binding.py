@@ -390,9 +390,16 @@ class _Borrowed:
 
 
 def cadnn_weights_parity_form(w):
+    """The stride-1 form of a stride-2 layer over the parity planes of its input (None if the layer has none):
+    4 c_in input channels (plane-major) for a 3x3 layer, c_in for a 1x1 layer, maps of ceil(h / 2) x ceil(w / 2)."""
     out = ctypes.c_void_p()
     _check(_lib.cadnn_weights_parity_form(w.handle, ctypes.byref(out)), "cadnn_weights_parity_form")
-    return _Borrowed(out, w.desc) if out.value else None
+    if not out.value:
+        return None
+    d = w.desc
+    dc = LayerDesc(4 * d.c_in if d.kh == 3 else d.c_in, d.c_out, d.kh, d.kw, 1, d.pad, d.groups, (d.in_h + 1) // 2,
+                   (d.in_w + 1) // 2, d.batch_hint, d.dtype, d.fmt, d.flags, d.pad_w)
+    return _Borrowed(out, dc)
 
 
 def cadnn_net_layout(net):

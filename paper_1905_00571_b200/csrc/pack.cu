@@ -1419,8 +1419,8 @@ cadnn_status pack_common(const cadnn_layer_desc *desc, const Src &src, cadnn_wei
         // layer is a stride-1 layer over the 4 c_in quarter planes (taps 0 and 1 of a padded 3x3 frame); a 1x1 layer
         // reads the (even, even) plane alone.
         const bool k3 = d.kh == 3 && d.kw == 3 && d.pad == 1 && d.pad_w == 1, k1 = d.kh == 1 && d.kw == 1 && d.pad == 0 && d.pad_w == 0;
-        if (st == CADNN_OK && d.dtype == CADNN_F32 && d.stride == 2 && d.groups == 1 && (k3 || k1) && h->has_planar && h->on_device &&
-            src.f && getenv("CADNN_NO_PARITY_PLANES") == nullptr) {
+        if (st == CADNN_OK && d.dtype == CADNN_F32 && d.stride == 2 && d.groups == 1 && (k3 || k1) && h->has_planar &&
+            (h->on_device || (d.flags & CADNN_PACK_HOST_ONLY)) && src.f && getenv("CADNN_NO_PARITY_PLANES") == nullptr) {
             cadnn_layer_desc dc = d;
             dc.stride = 1;
             dc.in_h = (d.in_h + 1) / 2;

@@ -167,3 +167,33 @@ def test_grouped_format_finds_the_dense_blocks_and_round_trips(B, monkeypatch):
     with pytest.raises(B.CadnnError):
         B.cadnn_pack_q8(B.make_desc(96, 128, 3, 3, 1, 1, 1, 20, 20, 1, "s8", host_only=True, fmt=B.FMT_GROUPED),
                         gen.int8_weights(g, (128, 3, 3, 96)), None)
+
+
+@pytest.mark.parametrize("k,h,w", [(3, 13, 17), (3, 14, 14), (3, 7, 8), (1, 13, 17), (1, 14, 14)])
+def test_parity_form_of_a_stride2_layer_is_the_same_layer(B, k, h, w):
+    """The packer's second form of a stride-2 layer - a stride-1 layer over the input split by row and column parity -
+    computes what the layer computes: the oracle's convolution of the split input with the rearranged weights equals
+    its stride-2 convolution of the input with the original ones."""
+    from oracle import ref
+    g = np.random.default_rng(100 * k + h + w)
+    c_in, c_out, pad = 6, 5, (1 if k == 3 else 0)
+    wt = g.standard_normal((c_out, k, k, c_in)).astype(np.float32)
+    mask = (g.random(wt.shape) < 0.4).astype(np.uint8)
+    d = B.make_desc(c_in, c_out, k, k, 2, pad, 1, h, w, 1, "f32", host_only=True)
+    wh = B.cadnn_pack(d, wt, mask)
+    form = B.cadnn_weights_parity_form(wh)
+    assert form is not None
+    w2, m2 = B.cadnn_weights_unpack(form)
+    assert int(m2.sum()) == int(mask.sum())
+    x = g.standard_normal((2, h, w, c_in)).astype(np.float32)
+    h2, wd2 = (h + 1) // 2, (w + 1) // 2
+    planes = np.zeros((2, h2, wd2, (4 if k == 3 else 1) * c_in), np.float32)
+    for py in range(2 if k == 3 else 1):
+        for px in range(2 if k == 3 else 1):
+            sub = x[:, py::2, px::2, :]
+            par = py * 2 + px
+            planes[:, :sub.shape[1], :sub.shape[2], par * c_in:(par + 1) * c_in] = sub
+    want = ref.conv2d_f32(x, wt, mask, 2, pad)
+    got = ref.conv2d_f32(planes, w2, m2, 1, pad)
+    assert got.shape == want.shape
+    np.testing.assert_allclose(got, want, rtol=1e-6, atol=1e-6)
