@@ -303,9 +303,9 @@ def run_ours(args):
               "families": {k: {"ms": v["ms"], "launches": v["launches"], "t_roof_us": v["t_roof_us"]} for k, v in fam.items()}}
 
     # the throughput regime beside the latency-limited batch-1 number: kernel-only fraction of the pruned 3x3
-    # layers at batch 32 (schedules from the packer's time model; per-layer times as above)
+    # layers at batch 32 (schedules timed at pack time like the batch-1 ones; per-layer times as above)
     if rank == 0 and world == 1 and args.workload == "resnet50" and not args.no_batch32:
-        pm32 = PackedModel(model, 32, dev, autotune=False)
+        pm32 = PackedModel(model, 32, dev, autotune=not args.no_autotune)
         x32 = torch.from_numpy(models.make_input(model, 32, seed=7)).to(dev)
         y32 = pm32.new_output()
         pm32.forward(x32, y32)

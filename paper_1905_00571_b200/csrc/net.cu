@@ -7,6 +7,7 @@
 #include <cstdlib>
 #include <new>
 #include <vector>
+#include <cstdio>
 #include "cadnn_internal.h"
 
 struct SlotInfo {
@@ -445,11 +446,18 @@ cadnn_status cadnn_net_create(const cadnn_op *ops, int n_ops, int n, int h, int 
             for (int i = 0; i < n_ops; ++i) {
                 const cadnn_weights *w = ops[i].kind == CADNN_OP_CONV ? ops[i].w : nullptr;
                 if (!w || !w->has_planar) continue;
-                const float tp = (w->has_ps && w->use_ps) ? w->ps_us : w->pl_us;
+                float tp = (w->has_ps && w->use_ps) ? w->ps_us : w->pl_us;
+                if (w->half) {   // a stride-2 layer would run in its parity-plane form where that measured faster
+                    const float th = (w->half->has_ps && w->half->use_ps) ? w->half->ps_us : w->half->pl_us;
+                    if (th > 0.0f && (tp <= 0.0f || th < tp)) tp = th;
+                }
                 if (tp <= 0.0f || w->nhwc_us <= 0.0f) { all = false; break; }
                 t_planar += tp;
                 t_nhwc += w->nhwc_us;
             }
+            if (getenv("CADNN_VERBOSE"))
+                fprintf(stderr, "cadnn_net_create: sparse convs timed at pack time: planar %.1f us, NHWC %.1f us%s\n", t_planar, t_nhwc,
+                        all ? "" : " (incomplete)");
             if (all && t_nhwc > 0.0 && t_planar > t_nhwc) planar = false;
         }
         net->planar = planar;
