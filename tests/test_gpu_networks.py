@@ -131,3 +131,33 @@ def test_mobilenet_v2_runs_channel_planar(image, batch, monkeypatch):
         _check_logits(y.cpu().numpy(), want)
         outs.append(y.cpu().numpy())
     assert_close_f32(outs[0], outs[1], "planar vs NHWC", floor=NET_FLOOR)
+
+
+@pytest.mark.parametrize("name", ["resnet50", "mobilenet_v2", "resnet50_int8"])
+def test_general_graph_scheduler_on_residual_networks(name, monkeypatch):
+    """The lane scheduler that captures independent branches as parallel graph branches (the default for networks with
+    concatenations) forced on residual networks: three replays with the input buffer overwritten in between - a missing
+    dependency would let a layer read a tensor of the previous replay - against the oracle."""
+    from paper_1905_00571_b200.network import PackedModel
+    monkeypatch.setenv("CADNN_GRAPH_LANES", "1")
+    monkeypatch.setenv("CADNN_FORCE_PARITY_PLANES", "1")
+    if name == "resnet50":
+        m = models.resnet50(width=0.25, image=64, classes=100)
+    elif name == "mobilenet_v2":
+        m = models.mobilenet_v2(width=0.5, image=64, classes=100)
+    else:
+        m = models.resnet50_int8(width=0.25, image=64, classes=100)
+    pm = PackedModel(m, 2, DEV)
+    y = pm.new_output()
+    xd = None
+    for seed in (11, 12, 13):
+        x = models.make_input(m, 2, seed=seed)
+        if xd is None:
+            xd = torch.from_numpy(x).to(DEV)
+        else:
+            xd.copy_(torch.from_numpy(x))
+        pm.forward(xd, y)
+        torch.cuda.synchronize()
+        want, _ = oracle_forward.forward(m, x)
+        got = y.cpu().numpy()
+        _check_logits(got, want)   # (the int8 network's pooled vector and classifier are float: close, not bit-equal)
